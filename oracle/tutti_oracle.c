@@ -1,0 +1,376 @@
+/*
+ * CPU oracle for the per-layer KV restore / save path and its descriptor build.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, obviously-correct
+ * statement of what the path computes.  It shares no code, header, table or
+ * helper with the CUDA library and must never be called from the product path;
+ * only the tests, the smoke check and the bench's CPU-baseline leg use it.
+ *
+ * What it states (paper sections in brackets):
+ *   orc_obj_layout     object id -> (device, byte offset): a "GPU file" holds
+ *                      2 x L objects, one key and one value object per layer;
+ *                      files are spread round-robin over the storage devices
+ *                      [Section 3.1, "Scalable GPU File Pool"].
+ *   orc_restore_layer  layer-wise Retrieve: for every cached token of every
+ *   orc_save_layer     request, the token's K and V bytes move between the
+ *                      contiguous object and the paged block the block table
+ *                      names; layer-wise Store is the same map reversed
+ *                      [Section 2.1 paged KV blocks; Section 3.1 layer-wise
+ *                      batched Store/Retrieve; Section 3.4 retrieve_layer /
+ *                      store_layer].
+ *   orc_build          the batch of I/O contexts for one layer: (file offset,
+ *                      length, scatter-gather list) per contiguous run, 16-byte
+ *                      SGL entries (address 8 B, length 4 B, identifier 4 B),
+ *                      packed into IOCBs of a fixed number of contexts
+ *                      [Section 3.1 "P2P Memory Mapping Table"; Section 3.2].
+ *   orc_exec           what executing such descriptors means (the transfer a
+ *                      device would perform for each context).
+ *
+ * The paper gives no sorting/coalescing rule (only the motivation that small
+ * scattered requests waste bandwidth, Section 2.3/2.4); the rule used here is
+ * the reading recorded in the design notes: order by (device, offset), merge
+ * exactly byte-adjacent neighbours on one device, stable on (request, chunk,
+ * K-before-V).
+ *
+ * Parity pins (tests/test_oracle_*.py): brute force on tiny pools against an
+ * independent Python byte loop, array-shaped (numpy advanced indexing)
+ * restatement, round-trip identity, untouched-byte checks, descriptor
+ * prefix-sum / coverage invariants, exec(build) == restore, and the counts the
+ * paper prints.  No function here is "parity unpinned".
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_OK 0
+#define ORC_EINVAL (-1)
+#define ORC_ENOSPC (-2)
+
+#define ORC_FILE_MAJOR 0
+#define ORC_LAYER_MAJOR 1
+
+#define ORC_OP_READ 0  /* object store -> paged pool (restore) */
+#define ORC_OP_WRITE 1 /* paged pool -> object store (save)    */
+
+typedef struct {
+    uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
+    uint32_t block_tokens, obj_tokens, n_devices, layout;
+    uint64_t n_slots;
+} orc_geom;
+
+typedef struct {
+    uint64_t token_bytes;   /* one token's K (or V) of one layer            */
+    uint64_t block_bytes;   /* one paged block's K (or V) of one layer      */
+    uint64_t obj_kv_bytes;  /* K half (= V half) of one object              */
+    uint64_t obj_bytes;     /* K half followed by V half                    */
+    uint64_t blocks_per_obj;
+    uint64_t n_slots_local; /* object slots per device                      */
+    uint64_t stride_kv, stride_layer, stride_slot;
+    uint64_t dev_bytes;     /* bytes of store needed on each device         */
+} orc_layout;
+
+typedef struct {
+    uint64_t src_off; /* object-side byte offset on device `dev`           */
+    uint64_t len;
+    uint32_t sgl_first, sgl_count;
+    uint32_t dev;
+    uint16_t opcode, layer;
+} orc_sqe;
+
+typedef struct {
+    uint64_t addr; /* pool-side address */
+    uint32_t len;
+    uint32_t id;   /* pool block id     */
+} orc_sgl;
+
+/* Section 3.1: object = K half then V half of obj_tokens tokens of one layer. */
+int orc_obj_layout(const orc_geom *g, orc_layout *o)
+{
+    if (!g || !o) return ORC_EINVAL;
+    if (g->n_layers == 0 || g->n_kv_heads == 0 || g->head_dim == 0 || g->elem_bytes == 0 ||
+        g->block_tokens == 0 || g->obj_tokens == 0 || g->n_devices == 0)
+        return ORC_EINVAL;
+    if (g->obj_tokens % g->block_tokens != 0) return ORC_EINVAL;
+    if (g->layout != ORC_FILE_MAJOR && g->layout != ORC_LAYER_MAJOR) return ORC_EINVAL;
+    o->token_bytes = (uint64_t)g->n_kv_heads * g->head_dim * g->elem_bytes;
+    o->block_bytes = o->token_bytes * g->block_tokens;
+    o->obj_kv_bytes = o->token_bytes * g->obj_tokens;
+    o->obj_bytes = 2 * o->obj_kv_bytes;
+    o->blocks_per_obj = g->obj_tokens / g->block_tokens;
+    o->n_slots_local = (g->n_slots + g->n_devices - 1) / g->n_devices;
+    o->stride_kv = o->obj_kv_bytes;
+    if (g->layout == ORC_FILE_MAJOR) {
+        /* a file = all layers of one chunk, files one after another */
+        o->stride_layer = o->obj_bytes;
+        o->stride_slot = (uint64_t)g->n_layers * o->obj_bytes;
+    } else {
+        /* all objects of a layer together, layers one after another */
+        o->stride_slot = o->obj_bytes;
+        o->stride_layer = o->n_slots_local * o->obj_bytes;
+    }
+    o->dev_bytes = o->n_slots_local * g->n_layers * o->obj_bytes;
+    return ORC_OK;
+}
+
+/* Device and byte offset of the K (kv=0) or V (kv=1) half of object `slot`. */
+static void object_location(const orc_geom *g, const orc_layout *lo, uint64_t slot,
+                            uint32_t layer, uint32_t kv, uint32_t *dev, uint64_t *off)
+{
+    *dev = (uint32_t)(slot % g->n_devices); /* round-robin over devices */
+    *off = (slot / g->n_devices) * lo->stride_slot + (uint64_t)layer * lo->stride_layer +
+           (uint64_t)kv * lo->stride_kv;
+}
+
+static int check_batch(const orc_geom *g, uint32_t layer, uint32_t n_req,
+                       const uint32_t *hit_tokens, const uint32_t *obj_start,
+                       const uint32_t *blk_start)
+{
+    if (layer >= g->n_layers) return ORC_EINVAL;
+    for (uint32_t r = 0; r < n_req; ++r) {
+        uint64_t hit = hit_tokens[r];
+        if (hit % g->block_tokens != 0) return ORC_EINVAL;
+        uint64_t need_obj = (hit + g->obj_tokens - 1) / g->obj_tokens;
+        uint64_t need_blk = hit / g->block_tokens;
+        if ((uint64_t)obj_start[r + 1] - obj_start[r] < need_obj) return ORC_EINVAL;
+        if ((uint64_t)blk_start[r + 1] - blk_start[r] < need_blk) return ORC_EINVAL;
+    }
+    return ORC_OK;
+}
+
+/*
+ * Location of token t of request r: where it sits in the object store and in
+ * which pool block / token row.  This is the whole map; restore and save only
+ * differ in the direction of the copy.
+ */
+static int token_location(const orc_geom *g, const orc_layout *lo, uint32_t layer,
+                          const uint32_t *obj_start, const uint32_t *obj_slot,
+                          const uint32_t *blk_start, const int32_t *block_ids, uint32_t r,
+                          uint64_t t, uint32_t kv, uint32_t *dev, uint64_t *store_off,
+                          int64_t *block, uint64_t *row_off)
+{
+    uint64_t slot = obj_slot[obj_start[r] + t / g->obj_tokens];
+    uint64_t off;
+    if (slot >= g->n_slots) return ORC_EINVAL;
+    object_location(g, lo, slot, layer, kv, dev, &off);
+    *store_off = off + (t % g->obj_tokens) * lo->token_bytes;
+    *block = block_ids[blk_start[r] + t / g->block_tokens];
+    *row_off = (t % g->block_tokens) * lo->token_bytes;
+    return ORC_OK;
+}
+
+int orc_token_location(const orc_geom *g, uint32_t layer, const uint32_t *obj_start,
+                       const uint32_t *obj_slot, const uint32_t *blk_start,
+                       const int32_t *block_ids, uint32_t r, uint64_t t, uint32_t kv,
+                       uint32_t *dev, uint64_t *store_off, int64_t *block, uint64_t *row_off)
+{
+    orc_layout lo;
+    int rc = orc_obj_layout(g, &lo);
+    if (rc) return rc;
+    return token_location(g, &lo, layer, obj_start, obj_slot, blk_start, block_ids, r, t, kv,
+                          dev, store_off, block, row_off);
+}
+
+static int move_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
+                      const uint32_t *hit_tokens, const uint32_t *obj_start,
+                      const uint32_t *obj_slot, const uint32_t *blk_start,
+                      const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
+                      uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks, int to_pool)
+{
+    orc_layout lo;
+    int rc = orc_obj_layout(g, &lo);
+    if (rc) return rc;
+    rc = check_batch(g, layer, n_req, hit_tokens, obj_start, blk_start);
+    if (rc) return rc;
+    for (uint32_t r = 0; r < n_req; ++r) {
+        for (uint64_t t = 0; t < hit_tokens[r]; ++t) {
+            for (uint32_t kv = 0; kv < 2; ++kv) {
+                uint32_t dev;
+                uint64_t soff, roff;
+                int64_t blk;
+                rc = token_location(g, &lo, layer, obj_start, obj_slot, blk_start, block_ids, r,
+                                    t, kv, &dev, &soff, &blk, &roff);
+                if (rc) return rc;
+                if (blk < 0 || (uint64_t)blk >= n_pool_blocks) return ORC_EINVAL;
+                uint8_t *in_pool = (kv ? pool_v : pool_k) + (uint64_t)blk * block_stride + roff;
+                uint8_t *in_store = store[dev] + soff;
+                if (to_pool)
+                    memcpy(in_pool, in_store, lo.token_bytes);
+                else
+                    memcpy(in_store, in_pool, lo.token_bytes);
+            }
+        }
+    }
+    return ORC_OK;
+}
+
+/* Layer-wise Retrieve (Section 3.1 / 3.4): object store -> paged pool. */
+int orc_restore_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
+                      const uint32_t *hit_tokens, const uint32_t *obj_start,
+                      const uint32_t *obj_slot, const uint32_t *blk_start,
+                      const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
+                      uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks)
+{
+    return move_layer(g, layer, n_req, hit_tokens, obj_start, obj_slot, blk_start, block_ids,
+                      store, pool_k, pool_v, block_stride, n_pool_blocks, 1);
+}
+
+/* Layer-wise Store (Section 3.1 / 3.4): paged pool -> object store. */
+int orc_save_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
+                   const uint32_t *hit_tokens, const uint32_t *obj_start,
+                   const uint32_t *obj_slot, const uint32_t *blk_start,
+                   const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
+                   uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks)
+{
+    return move_layer(g, layer, n_req, hit_tokens, obj_start, obj_slot, blk_start, block_ids,
+                      store, pool_k, pool_v, block_stride, n_pool_blocks, 0);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Descriptor build, step by step (sequential).                               */
+/* ------------------------------------------------------------------------- */
+
+typedef struct {
+    uint32_t dev;
+    uint64_t src_off;
+    uint64_t len;
+    uint32_t n_blk;
+    uint32_t r, c, kv;
+    uint32_t seq; /* position in (r, c, kv) generation order */
+} item_t;
+
+static int item_cmp(const void *pa, const void *pb)
+{
+    const item_t *a = (const item_t *)pa, *b = (const item_t *)pb;
+    if (a->dev != b->dev) return a->dev < b->dev ? -1 : 1;
+    if (a->src_off != b->src_off) return a->src_off < b->src_off ? -1 : 1;
+    /* equal keys keep generation order: this makes qsort behave as a stable sort */
+    if (a->seq != b->seq) return a->seq < b->seq ? -1 : 1;
+    return 0;
+}
+
+/*
+ * Build one layer's descriptors.
+ *   sqes[max_sqe], sgl[max_sgl], num_ioctx[max_iocb] are outputs; *n_sqe, *n_sgl,
+ *   *n_iocb the counts produced.  SQE k belongs to IOCB k / capacity at position
+ *   k % capacity.  n_iocb = ceil(n_sqe / capacity), at least 1 (an empty batch
+ *   yields one IOCB with num_ioctx = 0).
+ */
+int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req,
+              const uint32_t *hit_tokens, const uint32_t *obj_start, const uint32_t *obj_slot,
+              const uint32_t *blk_start, const int32_t *block_ids, uint64_t k_base_addr,
+              uint64_t v_base_addr, uint64_t block_stride, uint32_t capacity, orc_sqe *sqes,
+              uint32_t max_sqe, orc_sgl *sgl, uint32_t max_sgl, uint32_t *num_ioctx,
+              uint32_t max_iocb, uint32_t *n_sqe, uint32_t *n_sgl, uint32_t *n_iocb)
+{
+    orc_layout lo;
+    int rc = orc_obj_layout(g, &lo);
+    if (rc) return rc;
+    rc = check_batch(g, layer, n_req, hit_tokens, obj_start, blk_start);
+    if (rc) return rc;
+    if (capacity == 0 || (opcode != ORC_OP_READ && opcode != ORC_OP_WRITE)) return ORC_EINVAL;
+
+    /* step 1: items, one per hit object and per K / V half */
+    uint64_t n_items = 0;
+    for (uint32_t r = 0; r < n_req; ++r)
+        n_items += 2 * (((uint64_t)hit_tokens[r] + g->obj_tokens - 1) / g->obj_tokens);
+    item_t *items = (item_t *)malloc((n_items ? n_items : 1) * sizeof(item_t));
+    if (!items) return ORC_ENOSPC;
+    uint32_t q = 0;
+    for (uint32_t r = 0; r < n_req; ++r) {
+        uint64_t hit = hit_tokens[r];
+        uint64_t n_chunks = (hit + g->obj_tokens - 1) / g->obj_tokens;
+        for (uint64_t c = 0; c < n_chunks; ++c) {
+            uint64_t valid = hit - c * g->obj_tokens;
+            if (valid > g->obj_tokens) valid = g->obj_tokens;
+            uint64_t slot = obj_slot[obj_start[r] + c];
+            if (slot >= g->n_slots) { free(items); return ORC_EINVAL; }
+            for (uint32_t kv = 0; kv < 2; ++kv) {
+                item_t *it = &items[q];
+                object_location(g, &lo, slot, layer, kv, &it->dev, &it->src_off);
+                it->len = valid * lo.token_bytes;
+                it->n_blk = (uint32_t)(valid / g->block_tokens);
+                it->r = r; it->c = (uint32_t)c; it->kv = kv; it->seq = q;
+                ++q;
+            }
+        }
+    }
+
+    /* step 2: order by (device, offset), stable */
+    qsort(items, n_items, sizeof(item_t), item_cmp);
+
+    /* step 3 + 4: sweep, merging exactly adjacent neighbours; emit SGL entries */
+    uint32_t ns = 0, ne = 0;
+    for (uint64_t i = 0; i < n_items; ++i) {
+        const item_t *it = &items[i];
+        int fresh = (i == 0) || items[i - 1].dev != it->dev ||
+                    items[i - 1].src_off + items[i - 1].len != it->src_off;
+        if (fresh) {
+            if (ns >= max_sqe) { free(items); return ORC_ENOSPC; }
+            orc_sqe *s = &sqes[ns++];
+            s->src_off = it->src_off;
+            s->len = 0;
+            s->sgl_first = ne;
+            s->sgl_count = 0;
+            s->dev = it->dev;
+            s->opcode = (uint16_t)opcode;
+            s->layer = (uint16_t)layer;
+        }
+        orc_sqe *s = &sqes[ns - 1];
+        s->len += it->len;
+        s->sgl_count += it->n_blk;
+        for (uint32_t j = 0; j < it->n_blk; ++j) {
+            if (ne >= max_sgl) { free(items); return ORC_ENOSPC; }
+            int32_t id = block_ids[blk_start[it->r] + (uint64_t)it->c * lo.blocks_per_obj + j];
+            if (id < 0) { free(items); return ORC_EINVAL; }
+            sgl[ne].addr = (it->kv ? v_base_addr : k_base_addr) + (uint64_t)id * block_stride;
+            sgl[ne].len = (uint32_t)lo.block_bytes;
+            sgl[ne].id = (uint32_t)id;
+            ++ne;
+        }
+    }
+    free(items);
+
+    /* step 5: pack into IOCBs of `capacity` contexts */
+    uint32_t nb = (ns + capacity - 1) / capacity;
+    if (nb == 0) nb = 1;
+    if (nb > max_iocb) return ORC_ENOSPC;
+    for (uint32_t b = 0; b < nb; ++b) {
+        uint32_t left = ns - (ns < b * capacity ? ns : b * capacity);
+        num_ioctx[b] = left < capacity ? left : capacity;
+    }
+    *n_sqe = ns;
+    *n_sgl = ne;
+    *n_iocb = nb;
+    return ORC_OK;
+}
+
+/*
+ * Execute descriptors: for each context, walk its SGL entries with a cursor
+ * on the object side.  READ moves object bytes to the entry's address, WRITE
+ * the other way.  Pool addresses are translated to the host copy of the pool
+ * by  host = pool_host + (addr - pool_base_addr).
+ */
+int orc_exec(const orc_sqe *sqes, uint32_t n_sqe, const orc_sgl *sgl, uint32_t n_sgl,
+             uint8_t *const *store, const uint64_t *store_bytes, uint32_t n_devices,
+             uint8_t *pool_host, uint64_t pool_base_addr, uint64_t pool_bytes)
+{
+    for (uint32_t k = 0; k < n_sqe; ++k) {
+        const orc_sqe *s = &sqes[k];
+        if (s->dev >= n_devices) return ORC_EINVAL;
+        if ((uint64_t)s->sgl_first + s->sgl_count > n_sgl) return ORC_EINVAL;
+        uint64_t cursor = s->src_off;
+        for (uint32_t e = s->sgl_first; e < s->sgl_first + s->sgl_count; ++e) {
+            if (sgl[e].addr < pool_base_addr) return ORC_EINVAL;
+            uint64_t poff = sgl[e].addr - pool_base_addr;
+            if (poff + sgl[e].len > pool_bytes) return ORC_EINVAL;
+            if (cursor + sgl[e].len > store_bytes[s->dev]) return ORC_EINVAL;
+            if (s->opcode == ORC_OP_READ)
+                memcpy(pool_host + poff, store[s->dev] + cursor, sgl[e].len);
+            else
+                memcpy(store[s->dev] + cursor, pool_host + poff, sgl[e].len);
+            cursor += sgl[e].len;
+        }
+        if (cursor - s->src_off != s->len) return ORC_EINVAL;
+    }
+    return ORC_OK;
+}

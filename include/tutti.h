@@ -1,0 +1,326 @@
+/*
+ * tutti.h — C ABI of the B200 (sm_100a) KV-cache object-store hot path.
+ *
+ * The library moves prefix KV cache, one layer at a time, between contiguous
+ * per-layer KV objects (the storage tier; here an object store in HBM or in
+ * pinned host memory read zero-copy) and a fragmented, block-table-indexed paged
+ * KV pool in HBM, and builds the I/O submission descriptors for that transfer on
+ * the GPU, into a GPU-resident submission/completion ring.  The host does O(1)
+ * work per layer and no per-block work (paper Section 3.1, last paragraph).
+ *
+ * Conventions
+ *   - Every call returns TUTTI_OK (0) or a negative TUTTI_E* code.  Device-side
+ *     problems never trap: they arrive as `status` of the completion entry.
+ *   - "device pointer" = address valid in kernels on the context's GPU (HBM, or
+ *     the device alias of pinned mapped host memory).  "host pointer" = ordinary
+ *     host memory.  Streams are passed as `void*` holding a CUstream/cudaStream_t
+ *     (NULL = the legacy default stream).
+ *   - Nothing on the per-layer path (build / restore / save / poll) allocates
+ *     memory or synchronises the host with the device (Section 3.2, "Zero-Copy
+ *     Ring Buffers": no runtime allocation, copying or CPU-GPU synchronisation).
+ *   - One ring is driven by one host thread at a time (no internal locking).
+ */
+#ifndef TUTTI_H_
+#define TUTTI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TUTTI_OK 0
+#define TUTTI_EINVAL (-1)    /* bad argument or broken precondition                      */
+#define TUTTI_ENOMEM (-2)    /* allocation failed at create time                         */
+#define TUTTI_EAGAIN (-3)    /* ring / SGL arena full, or completion not there yet       */
+#define TUTTI_ETIMEDOUT (-4) /* a bounded device-side wait ran out                       */
+#define TUTTI_EFAULT (-5)    /* a block id or object slot points outside its region      */
+#define TUTTI_ECUDA (-6)     /* a CUDA call failed; see tutti_last_cuda_error()          */
+
+#define TUTTI_LAYOUT_FILE_MAJOR 0  /* a file = all layers of one chunk; files back to back */
+#define TUTTI_LAYOUT_LAYER_MAJOR 1 /* all objects of a layer together; layers back to back */
+
+#define TUTTI_OP_READ 0  /* object store -> paged pool  (restore / Retrieve) */
+#define TUTTI_OP_WRITE 1 /* paged pool  -> object store (save / Store)       */
+
+#define TUTTI_STORE_HBM 0
+#define TUTTI_STORE_HOST_PINNED 1
+
+#define TUTTI_MAX_DEVICES 8
+#define TUTTI_DEFAULT_IOCTX_PER_IOCB 2048 /* Section 3.2: one IOCB holds 2048 I/O contexts */
+
+/* Options for tutti_set_option(). */
+#define TUTTI_OPT_COPY_ENGINE 1 /* 0 auto, 1 vector load/store kernel, 2 bulk-async (TMA) kernel */
+#define TUTTI_OPT_WAIT_NS 2     /* budget of the device-side wait for an IOCB to become ready    */
+#define TUTTI_OPT_CTAS_PER_SM 3 /* resident CTAs per SM of the load/store kernel (grid mode)     */
+#define TUTTI_OPT_BULK_WARPS 4  /* copy warps per CTA of the bulk-async kernel                   */
+#define TUTTI_OPT_BULK_STAGES 5 /* shared-memory stages per copy warp of the bulk-async kernel   */
+#define TUTTI_OPT_CLAIM_CHUNKS 6 /* chunks (32 KiB each) taken per work claim                    */
+
+/*
+ * Geometry of the KV cache and of the object store (Section 3.1, "Scalable GPU
+ * File Pool").  An object holds obj_tokens tokens of one layer: its K half then
+ * its V half, each [obj_tokens][n_kv_heads][head_dim] elements; the paper's
+ * one-object-per-block case is obj_tokens == block_tokens.  Object slot s lives
+ * on storage device s mod n_devices (round-robin placement).
+ */
+typedef struct tutti_geom {
+    uint32_t n_layers;
+    uint32_t n_kv_heads;
+    uint32_t head_dim;
+    uint32_t elem_bytes;
+    uint32_t block_tokens; /* tokens per paged KV block                      */
+    uint32_t obj_tokens;   /* tokens per object; a multiple of block_tokens  */
+    uint32_t n_devices;    /* storage devices, 1..TUTTI_MAX_DEVICES          */
+    uint32_t layout;       /* TUTTI_LAYOUT_*                                 */
+    uint64_t n_slots;      /* object slots in the store, over all devices    */
+} tutti_geom_t;
+
+/* Derived sizes and strides.  Byte offset of the K (kv=0) / V (kv=1) half of slot s,
+ * layer l, on device s mod n_devices:
+ *     (s / n_devices) * stride_slot + l * stride_layer + kv * stride_kv          */
+typedef struct tutti_layout {
+    uint64_t token_bytes;   /* K (or V) of one token of one layer              */
+    uint64_t block_bytes;   /* K (or V) of one paged block of one layer        */
+    uint64_t obj_kv_bytes;  /* one half of an object                           */
+    uint64_t obj_bytes;     /* K half + V half                                 */
+    uint64_t blocks_per_obj;
+    uint64_t n_slots_local; /* slots per device = ceil(n_slots / n_devices)    */
+    uint64_t stride_kv;
+    uint64_t stride_layer;
+    uint64_t stride_slot;
+    uint64_t dev_bytes;     /* bytes each device's store region must provide   */
+} tutti_layout_t;
+
+/*
+ * One batch of prefix hits.  All five arrays are DEVICE pointers owned by the
+ * caller; they must stay valid and unchanged until every IOCB built from them has
+ * been polled.  CSR form: request r owns objects obj_slot[obj_start[r] ..
+ * obj_start[r+1]) in chunk order and pool blocks block_ids[blk_start[r] ..
+ * blk_start[r+1]) in logical block order.  hit_tokens[r] must be a multiple of
+ * block_tokens; row r must list at least ceil(hit/obj_tokens) objects and
+ * hit/block_tokens blocks (extra entries are never read).
+ * The scalar fields are host-known sizes: n_obj = obj_start[n_req], n_blk =
+ * blk_start[n_req].
+ * plan_epoch: 0 = the sorted/coalesced plan is recomputed on every build.  A
+ * non-zero value promises that a batch with the same epoch, pointers and sizes has
+ * the same contents, so the plan of the previous build on the ring is reused (it
+ * does not depend on the layer) and only the per-layer part is redone.
+ */
+typedef struct tutti_batch {
+    uint32_t n_req;
+    uint32_t n_obj;
+    uint32_t n_blk;
+    uint32_t plan_epoch;
+    const uint32_t *hit_tokens; /* [n_req]     */
+    const uint32_t *obj_start;  /* [n_req + 1] */
+    const uint32_t *obj_slot;   /* [n_obj]     */
+    const uint32_t *blk_start;  /* [n_req + 1] */
+    const int32_t *block_ids;   /* [n_blk]     */
+} tutti_batch_t;
+
+/* I/O context (Section 3.2: "SGL address, GPU file offset, and length"): one
+ * contiguous byte range of one storage device and the scatter-gather entries that
+ * cover it.  sgl_first counts from the first entry of the build the context
+ * belongs to. */
+typedef struct tutti_sqe {
+    uint64_t src_off; /* object-side byte offset on device `dev` (both directions) */
+    uint64_t len;
+    uint32_t sgl_first;
+    uint32_t sgl_count;
+    uint32_t dev;
+    uint16_t opcode;
+    uint16_t layer;
+} tutti_sqe_t;
+
+/* Scatter-gather entry, 16 bytes (Section 3.1: address 8 B, length 4 B, identifier
+ * 4 B).  addr is the pool-side device address, id the pool block id. */
+typedef struct tutti_sgl {
+    uint64_t addr;
+    uint32_t len;
+    uint32_t id;
+} tutti_sgl_t;
+
+/* Completion entry: the IOCB index the kernel writes to the CQ (Section 3.2, step
+ * 3), with a status and the bytes it moved. */
+typedef struct tutti_cqe {
+    uint32_t iocb_idx;
+    int32_t status;
+    uint64_t bytes;
+} tutti_cqe_t;
+
+/* Read-back of one IOCB header (inspection / tests). */
+typedef struct tutti_iocb_info {
+    uint32_t iocb_idx;
+    uint32_t ready;         /* 1 once its descriptors are published           */
+    uint32_t num_ioctx;
+    uint32_t opcode;
+    uint32_t layer;
+    int32_t status;
+    uint32_t sgl_base;      /* arena index of the build's first entry         */
+    uint32_t entry_first;   /* first entry of this IOCB, relative to sgl_base */
+    uint32_t total_entries;
+    uint32_t entry_len;     /* common entry length, 0 if lengths differ       */
+    uint64_t bytes;
+} tutti_iocb_info_t;
+
+typedef struct tutti_ctx tutti_ctx_t;
+typedef struct tutti_ring tutti_ring_t;
+
+/* ------------------------------------------------------------------------- */
+/* The five calls of the path                                                 */
+/* ------------------------------------------------------------------------- */
+
+/*
+ * Object id -> (device, byte offset, length): sizes and strides of the object
+ * store for a geometry (Section 3.1: a GPU file is 2 x L objects, one key and one
+ * value object per layer; files are placed round-robin across devices).
+ * Pure host function; both pointers are host memory.  TUTTI_EINVAL if a field is
+ * zero, obj_tokens is not a multiple of block_tokens, token_bytes is not a multiple
+ * of 16, n_devices > TUTTI_MAX_DEVICES or the layout is unknown.
+ */
+int tutti_obj_layout(const tutti_geom_t *geom, tutti_layout_t *out);
+
+/*
+ * Build one layer's I/O contexts on the GPU (Section 3.1 "block lookup and P2P
+ * table lookup to generate a batch of lightweight GPU I/O contexts"; Section 3.2
+ * step 2, get_iocb).  GPU threads turn (object slot, layer) into (device, offset,
+ * length) items, order them by (device, offset), merge exactly byte-adjacent
+ * neighbours into one context, emit one 16-byte SGL entry per pool block in
+ * object byte order, pack contexts into IOCBs of ioctx_per_iocb entries and
+ * publish them in the ring.
+ *   batch        host pointer to the struct; its arrays are device pointers.
+ *   first_iocb,  host out: indices of the reserved IOCBs, known without waiting
+ *   n_iocb       for the GPU: ceil(2*n_obj / ioctx_per_iocb), at least 1.  IOCBs
+ *                the build does not need are published with num_ioctx = 0.
+ * Asynchronous on `stream`.  TUTTI_EAGAIN if the ring or the SGL arena has no
+ * room (poll completed IOCBs first); TUTTI_EINVAL for layer >= n_layers, unknown
+ * opcode, unregistered pool layer / store device, or a batch larger than the ring
+ * was created for.  Bad batch contents (misaligned hit length, short rows, slot or
+ * block id out of range) are found by the kernel: the IOCBs then carry that status,
+ * move no bytes and complete with it.
+ */
+int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch,
+                     uint32_t layer, uint32_t opcode, void *stream, uint32_t *first_iocb,
+                     uint32_t *n_iocb);
+
+/*
+ * Layer-wise Retrieve (Section 3.1; retrieve_layer of Section 3.4; issue_io of
+ * Section 3.2 step 3): execute the READ IOCBs [first_iocb, first_iocb + n_iocb):
+ * for every context, the bytes at its object-store range are scattered to the
+ * pool addresses of its SGL entries.  sm_count = 0 runs on all SMs; otherwise
+ * that many persistent CTAs (one per SM) claim the work, for use beside compute
+ * kernels (Section 3.2 "SM Partitioning"; Section 3.3).  When the last byte of an
+ * IOCB has landed, the kernel writes its index to the completion queue.
+ * Asynchronous on `stream`; must be ordered after the build (same stream or an
+ * event).  TUTTI_EINVAL if an index was not reserved, or has the other opcode.
+ */
+int tutti_kv_restore_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t first_iocb,
+                           uint32_t n_iocb, uint32_t sm_count, void *stream);
+
+/*
+ * Layer-wise Store (store_layer of Section 3.4): the same transfer in the other
+ * direction for WRITE IOCBs: pool blocks are gathered into the object-store
+ * ranges.  Saving and restoring the same objects concurrently is the caller's
+ * race (the paper orders them with CUDA events, Section 3.2 step 2).
+ */
+int tutti_kv_save_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t first_iocb,
+                        uint32_t n_iocb, uint32_t sm_count, void *stream);
+
+/*
+ * wait_cqe (Section 3.2 step 4): look in the completion queue for one IOCB index.
+ * timeout_ns = 0 never blocks.  Returns TUTTI_OK and fills *out (host pointer)
+ * when the IOCB has completed — out->status carries a device-side error, if any;
+ * TUTTI_EAGAIN when it has not completed within the timeout; TUTTI_EINVAL when
+ * the index is not a live reservation.  A successful poll releases the IOCB (and,
+ * once all IOCBs of its build are polled, the build's SGL entries) for reuse.
+ */
+int tutti_ring_poll(tutti_ring_t *ring, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns);
+
+/* ------------------------------------------------------------------------- */
+/* Lifecycle                                                                  */
+/* ------------------------------------------------------------------------- */
+
+/* Create a context for `geom` on CUDA device `device` (host call; allocates the
+ * small registration tables).  TUTTI_ECUDA if no usable device. */
+int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out);
+int tutti_ctx_destroy(tutti_ctx_t *ctx);
+
+/* Register layer `layer` of the pre-allocated paged KV pool (Section 3.4: "register
+ * the pre-allocated KV memory block pool").  Block b's K bytes start at k_base +
+ * b * block_stride, its V bytes at v_base + b * block_stride (device pointers,
+ * 16-byte aligned, block_stride a multiple of 16 and >= block_bytes).  Layers may
+ * share memory.  The caller keeps ownership. */
+int tutti_pool_register(tutti_ctx_t *ctx, uint32_t layer, void *k_base, void *v_base,
+                        uint64_t block_stride, uint64_t n_blocks);
+
+/* Register the region of storage device `dev`: `base` is a device pointer (HBM,
+ * or the device alias of pinned mapped host memory for TUTTI_STORE_HOST_PINNED),
+ * 16-byte aligned, `bytes` >= layout.dev_bytes. */
+int tutti_store_register(tutti_ctx_t *ctx, uint32_t dev, void *base, uint64_t bytes, uint32_t kind);
+
+int tutti_set_option(tutti_ctx_t *ctx, uint32_t option, uint64_t value);
+
+/* init_queue(depth) (Section 3.2 step 1): a submission ring of `depth` IOCBs (a
+ * power of two) of ioctx_per_iocb contexts each, a completion queue of the same
+ * depth in pinned host memory, an SGL arena of sgl_capacity entries and plan
+ * scratch for batches of up to max_items = 2 * n_obj items.  All memory the
+ * per-layer path needs is allocated here. */
+int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
+                      uint32_t sgl_capacity, uint32_t max_items, tutti_ring_t **out);
+int tutti_ring_destroy(tutti_ring_t *ring);
+
+/* get_iocb(nums) for descriptors prepared by the CPU (the paper's own split,
+ * Section 3.2: "CPU-prepared, GPU-executed"): reserve n IOCBs and n_sgl arena
+ * entries without building anything. */
+int tutti_ring_reserve(tutti_ring_t *ring, uint32_t n_iocb, uint32_t n_sgl, uint32_t *first_iocb);
+
+/* Fill one reserved IOCB from host arrays and publish it: sqes[n_sqe] (sgl_first
+ * relative to sgl[0]) and sgl[n_sgl] are host pointers, copied before the call
+ * returns.  Entry lengths may differ.  `sgl_offset` places this IOCB's entries
+ * inside the reservation made by tutti_ring_reserve. */
+int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t iocb_idx,
+                         const tutti_sqe_t *sqes, uint32_t n_sqe, const tutti_sgl_t *sgl,
+                         uint32_t n_sgl, uint32_t sgl_offset, void *stream);
+
+/* Inspection (synchronises the device; not for the per-layer path): header, and up
+ * to max_sqes contexts, of a live IOCB into host memory; its SGL entries. */
+int tutti_ring_read_iocb(tutti_ring_t *ring, uint32_t iocb_idx, tutti_iocb_info_t *info,
+                         tutti_sqe_t *sqes, uint32_t max_sqes);
+int tutti_ring_read_sgl(tutti_ring_t *ring, uint32_t iocb_idx, tutti_sgl_t *sgl,
+                        uint32_t max_entries, uint32_t *n_entries);
+
+/* Counters since ring creation (host pointers): kernels launched by this ring's
+ * calls, host calls made on the per-layer path. */
+int tutti_ring_stats(tutti_ring_t *ring, uint64_t *kernel_launches, uint64_t *host_calls);
+
+/* SM partition for the capped mode (Section 3.2 "SM Partitioning For Accurate
+ * I/O": a compute domain and an I/O control domain isolated with green contexts).
+ * Splits the device's SMs into `io_sms` (rounded up to the hardware granularity)
+ * and the rest; returns one stream in each partition and the SM counts obtained.
+ * TUTTI_ECUDA if the driver refuses green contexts. */
+int tutti_sm_partition_create(tutti_ctx_t *ctx, uint32_t io_sms, void **io_stream,
+                              void **compute_stream, uint32_t *io_sms_got,
+                              uint32_t *compute_sms_got);
+int tutti_sm_partition_destroy(tutti_ctx_t *ctx);
+
+/* Host-side ring accounting on its own (no GPU involved; used by CPU tests):
+ * the reservation / release bookkeeping that tutti_build_sqes and tutti_ring_poll
+ * apply to IOCB indices and SGL arena ranges. */
+typedef struct tutti_hostring tutti_hostring_t;
+tutti_hostring_t *tutti_hostring_create(uint32_t depth, uint32_t sgl_capacity);
+void tutti_hostring_destroy(tutti_hostring_t *h);
+int tutti_hostring_reserve(tutti_hostring_t *h, uint32_t n_iocb, uint32_t n_sgl,
+                           uint32_t *first_iocb, uint32_t *sgl_base);
+int tutti_hostring_release(tutti_hostring_t *h, uint32_t iocb_idx); /* IOCB polled */
+int tutti_hostring_live(const tutti_hostring_t *h, uint32_t *iocbs, uint32_t *sgl_entries);
+
+const char *tutti_strerror(int code);
+const char *tutti_last_cuda_error(void);
+uint32_t tutti_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TUTTI_H_ */

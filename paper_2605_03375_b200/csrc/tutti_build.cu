@@ -1,0 +1,466 @@
+// Descriptor build on the GPU (paper Section 3.1 "block lookup and P2P table
+// lookup to generate a batch of lightweight GPU I/O contexts", Section 3.2 IOCB /
+// IOCTX format).  Two kernels:
+//
+//   plan_kernel   one CTA.  Items (object, K|V) -> keys (device, offset) -> sort ->
+//                 adjacency flags -> prefix sums -> contexts for layer 0.  The
+//                 result does not depend on the layer (a layer only adds a constant
+//                 to every offset), so it is kept in the ring and reused while the
+//                 caller's plan_epoch says the batch is unchanged.
+//   emit_kernel   wide.  Per layer: contexts rebased to the layer and packed into
+//                 IOCBs, one 16-byte SGL entry per pool block (block-table lookup),
+//                 the object-side address of every entry, then a release-publish of
+//                 the IOCB headers by the last CTA to finish.
+//
+// The paper prepares these descriptors on the CPU; here GPU threads do it so that
+// no CPU thread touches per-block work.
+#include "tutti_internal.h"
+
+namespace tutti {
+
+namespace {
+
+constexpr int PLAN_THREADS = 1024;
+constexpr uint32_t SMEM_SORT_ITEMS = 8192;   // (8 + 4) bytes each = 96 KiB
+constexpr unsigned long long KEY_NONE = ~0ull;
+
+__device__ __forceinline__ uint32_t find_request(const uint32_t *obj_start, uint32_t n_req,
+                                                 uint32_t o) {
+    // largest r with obj_start[r] <= o  (rows may be empty)
+    uint32_t lo = 0, hi = n_req;           // invariant: obj_start[lo] <= o < obj_start[hi]
+    while (hi - lo > 1) {
+        uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(obj_start + mid) <= o) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// tokens of chunk c of a request that are part of the hit
+__device__ __forceinline__ uint32_t valid_tokens(uint32_t hit, uint32_t c, uint32_t obj_tokens) {
+    unsigned long long start = (unsigned long long)c * obj_tokens;
+    if (start >= hit) return 0;
+    unsigned long long left = hit - start;
+    return left < obj_tokens ? (uint32_t)left : obj_tokens;
+}
+
+__device__ __forceinline__ void note_error(int32_t *where, int32_t code) {
+    atomicCAS(where, 0, code);
+}
+
+__device__ __forceinline__ bool pair_less(unsigned long long ka, uint32_t ia, unsigned long long kb,
+                                          uint32_t ib) {
+    return ka < kb || (ka == kb && ia < ib);
+}
+
+// In-place bitonic sort of (key, idx) pairs, ascending by (key, idx); n is a power
+// of two.  idx values are unique, so the order is total and equals a stable sort by key.
+__device__ void bitonic_sort(unsigned long long *key, uint32_t *idx, uint32_t n) {
+    for (uint32_t k = 2; k <= n; k <<= 1) {
+        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+            for (uint32_t t = threadIdx.x; t < (n >> 1); t += blockDim.x) {
+                // t-th compare-exchange of this stage: partner indices differ in bit j
+                uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                uint32_t p = i | j;
+                bool up = (i & k) == 0;
+                unsigned long long ka = key[i], kb = key[p];
+                uint32_t ia = idx[i], ib = idx[p];
+                bool swap = up ? pair_less(kb, ib, ka, ia) : pair_less(ka, ia, kb, ib);
+                if (swap) {
+                    key[i] = kb; key[p] = ka;
+                    idx[i] = ib; idx[p] = ia;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+struct ScanPair {
+    uint32_t a, b;
+};
+
+// Inclusive scan of (a, b) across the CTA for one element per thread, plus carry.
+__device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &carry) {
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t ua = __shfl_up_sync(0xffffffffu, v.a, d);
+        uint32_t ub = __shfl_up_sync(0xffffffffu, v.b, d);
+        if (lane >= (uint32_t)d) { v.a += ua; v.b += ub; }
+    }
+    if (lane == 31) warp_tot[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        ScanPair w = warp_tot[lane];       // blockDim.x == 1024 -> 32 warps
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t ua = __shfl_up_sync(0xffffffffu, w.a, d);
+            uint32_t ub = __shfl_up_sync(0xffffffffu, w.b, d);
+            if (lane >= (uint32_t)d) { w.a += ua; w.b += ub; }
+        }
+        warp_tot[lane] = w;
+    }
+    __syncthreads();
+    ScanPair off = carry;
+    if (warp > 0) { off.a += warp_tot[warp - 1].a; off.b += warp_tot[warp - 1].b; }
+    v.a += off.a; v.b += off.b;
+    ScanPair tot = warp_tot[31];
+    __syncthreads();
+    if (threadIdx.x == 0) { carry.a += tot.a; carry.b += tot.b; }
+    __syncthreads();
+    return v;
+}
+
+__global__ void __launch_bounds__(PLAN_THREADS, 1)
+plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem) {
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    __shared__ ScanPair warp_tot[32];
+    __shared__ ScanPair carry;
+    __shared__ int32_t s_status;
+    __shared__ uint32_t s_nact;
+
+    unsigned long long *key = use_smem ? reinterpret_cast<unsigned long long *>(dyn_smem)
+                                       : ring.plan_key;
+    uint32_t *idx = use_smem ? reinterpret_cast<uint32_t *>(dyn_smem + (size_t)np * 8)
+                             : ring.plan_idx;
+    const uint32_t n_raw = 2u * b.n_obj;
+
+    if (threadIdx.x == 0) { s_status = 0; s_nact = 0; carry.a = 0; carry.b = 0; }
+    __syncthreads();
+
+    // per-request preconditions
+    for (uint32_t r = threadIdx.x; r < b.n_req; r += blockDim.x) {
+        uint32_t hit = b.hit_tokens[r];
+        uint32_t n_o = b.obj_start[r + 1] - b.obj_start[r];
+        uint32_t n_b = b.blk_start[r + 1] - b.blk_start[r];
+        bool bad = (hit % g.block_tokens) != 0 ||
+                   b.obj_start[r + 1] < b.obj_start[r] || b.blk_start[r + 1] < b.blk_start[r] ||
+                   b.obj_start[r + 1] > b.n_obj || b.blk_start[r + 1] > b.n_blk ||
+                   (unsigned long long)n_o * g.obj_tokens < hit ||
+                   (unsigned long long)n_b * g.block_tokens < hit;
+        if (bad) note_error(&s_status, TUTTI_EINVAL);
+    }
+
+    // step 1: items and their keys (device, offset at layer 0)
+    for (uint32_t q = threadIdx.x; q < np; q += blockDim.x) {
+        unsigned long long k = KEY_NONE;
+        if (q < n_raw && b.n_req > 0) {
+            uint32_t o = q >> 1, kv = q & 1;
+            uint32_t r = find_request(b.obj_start, b.n_req, o);
+            if (o >= b.obj_start[r] && o < b.obj_start[r + 1]) {
+                uint32_t c = o - b.obj_start[r];
+                uint32_t valid = valid_tokens(b.hit_tokens[r], c, g.obj_tokens);
+                if (valid) {
+                    unsigned long long slot = b.obj_slot[o];
+                    if (slot >= g.n_slots) {
+                        note_error(&s_status, TUTTI_EFAULT);
+                    } else {
+                        unsigned long long dev = slot % g.n_devices;
+                        unsigned long long off = (slot / g.n_devices) * g.stride_slot +
+                                                 (unsigned long long)kv * g.stride_kv;
+                        k = (dev << 56) | off;
+                    }
+                }
+            }
+        }
+        key[q] = k;
+        idx[q] = q;
+    }
+    __syncthreads();
+
+    // step 2: order by (device, offset), ties by item id = (request, chunk, K before V)
+    bitonic_sort(key, idx, np);
+
+    // active items are the prefix before the first KEY_NONE
+    for (uint32_t i = threadIdx.x; i < np; i += blockDim.x)
+        if (key[i] != KEY_NONE && (i + 1 == np || key[i + 1] == KEY_NONE)) s_nact = i + 1;
+    __syncthreads();
+    const uint32_t n_act = s_status ? 0 : s_nact;
+
+    // blocks per item (kept in plan_sqe_of until the scans have run)
+    for (uint32_t i = threadIdx.x; i < n_act; i += blockDim.x) {
+        uint32_t q = idx[i], o = q >> 1;
+        uint32_t r = find_request(b.obj_start, b.n_req, o);
+        uint32_t valid = valid_tokens(b.hit_tokens[r], o - b.obj_start[r], g.obj_tokens);
+        ring.plan_sqe_of[i] = valid / g.block_tokens;
+        ring.plan_item[i] = q;
+    }
+    __syncthreads();
+
+    // steps 3-4: adjacency flags (an item starts a new context unless it begins exactly
+    // where its predecessor on the same device ends); packed with the block count
+    for (uint32_t i = threadIdx.x; i < n_act; i += blockDim.x) {
+        uint32_t head = 1;
+        if (i > 0) {
+            unsigned long long k = key[i], kp = key[i - 1];
+            unsigned long long end_prev = (kp & ((1ull << 56) - 1)) +
+                                          (unsigned long long)ring.plan_sqe_of[i - 1] * g.block_bytes;
+            head = ((kp >> 56) != (k >> 56)) || (end_prev != (k & ((1ull << 56) - 1)));
+        }
+        ring.plan_cumblk[i] = (head << 31) | ring.plan_sqe_of[i];
+    }
+    __syncthreads();
+
+    // step 5: prefix sums of (blocks, run heads); every thread touches only its own item
+    for (uint32_t base = 0; base < n_act; base += blockDim.x) {
+        uint32_t i = base + threadIdx.x;
+        ScanPair v{0, 0};
+        uint32_t nblk = 0, head = 0;
+        if (i < n_act) {
+            uint32_t packed = ring.plan_cumblk[i];
+            nblk = packed & 0x7fffffffu;
+            head = packed >> 31;
+            v.a = nblk; v.b = head;
+        }
+        ScanPair s = block_scan_incl(v, warp_tot, carry);
+        if (i < n_act) {
+            uint32_t excl = s.a - nblk;
+            uint32_t sq = s.b - 1;
+            ring.plan_cumblk[i] = excl;
+            ring.plan_sqe_of[i] = sq;
+            if (head) {
+                unsigned long long k = key[i];
+                tutti_sqe_t e;
+                e.src_off = k & ((1ull << 56) - 1);
+                e.len = 0;
+                e.sgl_first = excl;
+                e.sgl_count = 0;
+                e.dev = (uint32_t)(k >> 56);
+                e.opcode = 0;
+                e.layer = 0;
+                ring.plan_sqe[sq] = e;
+            }
+        }
+    }
+    __syncthreads();
+    const uint32_t n_entries = carry.a, n_sqe = carry.b;
+    if (threadIdx.x == 0) ring.plan_cumblk[n_act] = n_entries;
+    __syncthreads();
+
+    // close every run: length and entry count
+    for (uint32_t i = threadIdx.x; i < n_act; i += blockDim.x) {
+        uint32_t sq = ring.plan_sqe_of[i];
+        bool last = (i + 1 == n_act) || (ring.plan_sqe_of[i + 1] != sq);
+        if (last) {
+            uint32_t cnt = ring.plan_cumblk[i + 1] - ring.plan_sqe[sq].sgl_first;
+            ring.plan_sqe[sq].sgl_count = cnt;
+            ring.plan_sqe[sq].len = (unsigned long long)cnt * g.block_bytes;
+        }
+    }
+    if (threadIdx.x == 0) {
+        PlanCounts pc;
+        pc.n_items = n_act;
+        pc.n_sqe = n_sqe;
+        pc.n_entries = n_entries;
+        pc.status = s_status;
+        *ring.plan_counts = pc;
+    }
+}
+
+constexpr int EMIT_THREADS = 256;
+
+struct EmitParams {
+    uint32_t layer, opcode;
+    uint64_t k_base, v_base, block_stride, n_pool_blocks;
+    uint64_t store_base[TUTTI_MAX_DEVICES];
+    uint64_t store_bytes[TUTTI_MAX_DEVICES];
+    uint32_t first_iocb, n_iocb, sgl_base, sgl_reserved;
+};
+
+__global__ void __launch_bounds__(EMIT_THREADS)
+emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
+    const PlanCounts pc = *ring.plan_counts;
+    IocbHdr *hdr0 = &ring.hdrs[p.first_iocb & (ring.depth - 1)];
+    int32_t status = pc.status;
+    if (status == 0 && pc.n_entries > p.sgl_reserved) status = TUTTI_EINVAL;
+    const uint32_t n_sqe = status ? 0 : pc.n_sqe;
+    const uint32_t n_items = status ? 0 : pc.n_items;
+    const uint32_t n_entries = status ? 0 : pc.n_entries;
+    const unsigned long long layer_off = (unsigned long long)p.layer * g.stride_layer;
+
+    // IOCB headers (step 7 of the path): CTA 0
+    if (blockIdx.x == 0) {
+        for (uint32_t k = threadIdx.x; k < p.n_iocb; k += blockDim.x) {
+            uint32_t idx = p.first_iocb + k;
+            IocbHdr *h = &ring.hdrs[idx & (ring.depth - 1)];
+            unsigned long long s0 = (unsigned long long)k * ring.capacity;
+            unsigned long long s1 = s0 + ring.capacity;
+            uint32_t e0 = s0 < n_sqe ? ring.plan_sqe[s0].sgl_first : n_entries;
+            uint32_t e1 = s1 < n_sqe ? ring.plan_sqe[s1].sgl_first : n_entries;
+            h->num_ioctx = s0 < n_sqe ? (uint32_t)((s1 < n_sqe ? s1 : n_sqe) - s0) : 0;
+            h->opcode = p.opcode;
+            h->layer = p.layer;
+            h->status = status;
+            h->sgl_base = p.sgl_base;
+            h->entry_first = e0;
+            h->total_entries = e1 - e0;
+            h->entry_len = (uint32_t)g.block_bytes;
+            h->claim_cursor = 0;
+            h->done_bytes = 0;
+            h->bytes = (unsigned long long)(e1 - e0) * g.block_bytes;
+        }
+    }
+
+    // contexts, rebased to this layer and packed into IOCBs
+    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t gthreads = gridDim.x * blockDim.x;
+    for (uint32_t k = gtid; k < n_sqe; k += gthreads) {
+        tutti_sqe_t e = ring.plan_sqe[k];
+        e.src_off += layer_off;
+        e.opcode = (uint16_t)p.opcode;
+        e.layer = (uint16_t)p.layer;
+        uint32_t slot = (p.first_iocb + k / ring.capacity) & (ring.depth - 1);
+        ring.sqes[(size_t)slot * ring.capacity + k % ring.capacity] = e;
+    }
+
+    // SGL entries: one warp per item, lanes over the item's blocks
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t gwarp = gtid >> 5, nwarps = gthreads >> 5;
+    for (uint32_t i = gwarp; i < n_items; i += nwarps) {
+        uint32_t q = 0, e_first = 0, e_next = 0, sq = 0;
+        if (lane == 0) {
+            q = ring.plan_item[i];
+            e_first = ring.plan_cumblk[i];
+            e_next = ring.plan_cumblk[i + 1];
+            sq = ring.plan_sqe_of[i];
+        }
+        q = __shfl_sync(0xffffffffu, q, 0);
+        e_first = __shfl_sync(0xffffffffu, e_first, 0);
+        e_next = __shfl_sync(0xffffffffu, e_next, 0);
+        sq = __shfl_sync(0xffffffffu, sq, 0);
+        const uint32_t o = q >> 1, kv = q & 1;
+        unsigned long long meta0 = 0, meta1 = 0;   // (row start in block table, object-side address)
+        if (lane == 0) {
+            uint32_t r = find_request(b.obj_start, b.n_req, o);
+            uint32_t c = o - b.obj_start[r];
+            meta0 = (unsigned long long)b.blk_start[r] + (unsigned long long)c * g.blocks_per_obj;
+            // object-side address of the item's first byte: context start + bytes of the
+            // items that precede it in the same run
+            tutti_sqe_t run = ring.plan_sqe[sq];
+            unsigned long long off = run.src_off + layer_off +
+                                     (unsigned long long)(e_first - run.sgl_first) * g.block_bytes;
+            unsigned long long end = off + (unsigned long long)(e_next - e_first) * g.block_bytes;
+            if (end > p.store_bytes[run.dev]) {
+                note_error(&hdr0->emit_status, TUTTI_EFAULT);
+                meta1 = 0;
+            } else {
+                meta1 = p.store_base[run.dev] + off;
+            }
+        }
+        const unsigned long long row0 = __shfl_sync(0xffffffffu, meta0, 0);
+        const unsigned long long obj0 = __shfl_sync(0xffffffffu, meta1, 0);
+        const unsigned long long pool_base = kv ? p.v_base : p.k_base;
+        const uint32_t n_blk = e_next - e_first;
+        for (uint32_t j = lane; j < n_blk; j += 32) {
+            unsigned long long bi = row0 + j;
+            tutti_sgl_t ent;
+            ent.len = (uint32_t)g.block_bytes;
+            if (bi >= b.n_blk) {
+                note_error(&hdr0->emit_status, TUTTI_EFAULT);
+                continue;
+            }
+            int32_t id = b.block_ids[bi];
+            if (id < 0 || (unsigned long long)id >= p.n_pool_blocks) {
+                note_error(&hdr0->emit_status, TUTTI_EFAULT);
+                continue;
+            }
+            ent.addr = pool_base + (unsigned long long)id * p.block_stride;
+            ent.id = (uint32_t)id;
+            size_t at = (size_t)p.sgl_base + e_first + j;
+            ring.sgl[at] = ent;
+            ring.obj_ptr[at] = obj0 + (unsigned long long)j * g.block_bytes;
+        }
+    }
+
+    // publish: the last CTA to finish makes every IOCB of the build visible
+    __syncthreads();
+    __shared__ uint32_t s_last;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        uint32_t prev = atomicAdd(&hdr0->emit_done, 1u);
+        s_last = (prev == gridDim.x - 1);
+        __threadfence();
+    }
+    __syncthreads();
+    if (!s_last) return;
+    int32_t est = *((volatile int32_t *)&hdr0->emit_status);
+    for (uint32_t k = threadIdx.x; k < p.n_iocb; k += blockDim.x) {
+        uint32_t idx = p.first_iocb + k;
+        IocbHdr *h = &ring.hdrs[idx & (ring.depth - 1)];
+        if (est != 0) {
+            h->status = est;
+            h->total_entries = 0;
+            h->bytes = 0;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        hdr0->emit_done = 0;
+        hdr0->emit_status = 0;
+    }
+    __threadfence();
+    __syncthreads();
+    for (uint32_t k = threadIdx.x; k < p.n_iocb; k += blockDim.x) {
+        uint32_t idx = p.first_iocb + k;
+        IocbHdr *h = &ring.hdrs[idx & (ring.depth - 1)];
+        // release: descriptors before the state word
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&h->state),
+                     "r"(state_word(idx, PHASE_READY)) : "memory");
+    }
+}
+
+uint32_t next_pow2(uint32_t v) {
+    uint32_t p = 32;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+}  // namespace
+
+cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
+                        cudaStream_t stream) {
+    uint32_t np = next_pow2(2u * batch.n_obj);
+    int use_smem = np <= SMEM_SORT_ITEMS;
+    size_t smem = use_smem ? (size_t)np * 12 : 0;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(SMEM_SORT_ITEMS * 12));
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    plan_kernel<<<1, PLAN_THREADS, smem, stream>>>(ring, geom, batch, np, use_smem);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
+                        uint32_t layer, uint32_t opcode, const PoolLayer &pool,
+                        const uint64_t *store_base, const uint64_t *store_bytes,
+                        uint32_t first_iocb, uint32_t n_iocb, uint32_t sgl_base,
+                        uint32_t sgl_reserved, int device_sms, cudaStream_t stream) {
+    EmitParams p;
+    p.layer = layer;
+    p.opcode = opcode;
+    p.k_base = pool.k_base;
+    p.v_base = pool.v_base;
+    p.block_stride = pool.block_stride;
+    p.n_pool_blocks = pool.n_blocks;
+    for (int d = 0; d < TUTTI_MAX_DEVICES; ++d) {
+        p.store_base[d] = store_base[d];
+        p.store_bytes[d] = store_bytes[d];
+    }
+    p.first_iocb = first_iocb;
+    p.n_iocb = n_iocb;
+    p.sgl_base = sgl_base;
+    p.sgl_reserved = sgl_reserved;
+    // one warp per item, 8 warps per CTA; a few CTAs per SM at most
+    uint32_t items = 2u * batch.n_obj;
+    uint32_t ctas = (items + 7) / 8;
+    uint32_t cap = (uint32_t)device_sms * 2u;
+    if (ctas > cap) ctas = cap;
+    if (ctas == 0) ctas = 1;
+    emit_kernel<<<ctas, EMIT_THREADS, 0, stream>>>(ring, geom, batch, p);
+    return cudaGetLastError();
+}
+
+}  // namespace tutti

@@ -1,0 +1,523 @@
+// Paged scatter / gather between contiguous KV objects and the block-table-indexed
+// KV pool (layer-wise Retrieve / Store of paper Section 3.1 and 3.4), executed from
+// the IOCBs of the submission ring (Section 3.2 step 3, issue_io), with completion
+// entries written to the CQ by the kernel itself.
+//
+// Two engines over the same descriptors:
+//   ldst   256-thread CTAs; every lane moves 16 bytes per instruction, eight
+//          independent loads in flight per lane before the first store; a warp owns a
+//          4 KiB sub-range of a tile, its lanes 0..7 fetch the SGL entries of that
+//          sub-range once and broadcast them with shuffles.
+//   bulk   persistent CTAs whose warps each run a ring of shared-memory stages:
+//          cp.async.bulk global->shared (mbarrier completion) then shared->global,
+//          so a handful of threads keep >100 KiB in flight per SM.  This is the
+//          engine of the SM-capped mode.
+// Both claim work in chunks with one atomicAdd per claim on the IOCB's cursor and
+// account completion in bytes; the agent that lands the last byte writes the CQE.
+//
+// Every wait is bounded: a timed-out wait records TUTTI_ETIMEDOUT in the IOCB
+// status and the kernel still terminates normally.
+#include "tutti_internal.h"
+
+namespace tutti {
+
+namespace {
+
+constexpr uint32_t CHUNK_BYTES = 32768;       // work unit of both engines
+constexpr int LDST_THREADS = 256;
+constexpr uint32_t MBAR_TRY_LIMIT = 1u << 22;
+
+struct CopyParams {
+    RingDev ring;
+    uint32_t first_iocb, n_iocb, opcode;
+    unsigned long long wait_ns;
+    uint32_t claim_chunks;
+    uint32_t stages;        // bulk engine: stages per warp
+};
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Completion entry into pinned host memory: entry, system fence, then its sequence word.
+__device__ void post_cqe(const RingDev &ring, uint32_t iocb_idx, int32_t status,
+                         unsigned long long bytes) {
+    uint32_t pos = atomicAdd(ring.cq_reserve, 1u);
+    CqSlot *slot = &ring.cq[pos & (ring.depth - 1)];
+    volatile tutti_cqe_t *c = &slot->cqe;
+    c->iocb_idx = iocb_idx;
+    c->status = status;
+    c->bytes = bytes;
+    __threadfence_system();
+    *((volatile uint32_t *)&slot->seq) = pos + 1;
+    __threadfence_system();
+}
+
+enum { IOCB_RUN = 0, IOCB_SKIP = 1 };
+
+// One agent (thread) waits until the IOCB is published.  Returns IOCB_RUN when it is
+// ready, IOCB_SKIP when it is already complete or when the wait ran out (in which
+// case exactly one agent posts a TUTTI_ETIMEDOUT completion).
+__device__ int wait_iocb_ready(const RingDev &ring, IocbHdr *h, uint32_t idx,
+                               unsigned long long wait_ns) {
+    const uint32_t ready = state_word(idx, PHASE_READY), done = state_word(idx, PHASE_DONE);
+    const unsigned long long t0 = globaltimer_ns();
+    for (uint32_t it = 0;; ++it) {
+        uint32_t s = ld_acquire_u32(&h->state);
+        if (s == ready) return IOCB_RUN;
+        if (s == done) return IOCB_SKIP;
+        if (globaltimer_ns() - t0 > wait_ns || it > (1u << 24)) {
+            if (atomicCAS(&h->state, s, done) == s) {
+                __threadfence();
+                post_cqe(ring, idx, TUTTI_ETIMEDOUT, 0);
+                return IOCB_SKIP;
+            }
+        }
+        __nanosleep(64);
+    }
+}
+
+// An IOCB with nothing to move (empty, or carrying a build error): one agent wins the
+// READY -> DONE transition and posts the completion.
+__device__ void complete_empty(const RingDev &ring, IocbHdr *h, uint32_t idx) {
+    if (atomicCAS(&h->state, state_word(idx, PHASE_READY), state_word(idx, PHASE_DONE)) ==
+        state_word(idx, PHASE_READY))
+        post_cqe(ring, idx, h->status, 0);
+}
+
+// Account `bytes` landed; the agent that completes the IOCB posts the CQE.
+__device__ void account_done(const RingDev &ring, IocbHdr *h, uint32_t idx,
+                             unsigned long long bytes) {
+    if (bytes == 0) return;
+    __threadfence();
+    unsigned long long before = atomicAdd(&h->done_bytes, bytes);
+    if (before + bytes == h->bytes) {
+        __threadfence();
+        int32_t st = *((volatile int32_t *)&h->status);
+        *((volatile uint32_t *)&h->state) = state_word(idx, PHASE_DONE);
+        post_cqe(ring, idx, st, h->bytes);
+    }
+}
+
+__device__ __forceinline__ uint4 ld_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(void *p, const uint4 &v) {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};"
+                 ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// ---------------------------------------------------------------------------
+// ldst engine
+// ---------------------------------------------------------------------------
+template <int TO_POOL>
+__global__ void __launch_bounds__(LDST_THREADS)
+copy_ldst_kernel(CopyParams p) {
+    __shared__ uint32_t s_claim;
+    __shared__ int s_mode;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    for (uint32_t bi = 0; bi < p.n_iocb; ++bi) {
+        const uint32_t idx = p.first_iocb + bi;
+        IocbHdr *h = &p.ring.hdrs[idx & (p.ring.depth - 1)];
+        if (threadIdx.x == 0) s_mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
+        __syncthreads();
+        const int mode = s_mode;
+        __syncthreads();
+        if (mode == IOCB_SKIP) continue;
+        const uint32_t total = h->total_entries;
+        if (total == 0 || h->status != 0) {
+            if (threadIdx.x == 0) complete_empty(p.ring, h, idx);
+            continue;
+        }
+        const uint32_t elen = h->entry_len;
+        const size_t e_base = (size_t)h->sgl_base + h->entry_first;
+        const tutti_sgl_t *sgl = p.ring.sgl + e_base;
+        const uint64_t *obj = p.ring.obj_ptr + e_base;
+
+        if (elen != 0 && (elen & 511u) == 0) {
+            // uniform entries, every 512-byte warp row lies inside one entry
+            const unsigned long long total_bytes = (unsigned long long)total * elen;
+            const uint32_t n_tiles = (uint32_t)((total_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
+            const bool pow2 = (elen & (elen - 1)) == 0;
+            const uint32_t shift = 31 - __clz(elen);
+            for (;;) {
+                if (threadIdx.x == 0) s_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
+                __syncthreads();
+                const uint32_t t0 = s_claim;
+                if (t0 >= n_tiles) { __syncthreads(); break; }
+                const uint32_t t1 = min(t0 + p.claim_chunks, n_tiles);
+                for (uint32_t t = t0; t < t1; ++t) {
+                    // this warp's 4 KiB sub-range of the tile: 8 rows of 512 bytes
+                    const unsigned long long p0 = (unsigned long long)t * CHUNK_BYTES + warp * 4096u;
+                    if (p0 >= total_bytes) continue;
+                    const uint32_t e0 = pow2 ? (uint32_t)(p0 >> shift) : (uint32_t)(p0 / elen);
+                    // lanes 0..7 fetch the entries this sub-range can touch, once
+                    unsigned long long my_pool = 0, my_obj = 0;
+                    if (lane < 8 && e0 + lane < total) {
+                        my_pool = sgl[e0 + lane].addr;
+                        my_obj = obj[e0 + lane];
+                    }
+                    uint4 v[8];
+                    unsigned long long dst[8];
+                    bool ok[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const unsigned long long pk = p0 + (unsigned long long)k * 512u;
+                        ok[k] = pk < total_bytes;
+                        const uint32_t e = ok[k] ? (pow2 ? (uint32_t)(pk >> shift) : (uint32_t)(pk / elen)) : e0;
+                        const uint32_t off = (uint32_t)(pk - (unsigned long long)e * elen) + lane * 16u;
+                        const unsigned long long a_pool = __shfl_sync(0xffffffffu, my_pool, e - e0);
+                        const unsigned long long a_obj = __shfl_sync(0xffffffffu, my_obj, e - e0);
+                        const unsigned long long src = (TO_POOL ? a_obj : a_pool) + off;
+                        dst[k] = (TO_POOL ? a_pool : a_obj) + off;
+                        if (ok[k]) v[k] = ld_stream(reinterpret_cast<const void *>(src));
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (ok[k]) st_stream(reinterpret_cast<void *>(dst[k]), v[k]);
+                }
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    unsigned long long b0 = (unsigned long long)t0 * CHUNK_BYTES;
+                    unsigned long long b1 = min((unsigned long long)t1 * CHUNK_BYTES, total_bytes);
+                    account_done(p.ring, h, idx, b1 - b0);
+                }
+            }
+        } else {
+            // general entries (lengths may differ): one warp per entry
+            const uint32_t per_claim = 64;
+            for (;;) {
+                if (threadIdx.x == 0) s_claim = atomicAdd(&h->claim_cursor, per_claim);
+                __syncthreads();
+                const uint32_t c0 = s_claim;
+                if (c0 >= total) { __syncthreads(); break; }
+                const uint32_t c1 = min(c0 + per_claim, total);
+                unsigned long long moved = 0;
+                for (uint32_t e = c0 + warp; e < c1; e += LDST_THREADS / 32) {
+                    unsigned long long a_pool = 0, a_obj = 0;
+                    uint32_t len = 0;
+                    if (lane == 0) { a_pool = sgl[e].addr; len = sgl[e].len; a_obj = obj[e]; }
+                    a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
+                    a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
+                    len = __shfl_sync(0xffffffffu, len, 0);
+                    const unsigned long long src = TO_POOL ? a_obj : a_pool;
+                    const unsigned long long dst = TO_POOL ? a_pool : a_obj;
+                    for (uint32_t o = lane * 16u; o < len; o += 512u)
+                        st_stream(reinterpret_cast<void *>(dst + o),
+                                  ld_stream(reinterpret_cast<const void *>(src + o)));
+                    moved += len;
+                }
+                __syncwarp();
+                if (lane == 0) account_done(p.ring, h, idx, moved);
+                __syncthreads();
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// bulk-async engine
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait for a phase of an mbarrier; false when it gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < MBAR_TRY_LIMIT; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, unsigned long long src, uint32_t bytes,
+                                         uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(unsigned long long dst, uint32_t src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_read_1() {
+    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+constexpr int BULK_MAX_STAGES = 8;
+
+// Geometry of the chunks of one IOCB with uniform entry length.
+struct ChunkGeom {
+    uint32_t elen;       // entry length
+    uint32_t per_chunk;  // entries per chunk when elen <= CHUNK_BYTES (1..32), else 0
+    uint32_t pieces;     // pieces per entry when elen > CHUNK_BYTES, else 0
+    uint32_t n_chunks;
+    uint32_t total;
+};
+
+__device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen) {
+    ChunkGeom g;
+    g.elen = elen;
+    g.total = total;
+    if (elen <= CHUNK_BYTES) {
+        uint32_t pc = CHUNK_BYTES / elen;
+        g.per_chunk = pc > 32 ? 32 : pc;
+        g.pieces = 0;
+        g.n_chunks = (total + g.per_chunk - 1) / g.per_chunk;
+    } else {
+        g.per_chunk = 0;
+        g.pieces = (elen + CHUNK_BYTES - 1) / CHUNK_BYTES;
+        g.n_chunks = total * g.pieces;
+    }
+    return g;
+}
+
+// Each warp of the CTA is an independent agent with its own stage ring.
+// Shared memory: [warps][stages][CHUNK_BYTES] data, then [warps][stages] mbarriers,
+// then [warps][stages] chunk ids.
+template <int TO_POOL>
+__global__ void __launch_bounds__(256, 1)
+copy_bulk_kernel(CopyParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t n_warps = blockDim.x >> 5;
+    const uint32_t S = p.stages;
+    unsigned char *data = smem + (size_t)warp * S * CHUNK_BYTES;
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(
+        smem + (size_t)n_warps * S * CHUNK_BYTES) + warp * S;
+    uint32_t *chunk_of = reinterpret_cast<uint32_t *>(
+        smem + (size_t)n_warps * S * CHUNK_BYTES + (size_t)n_warps * S * 8) + warp * S;
+
+    if (lane == 0)
+        for (uint32_t s = 0; s < S; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+    __syncwarp();
+
+    uint32_t phase_bits = 0;   // parity of every stage's mbarrier (bit s)
+
+    for (uint32_t bi = 0; bi < p.n_iocb; ++bi) {
+        const uint32_t idx = p.first_iocb + bi;
+        IocbHdr *h = &p.ring.hdrs[idx & (p.ring.depth - 1)];
+        int mode = 0;
+        if (lane == 0) mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
+        mode = __shfl_sync(0xffffffffu, mode, 0);
+        if (mode == IOCB_SKIP) continue;
+        const uint32_t total = h->total_entries;
+        if (total == 0 || h->status != 0) {
+            if (lane == 0) complete_empty(p.ring, h, idx);
+            continue;
+        }
+        const ChunkGeom cg = chunk_geom(total, h->entry_len);
+        const size_t e_base = (size_t)h->sgl_base + h->entry_first;
+        const tutti_sgl_t *sgl = p.ring.sgl + e_base;
+        const uint64_t *obj = p.ring.obj_ptr + e_base;
+
+        uint32_t head = 0, tail = 0;            // stages issued / drained (monotonic)
+        uint32_t cur = 0, cur_end = 0;          // claimed chunk range
+        bool exhausted = false;
+        unsigned long long moved = 0;           // bytes this agent has stored
+        bool failed = false;
+
+        for (;;) {
+            // ---- issue loads while a stage is free (keep one stage of slack for the
+            //      store that is still reading shared memory)
+            while (!exhausted && head - tail < S - 1) {
+                if (cur == cur_end) {
+                    uint32_t c0 = 0;
+                    if (lane == 0) c0 = atomicAdd(&h->claim_cursor, p.claim_chunks);
+                    c0 = __shfl_sync(0xffffffffu, c0, 0);
+                    if (c0 >= cg.n_chunks) { exhausted = true; break; }
+                    cur = c0;
+                    cur_end = min(c0 + p.claim_chunks, cg.n_chunks);
+                }
+                const uint32_t c = cur++;
+                const uint32_t s = head % S;
+                // the store that last used this stage must have finished reading it:
+                // at most one newer store group may still be pending
+                bulk_wait_read_1();
+                __syncwarp();
+                const uint32_t bar = smem_u32(&bars[s]);
+                const uint32_t sbase = smem_u32(data + (size_t)s * CHUNK_BYTES);
+                if (cg.per_chunk) {
+                    const uint32_t e0 = c * cg.per_chunk;
+                    const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
+                    unsigned long long a_obj = 0, a_pool = 0;
+                    if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
+                    if (lane == 0) mbar_expect_tx(bar, n_e * cg.elen);
+                    __syncwarp();
+                    if (TO_POOL) {
+                        // object side is contiguous in runs: one load per run
+                        unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
+                        bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
+                        uint32_t heads = __ballot_sync(0xffffffffu, is_head);
+                        if (is_head) {
+                            uint32_t above = heads >> (lane + 1);
+                            uint32_t next = above ? lane + __ffs(above) : n_e;
+                            bulk_g2s(sbase + lane * cg.elen, a_obj, (next - lane) * cg.elen, bar);
+                        }
+                    } else {
+                        if (lane < n_e) bulk_g2s(sbase + lane * cg.elen, a_pool, cg.elen, bar);
+                    }
+                } else {
+                    const uint32_t e = c / cg.pieces, piece = c % cg.pieces;
+                    const uint32_t off = piece * CHUNK_BYTES;
+                    const uint32_t bytes = min(CHUNK_BYTES, cg.elen - off);
+                    if (lane == 0) {
+                        unsigned long long src = (TO_POOL ? obj[e] : sgl[e].addr) + off;
+                        mbar_expect_tx(bar, bytes);
+                        bulk_g2s(sbase, src, bytes, bar);
+                    }
+                }
+                if (lane == 0) chunk_of[s] = c;
+                __syncwarp();
+                ++head;
+            }
+            if (head == tail) break;
+
+            // ---- drain the oldest stage: wait for its bytes, store them
+            const uint32_t s = tail % S;
+            const uint32_t bar = smem_u32(&bars[s]);
+            const uint32_t sbase = smem_u32(data + (size_t)s * CHUNK_BYTES);
+            const uint32_t c = chunk_of[s];
+            bool arrived = mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
+            arrived = __all_sync(0xffffffffu, arrived);
+            phase_bits ^= (1u << s);
+            if (!arrived) failed = true;
+            fence_proxy_async();
+            if (cg.per_chunk) {
+                const uint32_t e0 = c * cg.per_chunk;
+                const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
+                unsigned long long a_obj = 0, a_pool = 0;
+                if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
+                if (arrived) {
+                    if (TO_POOL) {
+                        if (lane < n_e) bulk_s2g(a_pool, sbase + lane * cg.elen, cg.elen);
+                    } else {
+                        unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
+                        bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
+                        uint32_t heads = __ballot_sync(0xffffffffu, is_head);
+                        if (is_head) {
+                            uint32_t above = heads >> (lane + 1);
+                            uint32_t next = above ? lane + __ffs(above) : n_e;
+                            bulk_s2g(a_obj, sbase + lane * cg.elen, (next - lane) * cg.elen);
+                        }
+                    }
+                }
+                moved += (unsigned long long)n_e * cg.elen;
+            } else {
+                const uint32_t e = c / cg.pieces, piece = c % cg.pieces;
+                const uint32_t off = piece * CHUNK_BYTES;
+                const uint32_t bytes = min(CHUNK_BYTES, cg.elen - off);
+                if (lane == 0 && arrived) {
+                    unsigned long long dst = (TO_POOL ? sgl[e].addr : obj[e]) + off;
+                    bulk_s2g(dst, sbase, bytes);
+                }
+                moved += bytes;
+            }
+            bulk_commit();
+            ++tail;
+            if (failed) {
+                // stop taking new work; what is in flight is still drained above
+                exhausted = true;
+            }
+        }
+        // all of this agent's stores must have landed before they are accounted
+        bulk_wait_all();
+        __syncwarp();
+        if (lane == 0) {
+            if (failed) atomicCAS(&h->status, 0, TUTTI_ETIMEDOUT);
+            account_done(p.ring, h, idx, moved);
+        }
+        __syncwarp();
+    }
+}
+
+}  // namespace
+
+cudaError_t copy_kernels_setup() {
+    cudaError_t e;
+    const int max_smem = 227 * 1024;
+    e = cudaFuncSetAttribute(copy_bulk_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(copy_bulk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    return e;
+}
+
+cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
+                        uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
+                        cudaStream_t stream, uint32_t *launches) {
+    CopyParams p;
+    p.ring = ring;
+    p.first_iocb = first_iocb;
+    p.n_iocb = n_iocb;
+    p.opcode = opcode;
+    p.wait_ns = opt.wait_ns;
+    p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : 4;
+    uint32_t engine = opt.engine;
+    if (engine == 0) engine = (sm_count != 0 && !host_store) ? 2 : 1;
+    const uint32_t sms = sm_count ? sm_count : (uint32_t)device_sms;
+    if (engine == 2) {
+        uint32_t warps = opt.bulk_warps ? opt.bulk_warps : 2;
+        uint32_t stages = opt.bulk_stages ? opt.bulk_stages : 3;
+        if (warps > 8) warps = 8;
+        if (stages < 2) stages = 2;
+        if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
+        while ((size_t)warps * stages * (CHUNK_BYTES + 16) > 220u * 1024u) {
+            if (stages > 2) --stages; else --warps;
+        }
+        p.stages = stages;
+        size_t smem = (size_t)warps * stages * (CHUNK_BYTES + 8 + 4);
+        // a capped launch keeps one CTA per SM: pad shared memory so no second CTA fits
+        if (sm_count && smem < 120u * 1024u) smem = 120u * 1024u;
+        if (opcode == TUTTI_OP_READ)
+            copy_bulk_kernel<1><<<sms, warps * 32, smem, stream>>>(p);
+        else
+            copy_bulk_kernel<0><<<sms, warps * 32, smem, stream>>>(p);
+    } else {
+        p.stages = 0;
+        uint32_t per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 4;
+        if (opcode == TUTTI_OP_READ)
+            copy_ldst_kernel<1><<<sms * per_sm, LDST_THREADS, 0, stream>>>(p);
+        else
+            copy_ldst_kernel<0><<<sms * per_sm, LDST_THREADS, 0, stream>>>(p);
+    }
+    if (launches) *launches = 1;
+    return cudaGetLastError();
+}
+
+}  // namespace tutti

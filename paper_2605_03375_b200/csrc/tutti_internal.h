@@ -1,0 +1,120 @@
+// Internal definitions shared by the host side of the library and its kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/tutti.h"
+#include "host_ring.h"
+
+namespace tutti {
+
+// IOCB header in HBM (paper Section 3.2: an SQ entry is an IOCB holding up to
+// ioctx_per_iocb I/O contexts plus num_ioctx).  64 bytes, one per ring slot.
+// `state` carries the IOCB index so that a stale value from the slot's previous
+// use is never mistaken for the current one.
+struct __align__(64) IocbHdr {
+    uint32_t state;          // state_word(idx, phase)
+    uint32_t num_ioctx;
+    uint32_t opcode;
+    uint32_t layer;
+    int32_t status;          // first error found while building or copying (0 = none)
+    uint32_t sgl_base;       // arena index of the build's first SGL entry
+    uint32_t entry_first;    // first entry of this IOCB, relative to sgl_base
+    uint32_t total_entries;
+    uint32_t entry_len;      // common length of all entries, 0 = lengths differ
+    uint32_t claim_cursor;   // next unclaimed chunk
+    unsigned long long done_bytes;  // bytes that have landed
+    unsigned long long bytes;       // bytes this IOCB moves
+    uint32_t emit_done;      // build: CTAs finished (first IOCB of a build only)
+    int32_t emit_status;     // build: first error seen by any CTA
+};
+static_assert(sizeof(IocbHdr) == 64, "IocbHdr must be 64 bytes");
+
+enum : uint32_t { PHASE_FREE = 0, PHASE_READY = 1, PHASE_DONE = 2 };
+__host__ __device__ inline uint32_t state_word(uint32_t iocb_idx, uint32_t phase) {
+    return (iocb_idx << 2) | phase;
+}
+
+// Completion queue slot in pinned host memory: the entry, then a sequence word
+// written last (value = position in the CQ + 1).
+struct __align__(32) CqSlot {
+    tutti_cqe_t cqe;
+    uint32_t seq;
+    uint32_t pad[3];
+};
+static_assert(sizeof(CqSlot) == 32, "CqSlot must be 32 bytes");
+
+// Batch-level plan (independent of the layer): items in (device, offset) order.
+struct PlanCounts {
+    uint32_t n_items;    // active items (objects x {K,V} with at least one hit token)
+    uint32_t n_sqe;
+    uint32_t n_entries;
+    int32_t status;
+};
+
+struct PoolLayer {
+    uint64_t k_base, v_base, block_stride, n_blocks;
+    bool registered;
+};
+
+struct StoreDev {
+    uint64_t base, bytes;
+    uint32_t kind;
+    bool registered;
+};
+
+// Device-side view of a ring, passed by value to kernels.
+struct RingDev {
+    IocbHdr *hdrs;            // [depth]
+    tutti_sqe_t *sqes;        // [depth * capacity]
+    tutti_sgl_t *sgl;         // [sgl_capacity]   pool side of every entry
+    uint64_t *obj_ptr;        // [sgl_capacity]   object-store side of every entry
+    CqSlot *cq;               // [depth]          device alias of pinned host memory
+    uint32_t *cq_reserve;     // CQ position counter (HBM)
+    uint32_t depth;           // power of two
+    uint32_t capacity;        // contexts per IOCB
+    // plan scratch
+    uint32_t *plan_item;      // [max_items]  item id (2*object + kv) in sorted order
+    uint32_t *plan_cumblk;    // [max_items+1] exclusive prefix of blocks per item
+    uint32_t *plan_sqe_of;    // [max_items]  context index of each item
+    tutti_sqe_t *plan_sqe;    // [max_items]  contexts for layer 0, opcode unset
+    unsigned long long *plan_key;  // [pow2(max_items)] sort keys when they do not fit in shared memory
+    uint32_t *plan_idx;       // [pow2(max_items)] sort payload, same
+    PlanCounts *plan_counts;
+    uint32_t max_items;
+};
+
+struct GeomDev {
+    uint32_t block_tokens, obj_tokens, blocks_per_obj, n_devices;
+    uint64_t token_bytes, block_bytes, stride_kv, stride_layer, stride_slot, n_slots;
+    uint64_t dev_bytes;
+};
+
+struct BatchDev {
+    uint32_t n_req, n_obj, n_blk;
+    const uint32_t *hit_tokens, *obj_start, *obj_slot, *blk_start;
+    const int32_t *block_ids;
+};
+
+struct CopyOptions {
+    uint32_t engine;        // 0 auto, 1 ld/st, 2 bulk
+    uint64_t wait_ns;
+    uint32_t ctas_per_sm;
+    uint32_t bulk_warps, bulk_stages;
+    uint32_t claim_chunks;
+};
+
+// kernels (tutti_build.cu / tutti_copy.cu)
+cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
+                        cudaStream_t stream);
+cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
+                        uint32_t layer, uint32_t opcode, const PoolLayer &pool,
+                        const uint64_t *store_base, const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
+                        uint32_t sgl_base, uint32_t sgl_reserved, int device_sms,
+                        cudaStream_t stream);
+cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
+                        uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
+                        cudaStream_t stream, uint32_t *launches);
+cudaError_t copy_kernels_setup();
+
+}  // namespace tutti

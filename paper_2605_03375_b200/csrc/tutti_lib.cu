@@ -1,0 +1,606 @@
+// Host side of the C ABI declared in include/tutti.h: contexts, registration
+// tables, the ring and its completion queue.  All device work is in
+// tutti_build.cu / tutti_copy.cu; nothing here falls back to the CPU.
+#include <chrono>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "tutti_internal.h"
+
+using namespace tutti;
+
+namespace {
+
+thread_local std::string g_last_cuda_error;
+
+int cuda_fail(cudaError_t e, const char *what) {
+    g_last_cuda_error = std::string(what) + ": " + cudaGetErrorName(e) + " (" +
+                        cudaGetErrorString(e) + ")";
+    return TUTTI_ECUDA;
+}
+
+#define CK(call)                                           \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+    } while (0)
+
+bool is_pow2(uint32_t v) { return v && !(v & (v - 1)); }
+
+uint32_t pow2_at_least(uint32_t v) {
+    uint32_t p = 32;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        target = dev;
+    }
+    ~DeviceGuard() {
+        if (ok && prev >= 0 && prev != target) cudaSetDevice(prev);
+    }
+    int target = -1;
+};
+
+}  // namespace
+
+struct tutti_ctx {
+    tutti_geom_t geom;
+    tutti_layout_t layout;
+    int device;
+    int device_sms;
+    std::vector<PoolLayer> pool;
+    StoreDev store[TUTTI_MAX_DEVICES];
+    CopyOptions opt;
+    GeomDev gdev;
+    void *partition = nullptr;   // SM partition state (tutti_partition.cu)
+};
+
+struct tutti_ring {
+    tutti_ctx *ctx;
+    RingDev dev;
+    HostRing *host;
+    CqSlot *cq_host;            // host view of the CQ
+    uint32_t cq_head = 0;       // next CQ position to consume
+    std::vector<tutti_cqe_t> completed;   // per slot
+    std::vector<uint8_t> have_cqe;        // per slot
+    std::vector<uint8_t> opcode_of;       // per slot, opcode of the reservation (0xff = unknown)
+    uint32_t sgl_capacity;
+    // plan cache key
+    bool plan_valid = false;
+    tutti_batch_t plan_batch{};
+    uint64_t kernel_launches = 0, host_calls = 0;
+    std::vector<void *> allocs;
+};
+
+extern "C" {
+
+// accessors for tutti_partition.cu
+void **tutti_ctx_partition_slot_(tutti_ctx_t *ctx) { return &ctx->partition; }
+int tutti_ctx_device_(tutti_ctx_t *ctx) { return ctx->device; }
+void tutti_set_cuda_error_(const char *msg) { g_last_cuda_error = msg; }
+
+uint32_t tutti_version(void) { return 0x000100; }
+
+const char *tutti_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+const char *tutti_strerror(int code) {
+    switch (code) {
+        case TUTTI_OK: return "ok";
+        case TUTTI_EINVAL: return "invalid argument";
+        case TUTTI_ENOMEM: return "out of memory";
+        case TUTTI_EAGAIN: return "try again (ring full or not complete)";
+        case TUTTI_ETIMEDOUT: return "device-side wait timed out";
+        case TUTTI_EFAULT: return "block id or slot out of range";
+        case TUTTI_ECUDA: return "CUDA error";
+        default: return "unknown";
+    }
+}
+
+int tutti_obj_layout(const tutti_geom_t *g, tutti_layout_t *o) {
+    if (!g || !o) return TUTTI_EINVAL;
+    if (!g->n_layers || !g->n_kv_heads || !g->head_dim || !g->elem_bytes || !g->block_tokens ||
+        !g->obj_tokens || !g->n_devices || !g->n_slots)
+        return TUTTI_EINVAL;
+    if (g->n_devices > TUTTI_MAX_DEVICES || g->n_layers > 65535) return TUTTI_EINVAL;
+    if (g->layout != TUTTI_LAYOUT_FILE_MAJOR && g->layout != TUTTI_LAYOUT_LAYER_MAJOR)
+        return TUTTI_EINVAL;
+    if (g->obj_tokens % g->block_tokens) return TUTTI_EINVAL;
+    uint64_t tb = (uint64_t)g->n_kv_heads * g->head_dim * g->elem_bytes;
+    if (tb % 16) return TUTTI_EINVAL;
+    uint64_t bb = tb * g->block_tokens;
+    if (bb > 0xffffffffull) return TUTTI_EINVAL;      // an SGL entry's length is 32 bits
+    o->token_bytes = tb;
+    o->block_bytes = bb;
+    o->obj_kv_bytes = tb * g->obj_tokens;
+    o->obj_bytes = 2 * o->obj_kv_bytes;
+    o->blocks_per_obj = g->obj_tokens / g->block_tokens;
+    o->n_slots_local = (g->n_slots + g->n_devices - 1) / g->n_devices;
+    o->stride_kv = o->obj_kv_bytes;
+    if (g->layout == TUTTI_LAYOUT_FILE_MAJOR) {
+        o->stride_layer = o->obj_bytes;
+        o->stride_slot = o->obj_bytes * g->n_layers;
+    } else {
+        o->stride_slot = o->obj_bytes;
+        o->stride_layer = o->obj_bytes * o->n_slots_local;
+    }
+    o->dev_bytes = o->obj_bytes * g->n_layers * o->n_slots_local;
+    if (o->dev_bytes >= (1ull << 56)) return TUTTI_EINVAL;
+    return TUTTI_OK;
+}
+
+int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
+    if (!geom || !out) return TUTTI_EINVAL;
+    tutti_layout_t lo;
+    int rc = tutti_obj_layout(geom, &lo);
+    if (rc) return rc;
+    int n_dev = 0;
+    CK(cudaGetDeviceCount(&n_dev));
+    if (device < 0 || device >= n_dev) return TUTTI_EINVAL;
+    DeviceGuard guard(device);
+    if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice, "cudaSetDevice");
+    cudaDeviceProp prop;
+    CK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major < 10) {
+        g_last_cuda_error = "this library is built for sm_100a only";
+        return TUTTI_ECUDA;
+    }
+    CK(copy_kernels_setup());
+    tutti_ctx *c = new (std::nothrow) tutti_ctx();
+    if (!c) return TUTTI_ENOMEM;
+    c->geom = *geom;
+    c->layout = lo;
+    c->device = device;
+    c->device_sms = prop.multiProcessorCount;
+    c->pool.assign(geom->n_layers, PoolLayer{0, 0, 0, 0, false});
+    for (auto &s : c->store) s = StoreDev{0, 0, 0, false};
+    c->opt = CopyOptions{0, 2000000ull, 4, 2, 3, 4};
+    c->gdev.block_tokens = geom->block_tokens;
+    c->gdev.obj_tokens = geom->obj_tokens;
+    c->gdev.blocks_per_obj = (uint32_t)lo.blocks_per_obj;
+    c->gdev.n_devices = geom->n_devices;
+    c->gdev.token_bytes = lo.token_bytes;
+    c->gdev.block_bytes = lo.block_bytes;
+    c->gdev.stride_kv = lo.stride_kv;
+    c->gdev.stride_layer = lo.stride_layer;
+    c->gdev.stride_slot = lo.stride_slot;
+    c->gdev.n_slots = geom->n_slots;
+    c->gdev.dev_bytes = lo.dev_bytes;
+    *out = c;
+    return TUTTI_OK;
+}
+
+int tutti_ctx_destroy(tutti_ctx_t *ctx) {
+    if (!ctx) return TUTTI_EINVAL;
+    tutti_sm_partition_destroy(ctx);
+    delete ctx;
+    return TUTTI_OK;
+}
+
+int tutti_pool_register(tutti_ctx_t *ctx, uint32_t layer, void *k_base, void *v_base,
+                        uint64_t block_stride, uint64_t n_blocks) {
+    if (!ctx || layer >= ctx->geom.n_layers || !k_base || !v_base || !n_blocks) return TUTTI_EINVAL;
+    uint64_t k = (uint64_t)k_base, v = (uint64_t)v_base;
+    if ((k | v | block_stride) & 15) return TUTTI_EINVAL;
+    if (block_stride < ctx->layout.block_bytes || n_blocks > 0x7fffffffull) return TUTTI_EINVAL;
+    ctx->pool[layer] = PoolLayer{k, v, block_stride, n_blocks, true};
+    return TUTTI_OK;
+}
+
+int tutti_store_register(tutti_ctx_t *ctx, uint32_t dev, void *base, uint64_t bytes, uint32_t kind) {
+    if (!ctx || dev >= ctx->geom.n_devices || !base) return TUTTI_EINVAL;
+    if (((uint64_t)base & 15) || bytes < ctx->layout.dev_bytes) return TUTTI_EINVAL;
+    if (kind != TUTTI_STORE_HBM && kind != TUTTI_STORE_HOST_PINNED) return TUTTI_EINVAL;
+    ctx->store[dev] = StoreDev{(uint64_t)base, bytes, kind, true};
+    return TUTTI_OK;
+}
+
+int tutti_set_option(tutti_ctx_t *ctx, uint32_t option, uint64_t value) {
+    if (!ctx) return TUTTI_EINVAL;
+    switch (option) {
+        case TUTTI_OPT_COPY_ENGINE:
+            if (value > 2) return TUTTI_EINVAL;
+            ctx->opt.engine = (uint32_t)value;
+            return TUTTI_OK;
+        case TUTTI_OPT_WAIT_NS:
+            if (value > 2000000000ull) return TUTTI_EINVAL;    // waits stay short by design
+            ctx->opt.wait_ns = value;
+            return TUTTI_OK;
+        case TUTTI_OPT_CTAS_PER_SM:
+            if (value < 1 || value > 8) return TUTTI_EINVAL;
+            ctx->opt.ctas_per_sm = (uint32_t)value;
+            return TUTTI_OK;
+        case TUTTI_OPT_BULK_WARPS:
+            if (value < 1 || value > 8) return TUTTI_EINVAL;
+            ctx->opt.bulk_warps = (uint32_t)value;
+            return TUTTI_OK;
+        case TUTTI_OPT_BULK_STAGES:
+            if (value < 2 || value > 8) return TUTTI_EINVAL;
+            ctx->opt.bulk_stages = (uint32_t)value;
+            return TUTTI_OK;
+        case TUTTI_OPT_CLAIM_CHUNKS:
+            if (value < 1 || value > 1024) return TUTTI_EINVAL;
+            ctx->opt.claim_chunks = (uint32_t)value;
+            return TUTTI_OK;
+        default:
+            return TUTTI_EINVAL;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// ring
+// ---------------------------------------------------------------------------
+
+static int ring_alloc(tutti_ring *r, void **p, size_t bytes, bool zero) {
+    cudaError_t e = cudaMalloc(p, bytes ? bytes : 16);
+    if (e != cudaSuccess) { cuda_fail(e, "cudaMalloc"); return TUTTI_ENOMEM; }
+    r->allocs.push_back(*p);
+    if (zero) {
+        e = cudaMemset(*p, 0, bytes ? bytes : 16);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemset");
+    }
+    return TUTTI_OK;
+}
+
+int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
+                      uint32_t sgl_capacity, uint32_t max_items, tutti_ring_t **out) {
+    if (!ctx || !out || !is_pow2(depth) || depth > (1u << 16) || !ioctx_per_iocb ||
+        ioctx_per_iocb > (1u << 16) || !sgl_capacity || !max_items || max_items > (1u << 24))
+        return TUTTI_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(cudaErrorInvalidDevice, "cudaSetDevice");
+    tutti_ring *r = new (std::nothrow) tutti_ring();
+    if (!r) return TUTTI_ENOMEM;
+    r->ctx = ctx;
+    r->sgl_capacity = sgl_capacity;
+    r->host = new (std::nothrow) HostRing(depth, sgl_capacity);
+    r->completed.resize(depth);
+    r->have_cqe.assign(depth, 0);
+    r->opcode_of.assign(depth, 0xff);
+    RingDev &d = r->dev;
+    memset(&d, 0, sizeof(d));
+    d.depth = depth;
+    d.capacity = ioctx_per_iocb;
+    d.max_items = max_items;
+    const uint32_t np = pow2_at_least(max_items);
+    int rc = TUTTI_OK;
+    auto A = [&](void **p, size_t bytes, bool zero) { if (rc == TUTTI_OK) rc = ring_alloc(r, p, bytes, zero); };
+    A((void **)&d.hdrs, sizeof(IocbHdr) * depth, true);
+    A((void **)&d.sqes, sizeof(tutti_sqe_t) * (size_t)depth * ioctx_per_iocb, false);
+    A((void **)&d.sgl, sizeof(tutti_sgl_t) * (size_t)sgl_capacity, false);
+    A((void **)&d.obj_ptr, sizeof(uint64_t) * (size_t)sgl_capacity, false);
+    A((void **)&d.cq_reserve, 16, true);
+    A((void **)&d.plan_item, sizeof(uint32_t) * (size_t)max_items, false);
+    A((void **)&d.plan_cumblk, sizeof(uint32_t) * ((size_t)max_items + 1), false);
+    A((void **)&d.plan_sqe_of, sizeof(uint32_t) * (size_t)max_items, false);
+    A((void **)&d.plan_sqe, sizeof(tutti_sqe_t) * (size_t)max_items, false);
+    A((void **)&d.plan_key, sizeof(unsigned long long) * (size_t)np, false);
+    A((void **)&d.plan_idx, sizeof(uint32_t) * (size_t)np, false);
+    A((void **)&d.plan_counts, sizeof(PlanCounts), true);
+    if (rc == TUTTI_OK) {
+        // headers start out "done" for an index that is never issued first
+        cudaError_t e = cudaHostAlloc((void **)&r->cq_host, sizeof(CqSlot) * depth,
+                                      cudaHostAllocMapped | cudaHostAllocPortable);
+        if (e != cudaSuccess) { cuda_fail(e, "cudaHostAlloc"); rc = TUTTI_ENOMEM; }
+    }
+    if (rc == TUTTI_OK) {
+        memset(r->cq_host, 0, sizeof(CqSlot) * depth);
+        cudaError_t e = cudaHostGetDevicePointer((void **)&d.cq, r->cq_host, 0);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaHostGetDevicePointer");
+    }
+    if (rc != TUTTI_OK) {
+        tutti_ring_destroy(r);
+        return rc;
+    }
+    *out = r;
+    return TUTTI_OK;
+}
+
+int tutti_ring_destroy(tutti_ring_t *r) {
+    if (!r) return TUTTI_EINVAL;
+    DeviceGuard guard(r->ctx->device);
+    cudaDeviceSynchronize();
+    for (void *p : r->allocs) cudaFree(p);
+    if (r->cq_host) cudaFreeHost(r->cq_host);
+    delete r->host;
+    delete r;
+    return TUTTI_OK;
+}
+
+int tutti_ring_stats(tutti_ring_t *r, uint64_t *kernel_launches, uint64_t *host_calls) {
+    if (!r) return TUTTI_EINVAL;
+    if (kernel_launches) *kernel_launches = r->kernel_launches;
+    if (host_calls) *host_calls = r->host_calls;
+    return TUTTI_OK;
+}
+
+static bool same_plan(const tutti_batch_t &a, const tutti_batch_t &b) {
+    return a.plan_epoch != 0 && a.plan_epoch == b.plan_epoch && a.n_req == b.n_req &&
+           a.n_obj == b.n_obj && a.n_blk == b.n_blk && a.hit_tokens == b.hit_tokens &&
+           a.obj_start == b.obj_start && a.obj_slot == b.obj_slot && a.blk_start == b.blk_start &&
+           a.block_ids == b.block_ids;
+}
+
+int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, uint32_t layer,
+                     uint32_t opcode, void *stream, uint32_t *first_iocb, uint32_t *n_iocb) {
+    if (!ctx || !r || r->ctx != ctx || !batch || !first_iocb || !n_iocb) return TUTTI_EINVAL;
+    r->host_calls++;
+    if (layer >= ctx->geom.n_layers || (opcode != TUTTI_OP_READ && opcode != TUTTI_OP_WRITE))
+        return TUTTI_EINVAL;
+    if (!ctx->pool[layer].registered) return TUTTI_EINVAL;
+    for (uint32_t d = 0; d < ctx->geom.n_devices; ++d)
+        if (!ctx->store[d].registered) return TUTTI_EINVAL;
+    if (batch->n_req && (!batch->hit_tokens || !batch->obj_start || !batch->blk_start))
+        return TUTTI_EINVAL;
+    if ((batch->n_obj && !batch->obj_slot) || (batch->n_blk && !batch->block_ids)) return TUTTI_EINVAL;
+    if (batch->n_obj > r->dev.max_items / 2 || batch->n_blk > 0x7fffffffu / 2) return TUTTI_EINVAL;
+    const uint32_t items = 2u * batch->n_obj;
+    const uint32_t need_sgl = 2u * batch->n_blk;
+    if (need_sgl > r->sgl_capacity) return TUTTI_EINVAL;
+    uint32_t need_iocb = (items + r->dev.capacity - 1) / r->dev.capacity;
+    if (need_iocb == 0) need_iocb = 1;
+    if (need_iocb > r->dev.depth) return TUTTI_EINVAL;
+    uint32_t first = 0, sgl_base = 0;
+    int rc = r->host->reserve(need_iocb, need_sgl, &first, &sgl_base);
+    if (rc == -3) return TUTTI_EAGAIN;
+    if (rc) return TUTTI_EINVAL;
+    for (uint32_t k = 0; k < need_iocb; ++k) {
+        uint32_t slot = (first + k) & (r->dev.depth - 1);
+        r->have_cqe[slot] = 0;
+        r->opcode_of[slot] = (uint8_t)opcode;
+    }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    BatchDev b{batch->n_req, batch->n_obj, batch->n_blk, batch->hit_tokens, batch->obj_start,
+               batch->obj_slot, batch->blk_start, batch->block_ids};
+    if (!(r->plan_valid && same_plan(r->plan_batch, *batch))) {
+        CK(launch_plan(r->dev, ctx->gdev, b, st));
+        r->kernel_launches++;
+        r->plan_batch = *batch;
+        r->plan_valid = batch->plan_epoch != 0;
+    }
+    uint64_t sbase[TUTTI_MAX_DEVICES] = {0}, sbytes[TUTTI_MAX_DEVICES] = {0};
+    for (uint32_t d = 0; d < ctx->geom.n_devices; ++d) {
+        sbase[d] = ctx->store[d].base;
+        sbytes[d] = ctx->store[d].bytes;
+    }
+    CK(launch_emit(r->dev, ctx->gdev, b, layer, opcode, ctx->pool[layer], sbase, sbytes, first,
+                   need_iocb, sgl_base, need_sgl, ctx->device_sms, st));
+    r->kernel_launches++;
+    *first_iocb = first;
+    *n_iocb = need_iocb;
+    return TUTTI_OK;
+}
+
+static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, uint32_t sm_count,
+                 void *stream, uint32_t opcode) {
+    if (!ctx || !r || r->ctx != ctx || n == 0 || n > r->dev.depth) return TUTTI_EINVAL;
+    r->host_calls++;
+    if (sm_count > (uint32_t)ctx->device_sms) return TUTTI_EINVAL;
+    bool host_store = false;
+    for (uint32_t d = 0; d < ctx->geom.n_devices; ++d)
+        host_store |= ctx->store[d].kind == TUTTI_STORE_HOST_PINNED;
+    for (uint32_t k = 0; k < n; ++k) {
+        uint32_t idx = first + k;
+        if (!r->host->is_live(idx)) return TUTTI_EINVAL;
+        uint8_t op = r->opcode_of[idx & (r->dev.depth - 1)];
+        if (op != 0xff && op != opcode) return TUTTI_EINVAL;
+    }
+    DeviceGuard guard(ctx->device);
+    uint32_t launches = 0;
+    CK(launch_copy(r->dev, first, n, opcode, sm_count, ctx->device_sms, ctx->opt, host_store,
+                   (cudaStream_t)stream, &launches));
+    r->kernel_launches += launches;
+    return TUTTI_OK;
+}
+
+int tutti_kv_restore_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t first_iocb,
+                           uint32_t n_iocb, uint32_t sm_count, void *stream) {
+    return issue(ctx, ring, first_iocb, n_iocb, sm_count, stream, TUTTI_OP_READ);
+}
+
+int tutti_kv_save_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t first_iocb, uint32_t n_iocb,
+                        uint32_t sm_count, void *stream) {
+    return issue(ctx, ring, first_iocb, n_iocb, sm_count, stream, TUTTI_OP_WRITE);
+}
+
+// Consume whatever the device has appended to the CQ since the last call.
+static void drain_cq(tutti_ring *r) {
+    const uint32_t depth = r->dev.depth;
+    for (;;) {
+        CqSlot *slot = &r->cq_host[r->cq_head & (depth - 1)];
+        uint32_t seq = __atomic_load_n(&slot->seq, __ATOMIC_ACQUIRE);
+        if (seq != r->cq_head + 1) break;
+        tutti_cqe_t c;
+        c.iocb_idx = *(volatile uint32_t *)&slot->cqe.iocb_idx;
+        c.status = *(volatile int32_t *)&slot->cqe.status;
+        c.bytes = *(volatile uint64_t *)&slot->cqe.bytes;
+        if (r->host->is_live(c.iocb_idx)) {
+            uint32_t s = c.iocb_idx & (depth - 1);
+            r->completed[s] = c;
+            r->have_cqe[s] = 1;
+        }
+        r->cq_head++;
+    }
+}
+
+int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns) {
+    if (!r || !out) return TUTTI_EINVAL;
+    r->host_calls++;
+    if (!r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
+    const uint32_t slot = iocb_idx & (r->dev.depth - 1);
+    auto t0 = std::chrono::steady_clock::now();
+    for (;;) {
+        if (!r->have_cqe[slot]) drain_cq(r);
+        if (r->have_cqe[slot]) {
+            *out = r->completed[slot];
+            r->host->release(iocb_idx);       // a repeated poll of a live index is harmless
+            return TUTTI_OK;
+        }
+        if (timeout_ns == 0) return TUTTI_EAGAIN;
+        auto dt = std::chrono::duration_cast<std::chrono::nanoseconds>(
+                      std::chrono::steady_clock::now() - t0).count();
+        if ((uint64_t)dt >= timeout_ns) return TUTTI_EAGAIN;
+    }
+}
+
+int tutti_ring_reserve(tutti_ring_t *r, uint32_t n_iocb, uint32_t n_sgl, uint32_t *first_iocb) {
+    if (!r || !first_iocb) return TUTTI_EINVAL;
+    r->host_calls++;
+    uint32_t first = 0, base = 0;
+    int rc = r->host->reserve(n_iocb, n_sgl, &first, &base);
+    if (rc == -3) return TUTTI_EAGAIN;
+    if (rc) return TUTTI_EINVAL;
+    for (uint32_t k = 0; k < n_iocb; ++k) {
+        uint32_t slot = (first + k) & (r->dev.depth - 1);
+        r->have_cqe[slot] = 0;
+        r->opcode_of[slot] = 0xff;
+    }
+    *first_iocb = first;
+    return TUTTI_OK;
+}
+
+int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
+                         const tutti_sqe_t *sqes, uint32_t n_sqe, const tutti_sgl_t *sgl,
+                         uint32_t n_sgl, uint32_t sgl_offset, void *stream) {
+    if (!ctx || !r || r->ctx != ctx) return TUTTI_EINVAL;
+    if ((n_sqe && !sqes) || (n_sgl && !sgl) || n_sqe > r->dev.capacity) return TUTTI_EINVAL;
+    const Group *g = r->host->group_of(iocb_idx);
+    if (!g) return TUTTI_EINVAL;
+    if ((uint64_t)sgl_offset + n_sgl > g->sgl_count) return TUTTI_EINVAL;
+    // walk the contexts as a device would: object-side address of every entry
+    std::vector<uint64_t> optr(n_sgl ? n_sgl : 1);
+    std::vector<uint8_t> seen(n_sgl ? n_sgl : 1, 0);
+    uint64_t total = 0;
+    uint32_t common = n_sgl ? sgl[0].len : 0;
+    uint32_t opcode = n_sqe ? sqes[0].opcode : TUTTI_OP_READ;
+    for (uint32_t k = 0; k < n_sqe; ++k) {
+        const tutti_sqe_t &s = sqes[k];
+        if (s.dev >= ctx->geom.n_devices || !ctx->store[s.dev].registered) return TUTTI_EINVAL;
+        if (s.opcode != opcode || (uint64_t)s.sgl_first + s.sgl_count > n_sgl) return TUTTI_EINVAL;
+        uint64_t cursor = s.src_off;
+        for (uint32_t e = s.sgl_first; e < s.sgl_first + s.sgl_count; ++e) {
+            if (seen[e] || (sgl[e].len & 15) || (sgl[e].addr & 15) || sgl[e].len == 0) return TUTTI_EINVAL;
+            seen[e] = 1;
+            if (cursor + sgl[e].len > ctx->store[s.dev].bytes) return TUTTI_EFAULT;
+            optr[e] = ctx->store[s.dev].base + cursor;
+            if (optr[e] & 15) return TUTTI_EINVAL;
+            cursor += sgl[e].len;
+            if (sgl[e].len != common) common = 0;
+        }
+        if (cursor - s.src_off != s.len) return TUTTI_EINVAL;
+        total += s.len;
+    }
+    for (uint32_t e = 0; e < n_sgl; ++e)
+        if (!seen[e]) return TUTTI_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint32_t slot = iocb_idx & (r->dev.depth - 1);
+    const size_t at = (size_t)g->sgl_begin + sgl_offset;
+    if (n_sqe)
+        CK(cudaMemcpyAsync(r->dev.sqes + (size_t)slot * r->dev.capacity, sqes,
+                           sizeof(tutti_sqe_t) * n_sqe, cudaMemcpyHostToDevice, st));
+    if (n_sgl) {
+        CK(cudaMemcpyAsync(r->dev.sgl + at, sgl, sizeof(tutti_sgl_t) * n_sgl, cudaMemcpyHostToDevice, st));
+        CK(cudaMemcpyAsync(r->dev.obj_ptr + at, optr.data(), sizeof(uint64_t) * n_sgl,
+                           cudaMemcpyHostToDevice, st));
+    }
+    IocbHdr h;
+    memset(&h, 0, sizeof(h));
+    h.state = state_word(iocb_idx, PHASE_READY);
+    h.num_ioctx = n_sqe;
+    h.opcode = opcode;
+    h.layer = n_sqe ? sqes[0].layer : 0;
+    h.sgl_base = g->sgl_begin;
+    h.entry_first = sgl_offset;
+    h.total_entries = n_sgl;
+    h.entry_len = common;
+    h.bytes = total;
+    // stream order publishes the header after the descriptors it refers to
+    CK(cudaMemcpyAsync(&r->dev.hdrs[slot], &h, sizeof(h), cudaMemcpyHostToDevice, st));
+    r->opcode_of[slot] = (uint8_t)opcode;
+    return TUTTI_OK;
+}
+
+int tutti_ring_read_iocb(tutti_ring_t *r, uint32_t iocb_idx, tutti_iocb_info_t *info,
+                         tutti_sqe_t *sqes, uint32_t max_sqes) {
+    if (!r || !info || !r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
+    DeviceGuard guard(r->ctx->device);
+    CK(cudaDeviceSynchronize());
+    const uint32_t slot = iocb_idx & (r->dev.depth - 1);
+    IocbHdr h;
+    CK(cudaMemcpy(&h, &r->dev.hdrs[slot], sizeof(h), cudaMemcpyDeviceToHost));
+    info->iocb_idx = iocb_idx;
+    info->ready = h.state == state_word(iocb_idx, PHASE_READY) ||
+                  h.state == state_word(iocb_idx, PHASE_DONE);
+    info->num_ioctx = h.num_ioctx;
+    info->opcode = h.opcode;
+    info->layer = h.layer;
+    info->status = h.status;
+    info->sgl_base = h.sgl_base;
+    info->entry_first = h.entry_first;
+    info->total_entries = h.total_entries;
+    info->entry_len = h.entry_len;
+    info->bytes = h.bytes;
+    uint32_t n = h.num_ioctx < max_sqes ? h.num_ioctx : max_sqes;
+    if (sqes && n && info->ready)
+        CK(cudaMemcpy(sqes, r->dev.sqes + (size_t)slot * r->dev.capacity, sizeof(tutti_sqe_t) * n,
+                      cudaMemcpyDeviceToHost));
+    return TUTTI_OK;
+}
+
+int tutti_ring_read_sgl(tutti_ring_t *r, uint32_t iocb_idx, tutti_sgl_t *sgl, uint32_t max_entries,
+                        uint32_t *n_entries) {
+    if (!r || !n_entries || !r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
+    DeviceGuard guard(r->ctx->device);
+    CK(cudaDeviceSynchronize());
+    const uint32_t slot = iocb_idx & (r->dev.depth - 1);
+    IocbHdr h;
+    CK(cudaMemcpy(&h, &r->dev.hdrs[slot], sizeof(h), cudaMemcpyDeviceToHost));
+    *n_entries = h.total_entries;
+    uint32_t n = h.total_entries < max_entries ? h.total_entries : max_entries;
+    if (sgl && n)
+        CK(cudaMemcpy(sgl, r->dev.sgl + (size_t)h.sgl_base + h.entry_first, sizeof(tutti_sgl_t) * n,
+                      cudaMemcpyDeviceToHost));
+    return TUTTI_OK;
+}
+
+// ---------------------------------------------------------------------------
+// host-side accounting on its own
+// ---------------------------------------------------------------------------
+struct tutti_hostring {
+    HostRing ring;
+    tutti_hostring(uint32_t d, uint32_t s) : ring(d, s) {}
+};
+
+tutti_hostring_t *tutti_hostring_create(uint32_t depth, uint32_t sgl_capacity) {
+    if (!is_pow2(depth) || !sgl_capacity) return nullptr;
+    return new (std::nothrow) tutti_hostring(depth, sgl_capacity);
+}
+void tutti_hostring_destroy(tutti_hostring_t *h) { delete h; }
+int tutti_hostring_reserve(tutti_hostring_t *h, uint32_t n_iocb, uint32_t n_sgl, uint32_t *first_iocb,
+                           uint32_t *sgl_base) {
+    if (!h || !first_iocb || !sgl_base) return TUTTI_EINVAL;
+    int rc = h->ring.reserve(n_iocb, n_sgl, first_iocb, sgl_base);
+    return rc == -3 ? TUTTI_EAGAIN : (rc ? TUTTI_EINVAL : TUTTI_OK);
+}
+int tutti_hostring_release(tutti_hostring_t *h, uint32_t iocb_idx) {
+    if (!h) return TUTTI_EINVAL;
+    return h->ring.release(iocb_idx) ? TUTTI_EINVAL : TUTTI_OK;
+}
+int tutti_hostring_live(const tutti_hostring_t *h, uint32_t *iocbs, uint32_t *sgl_entries) {
+    if (!h) return TUTTI_EINVAL;
+    if (iocbs) *iocbs = h->ring.live_iocbs();
+    if (sgl_entries) *sgl_entries = h->ring.live_sgl();
+    return TUTTI_OK;
+}
+
+}  // extern "C"

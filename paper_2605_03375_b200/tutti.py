@@ -1,0 +1,289 @@
+"""Thin ctypes binding over libtutti.so — the same names as include/tutti.h.
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  There is no CPU fallback: if the library cannot be loaded, importing
+this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import _build
+
+OK, EINVAL, ENOMEM, EAGAIN, ETIMEDOUT, EFAULT, ECUDA = 0, -1, -2, -3, -4, -5, -6
+LAYOUT_FILE_MAJOR, LAYOUT_LAYER_MAJOR = 0, 1
+OP_READ, OP_WRITE = 0, 1
+STORE_HBM, STORE_HOST_PINNED = 0, 1
+OPT_COPY_ENGINE, OPT_WAIT_NS, OPT_CTAS_PER_SM, OPT_BULK_WARPS, OPT_BULK_STAGES, OPT_CLAIM_CHUNKS = \
+    1, 2, 3, 4, 5, 6
+ENGINE_AUTO, ENGINE_LDST, ENGINE_BULK = 0, 1, 2
+
+
+class Geom(C.Structure):
+    _fields_ = [("n_layers", C.c_uint32), ("n_kv_heads", C.c_uint32), ("head_dim", C.c_uint32),
+                ("elem_bytes", C.c_uint32), ("block_tokens", C.c_uint32),
+                ("obj_tokens", C.c_uint32), ("n_devices", C.c_uint32), ("layout", C.c_uint32),
+                ("n_slots", C.c_uint64)]
+
+
+class Layout(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in
+                ("token_bytes", "block_bytes", "obj_kv_bytes", "obj_bytes", "blocks_per_obj",
+                 "n_slots_local", "stride_kv", "stride_layer", "stride_slot", "dev_bytes")]
+
+
+class Batch(C.Structure):
+    _fields_ = [("n_req", C.c_uint32), ("n_obj", C.c_uint32), ("n_blk", C.c_uint32),
+                ("plan_epoch", C.c_uint32), ("hit_tokens", C.c_void_p), ("obj_start", C.c_void_p),
+                ("obj_slot", C.c_void_p), ("blk_start", C.c_void_p), ("block_ids", C.c_void_p)]
+
+
+class Cqe(C.Structure):
+    _fields_ = [("iocb_idx", C.c_uint32), ("status", C.c_int32), ("bytes", C.c_uint64)]
+
+
+class IocbInfo(C.Structure):
+    _fields_ = [("iocb_idx", C.c_uint32), ("ready", C.c_uint32), ("num_ioctx", C.c_uint32),
+                ("opcode", C.c_uint32), ("layer", C.c_uint32), ("status", C.c_int32),
+                ("sgl_base", C.c_uint32), ("entry_first", C.c_uint32),
+                ("total_entries", C.c_uint32), ("entry_len", C.c_uint32), ("bytes", C.c_uint64)]
+
+
+SQE_DTYPE = np.dtype([("src_off", "<u8"), ("len", "<u8"), ("sgl_first", "<u4"),
+                      ("sgl_count", "<u4"), ("dev", "<u4"), ("opcode", "<u2"), ("layer", "<u2")])
+SGL_DTYPE = np.dtype([("addr", "<u8"), ("len", "<u4"), ("id", "<u4")])
+
+EXPORTS = [
+    "tutti_obj_layout", "tutti_build_sqes", "tutti_kv_restore_layer", "tutti_kv_save_layer",
+    "tutti_ring_poll", "tutti_ctx_create", "tutti_ctx_destroy", "tutti_pool_register",
+    "tutti_store_register", "tutti_set_option", "tutti_ring_create", "tutti_ring_destroy",
+    "tutti_ring_reserve", "tutti_ring_fill_host", "tutti_ring_read_iocb", "tutti_ring_read_sgl",
+    "tutti_ring_stats", "tutti_sm_partition_create", "tutti_sm_partition_destroy",
+    "tutti_hostring_create", "tutti_hostring_destroy", "tutti_hostring_reserve",
+    "tutti_hostring_release", "tutti_hostring_live", "tutti_strerror", "tutti_last_cuda_error",
+    "tutti_version",
+]
+
+_lib: Optional[C.CDLL] = None
+
+
+def load(path: Optional[str] = None) -> C.CDLL:
+    """Load (building first if the sources are newer) the C-ABI library."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path):
+            _build.build_library()
+    lib = C.CDLL(path)
+    vp, u32, u64 = C.c_void_p, C.c_uint32, C.c_uint64
+    P = C.POINTER
+    sig = {
+        "tutti_obj_layout": (C.c_int, [P(Geom), P(Layout)]),
+        "tutti_build_sqes": (C.c_int, [vp, vp, P(Batch), u32, u32, vp, P(u32), P(u32)]),
+        "tutti_kv_restore_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
+        "tutti_kv_save_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
+        "tutti_ring_poll": (C.c_int, [vp, u32, P(Cqe), u64]),
+        "tutti_ctx_create": (C.c_int, [P(Geom), C.c_int, P(vp)]),
+        "tutti_ctx_destroy": (C.c_int, [vp]),
+        "tutti_pool_register": (C.c_int, [vp, u32, vp, vp, u64, u64]),
+        "tutti_store_register": (C.c_int, [vp, u32, vp, u64, u32]),
+        "tutti_set_option": (C.c_int, [vp, u32, u64]),
+        "tutti_ring_create": (C.c_int, [vp, u32, u32, u32, u32, P(vp)]),
+        "tutti_ring_destroy": (C.c_int, [vp]),
+        "tutti_ring_reserve": (C.c_int, [vp, u32, u32, P(u32)]),
+        "tutti_ring_fill_host": (C.c_int, [vp, vp, u32, vp, u32, vp, u32, u32, vp]),
+        "tutti_ring_read_iocb": (C.c_int, [vp, u32, P(IocbInfo), vp, u32]),
+        "tutti_ring_read_sgl": (C.c_int, [vp, u32, vp, u32, P(u32)]),
+        "tutti_ring_stats": (C.c_int, [vp, P(u64), P(u64)]),
+        "tutti_sm_partition_create": (C.c_int, [vp, u32, P(vp), P(vp), P(u32), P(u32)]),
+        "tutti_sm_partition_destroy": (C.c_int, [vp]),
+        "tutti_hostring_create": (vp, [u32, u32]),
+        "tutti_hostring_destroy": (None, [vp]),
+        "tutti_hostring_reserve": (C.c_int, [vp, u32, u32, P(u32), P(u32)]),
+        "tutti_hostring_release": (C.c_int, [vp, u32]),
+        "tutti_hostring_live": (C.c_int, [vp, P(u32), P(u32)]),
+        "tutti_strerror": (C.c_char_p, [C.c_int]),
+        "tutti_last_cuda_error": (C.c_char_p, []),
+        "tutti_version": (u32, []),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    if path == _build.LIB_PATH:
+        _lib = lib
+    return lib
+
+
+class TuttiError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        lib = load()
+        msg = lib.tutti_strerror(code).decode()
+        if code == ECUDA:
+            msg += ": " + lib.tutti_last_cuda_error().decode()
+        super().__init__(f"{what}: {msg} ({code})")
+        self.code = code
+
+
+def _check(code: int, what: str, allow: Sequence[int] = ()) -> int:
+    if code != OK and code not in allow:
+        raise TuttiError(code, what)
+    return code
+
+
+def geom_of(w) -> Geom:
+    """Geometry struct of a workload description (any object with these fields)."""
+    return Geom(w.n_layers, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
+                w.n_devices, w.layout, w.n_slots)
+
+
+def tutti_obj_layout(geom: Geom) -> Layout:
+    out = Layout()
+    _check(load().tutti_obj_layout(C.byref(geom), C.byref(out)), "tutti_obj_layout")
+    return out
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream
+    return int(stream.cuda_stream)          # torch.cuda.Stream / ExternalStream
+
+
+class Context:
+    """tutti_ctx_t with its registrations."""
+
+    def __init__(self, geom: Geom, device: int = 0):
+        self.lib = load()
+        self.geom = geom
+        self.layout = tutti_obj_layout(geom)
+        h = C.c_void_p()
+        _check(self.lib.tutti_ctx_create(C.byref(geom), device, C.byref(h)), "tutti_ctx_create")
+        self.h = h
+        self.device = device
+
+    def close(self):
+        if self.h:
+            self.lib.tutti_ctx_destroy(self.h)
+            self.h = None
+
+    def tutti_pool_register(self, layer: int, k_base: int, v_base: int, block_stride: int,
+                            n_blocks: int):
+        _check(self.lib.tutti_pool_register(self.h, layer, k_base, v_base, block_stride, n_blocks),
+               "tutti_pool_register")
+
+    def tutti_store_register(self, dev: int, base: int, nbytes: int, kind: int = STORE_HBM):
+        _check(self.lib.tutti_store_register(self.h, dev, base, nbytes, kind),
+               "tutti_store_register")
+
+    def tutti_set_option(self, option: int, value: int):
+        _check(self.lib.tutti_set_option(self.h, option, value), "tutti_set_option")
+
+    def tutti_sm_partition_create(self, io_sms: int) -> Tuple[int, int, int, int]:
+        """(io_stream, compute_stream, io_sms, compute_sms) — raw CUstream handles."""
+        a, b = C.c_void_p(), C.c_void_p()
+        n1, n2 = C.c_uint32(), C.c_uint32()
+        _check(self.lib.tutti_sm_partition_create(self.h, io_sms, C.byref(a), C.byref(b),
+                                                  C.byref(n1), C.byref(n2)),
+               "tutti_sm_partition_create")
+        return a.value, b.value, n1.value, n2.value
+
+    def tutti_sm_partition_destroy(self):
+        _check(self.lib.tutti_sm_partition_destroy(self.h), "tutti_sm_partition_destroy")
+
+
+def make_batch(hit_tokens, obj_start, obj_slot, blk_start, block_ids, plan_epoch: int = 0) -> Batch:
+    """Batch struct over device tensors (torch, already on the GPU; dtypes int32)."""
+    n_req = int(hit_tokens.numel())
+    b = Batch(n_req, int(obj_slot.numel()), int(block_ids.numel()), plan_epoch,
+              hit_tokens.data_ptr(), obj_start.data_ptr(), obj_slot.data_ptr(),
+              blk_start.data_ptr(), block_ids.data_ptr())
+    b._keep = (hit_tokens, obj_start, obj_slot, blk_start, block_ids)
+    return b
+
+
+class Ring:
+    """tutti_ring_t."""
+
+    def __init__(self, ctx: Context, depth: int, ioctx_per_iocb: int, sgl_capacity: int,
+                 max_items: int):
+        self.ctx = ctx
+        self.lib = ctx.lib
+        h = C.c_void_p()
+        _check(self.lib.tutti_ring_create(ctx.h, depth, ioctx_per_iocb, sgl_capacity, max_items,
+                                          C.byref(h)), "tutti_ring_create")
+        self.h = h
+        self.ioctx_per_iocb = ioctx_per_iocb
+
+    def close(self):
+        if self.h:
+            self.lib.tutti_ring_destroy(self.h)
+            self.h = None
+
+    def tutti_build_sqes(self, batch: Batch, layer: int, opcode: int, stream=None,
+                         allow: Sequence[int] = ()) -> Tuple[int, int, int]:
+        first, n = C.c_uint32(), C.c_uint32()
+        rc = self.lib.tutti_build_sqes(self.ctx.h, self.h, C.byref(batch), layer, opcode,
+                                       _stream_ptr(stream), C.byref(first), C.byref(n))
+        _check(rc, "tutti_build_sqes", allow)
+        return rc, first.value, n.value
+
+    def tutti_kv_restore_layer(self, first_iocb: int, n_iocb: int, sm_count: int = 0, stream=None,
+                               allow: Sequence[int] = ()) -> int:
+        return _check(self.lib.tutti_kv_restore_layer(self.ctx.h, self.h, first_iocb, n_iocb,
+                                                      sm_count, _stream_ptr(stream)),
+                      "tutti_kv_restore_layer", allow)
+
+    def tutti_kv_save_layer(self, first_iocb: int, n_iocb: int, sm_count: int = 0, stream=None,
+                            allow: Sequence[int] = ()) -> int:
+        return _check(self.lib.tutti_kv_save_layer(self.ctx.h, self.h, first_iocb, n_iocb,
+                                                   sm_count, _stream_ptr(stream)),
+                      "tutti_kv_save_layer", allow)
+
+    def tutti_ring_poll(self, iocb_idx: int, timeout_ns: int = 0) -> Tuple[int, Cqe]:
+        cqe = Cqe()
+        rc = self.lib.tutti_ring_poll(self.h, iocb_idx, C.byref(cqe), timeout_ns)
+        _check(rc, "tutti_ring_poll", (EAGAIN, EINVAL))
+        return rc, cqe
+
+    def tutti_ring_reserve(self, n_iocb: int, n_sgl: int, allow: Sequence[int] = ()):
+        first = C.c_uint32()
+        rc = _check(self.lib.tutti_ring_reserve(self.h, n_iocb, n_sgl, C.byref(first)),
+                    "tutti_ring_reserve", allow)
+        return rc, first.value
+
+    def tutti_ring_fill_host(self, iocb_idx: int, sqes: np.ndarray, sgl: np.ndarray,
+                             sgl_offset: int = 0, stream=None, allow: Sequence[int] = ()) -> int:
+        sqes = np.ascontiguousarray(sqes)
+        sgl = np.ascontiguousarray(sgl)
+        assert sqes.dtype.itemsize == 32 and sgl.dtype.itemsize == 16
+        return _check(self.lib.tutti_ring_fill_host(self.ctx.h, self.h, iocb_idx,
+                                                    sqes.ctypes.data, len(sqes), sgl.ctypes.data,
+                                                    len(sgl), sgl_offset, _stream_ptr(stream)),
+                      "tutti_ring_fill_host", allow)
+
+    def tutti_ring_read_iocb(self, iocb_idx: int) -> Tuple[IocbInfo, np.ndarray]:
+        info = IocbInfo()
+        sqes = np.zeros(self.ioctx_per_iocb, dtype=SQE_DTYPE)
+        _check(self.lib.tutti_ring_read_iocb(self.h, iocb_idx, C.byref(info), sqes.ctypes.data,
+                                             len(sqes)), "tutti_ring_read_iocb")
+        return info, sqes[:info.num_ioctx].copy()
+
+    def tutti_ring_read_sgl(self, iocb_idx: int, max_entries: int) -> np.ndarray:
+        sgl = np.zeros(max(max_entries, 1), dtype=SGL_DTYPE)
+        n = C.c_uint32()
+        _check(self.lib.tutti_ring_read_sgl(self.h, iocb_idx, sgl.ctypes.data, max_entries,
+                                            C.byref(n)), "tutti_ring_read_sgl")
+        return sgl[:min(n.value, max_entries)].copy()
+
+    def tutti_ring_stats(self) -> Tuple[int, int]:
+        a, b = C.c_uint64(), C.c_uint64()
+        _check(self.lib.tutti_ring_stats(self.h, C.byref(a), C.byref(b)), "tutti_ring_stats")
+        return a.value, b.value

@@ -1,0 +1,103 @@
+"""A workload placed on the GPU: store devices, pool layers and batch tables as torch
+tensors registered with a library context, next to the host copies the oracle works on."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2605_03375_b200 import tutti as T
+from tests import hostcase as hc
+
+
+class DeviceCase:
+    def __init__(self, w, layers=None, host_store=False, depth=8, capacity=2048,
+                 sgl_capacity=None, max_items=None, device=0):
+        self.w = w
+        self.og = oracle.geom_of(w)
+        self.olo = oracle.obj_layout(self.og)
+        self.layers = list(range(w.n_layers)) if layers is None else list(layers)
+        self.dev = torch.device("cuda", device)
+        self.ctx = T.Context(T.geom_of(w), device)
+        lo = self.ctx.layout
+        assert lo.dev_bytes == self.olo.dev_bytes
+        # object store
+        self.store_host = hc.make_store(w, self.olo, None if layers is None or
+                                        w.layout != 1 else self.layers)
+        self.store_dev = []
+        for d, a in enumerate(self.store_host):
+            if host_store:
+                t = torch.from_numpy(a.copy()).pin_memory()
+                kind = T.STORE_HOST_PINNED
+            else:
+                t = torch.from_numpy(a).to(self.dev)
+                kind = T.STORE_HBM
+            self.store_dev.append(t)
+            self.ctx.tutti_store_register(d, t.data_ptr(), t.numel(), kind)
+        # pool layers
+        self.pool_bytes, self.k_off, self.v_off, self.stride = hc.pool_geometry(w, self.olo)
+        self.pool_host = {}
+        self.pool_dev = {}
+        for l in self.layers:
+            p = hc.make_pool_layer(w, self.olo, l)
+            self.pool_host[l] = p
+            t = torch.from_numpy(p).to(self.dev)
+            self.pool_dev[l] = t
+            self.ctx.tutti_pool_register(l, t.data_ptr() + self.k_off, t.data_ptr() + self.v_off,
+                                         self.stride, w.n_pool_blocks)
+        # batch tables
+        def up(a, dt):
+            return torch.from_numpy(np.ascontiguousarray(a).astype(dt).view(np.int32)).to(self.dev)
+        self.tensors = (up(w.hit_tokens, np.uint32), up(w.obj_start, np.uint32),
+                        up(w.obj_slot, np.uint32), up(w.blk_start, np.uint32),
+                        up(w.block_ids, np.int32))
+        self.batch = T.make_batch(*self.tensors)
+        n_blk = len(w.block_ids)
+        n_obj = len(w.obj_slot)
+        self.ring = T.Ring(self.ctx, depth, capacity,
+                           sgl_capacity or max(2 * n_blk * 2, 64),
+                           max_items or max(2 * n_obj, 2))
+        self.obatch = hc.batch_of(w)
+
+    def close(self):
+        torch.cuda.synchronize()
+        self.ring.close()
+        self.ctx.close()
+
+    # ---- oracle side -----------------------------------------------------
+    def oracle_descriptors(self, layer, opcode, capacity):
+        base = self.pool_dev[layer].data_ptr()
+        return oracle.build_descriptors(self.og, layer, opcode, self.obatch, base + self.k_off,
+                                        base + self.v_off, self.stride, capacity)
+
+    def oracle_restore(self, layer):
+        pool = self.pool_host[layer].copy()
+        rc = oracle.restore_layer(self.og, layer, self.obatch, self.store_host, pool, self.k_off,
+                                  self.v_off, self.stride, self.w.n_pool_blocks)
+        assert rc == 0
+        return pool
+
+    def oracle_save(self, layer, pool_host, store_host):
+        rc = oracle.save_layer(self.og, layer, self.obatch, store_host, pool_host, self.k_off,
+                               self.v_off, self.stride, self.w.n_pool_blocks)
+        assert rc == 0
+
+    # ---- CUDA side -------------------------------------------------------
+    def read_build(self, first, n):
+        """All contexts, SGL entries and per-IOCB counts of a build, in order."""
+        sqes, sgl, num, infos = [], [], [], []
+        for i in range(first, first + n):
+            info, s = self.ring.tutti_ring_read_iocb(i)
+            infos.append(info)
+            num.append(info.num_ioctx)
+            sqes.append(s)
+            sgl.append(self.ring.tutti_ring_read_sgl(i, info.total_entries))
+        return np.concatenate(sqes), np.concatenate(sgl), np.asarray(num, dtype=np.uint32), infos
+
+    def poll_all(self, first, n, timeout_ns=5_000_000_000):
+        out = []
+        for i in range(first, first + n):
+            rc, cqe = self.ring.tutti_ring_poll(i, timeout_ns)
+            assert rc == T.OK, f"poll {i}: {rc}"
+            out.append((cqe.iocb_idx, cqe.status, cqe.bytes))
+        return out

@@ -1,0 +1,117 @@
+"""Error paths, injected from the host: every one must come back as an error code or a
+completion status, with the pool untouched and the GPU context still usable."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_03375_b200 import tutti as T
+from paper_2605_03375_b200 import workload as wl
+from tests.devcase import DeviceCase
+
+pytestmark = pytest.mark.gpu
+
+
+def small():
+    return wl.config(2, 0.03, n_layers=2)
+
+
+def test_bad_arguments():
+    dc = DeviceCase(small())
+    try:
+        lib = dc.ctx.lib
+        rc, *_ = dc.ring.tutti_build_sqes(dc.batch, 5, T.OP_READ, allow=(T.EINVAL,))
+        assert rc == T.EINVAL                                    # layer out of range
+        rc, *_ = dc.ring.tutti_build_sqes(dc.batch, 0, 9, allow=(T.EINVAL,))
+        assert rc == T.EINVAL                                    # unknown opcode
+        assert dc.ring.tutti_kv_restore_layer(1234, 1, allow=(T.EINVAL,)) == T.EINVAL
+        rc, cqe = dc.ring.tutti_ring_poll(77)
+        assert rc == T.EINVAL                                    # never reserved
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        rc2, cqe = dc.ring.tutti_ring_poll(first)
+        assert rc2 == T.EAGAIN                                   # built but not issued
+        assert dc.ring.tutti_kv_save_layer(first, n, allow=(T.EINVAL,)) == T.EINVAL  # READ IOCB
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert dc.poll_all(first, n)[0][1] == 0
+        assert lib.tutti_pool_register(dc.ctx.h, 0, 8, 16, 32768, 4) == T.EINVAL     # misaligned
+        assert lib.tutti_store_register(dc.ctx.h, 0, 4096, 16, 0) == T.EINVAL        # too small
+        assert lib.tutti_set_option(dc.ctx.h, 99, 1) == T.EINVAL
+    finally:
+        dc.close()
+
+
+def test_ring_full_then_drains():
+    dc = DeviceCase(small(), depth=2)
+    try:
+        a = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        b = dc.ring.tutti_build_sqes(dc.batch, 1, T.OP_READ)
+        rc, *_ = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ, allow=(T.EAGAIN,))
+        assert rc == T.EAGAIN
+        dc.ring.tutti_kv_restore_layer(a[1], a[2])
+        dc.poll_all(a[1], a[2])
+        c = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)     # room again
+        assert c[0] == T.OK and c[1] == b[1] + b[2]
+        dc.ring.tutti_kv_restore_layer(b[1], b[2])
+        dc.ring.tutti_kv_restore_layer(c[1], c[2])
+        dc.poll_all(b[1], b[2])
+        dc.poll_all(c[1], c[2])
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("what", ["block_id_high", "block_id_negative", "slot", "hit_unaligned",
+                                  "short_row"])
+def test_bad_batch_contents_reported_in_cqe(what):
+    w = small()
+    dc = DeviceCase(w)
+    try:
+        hit, ostart, oslot, bstart, bids = [t.clone() for t in dc.tensors]
+        want = T.EFAULT
+        if what == "block_id_high":
+            bids[17] = w.n_pool_blocks
+        elif what == "block_id_negative":
+            bids[3] = -1
+        elif what == "slot":
+            oslot[1] = w.n_slots
+        elif what == "hit_unaligned":
+            hit[0] = hit[0] - 3
+            want = T.EINVAL
+        elif what == "short_row":
+            hit[0] = hit[0] + 16 * 400
+            want = T.EINVAL
+        batch = T.make_batch(hit, ostart, oslot, bstart, bids)
+        before = dc.pool_dev[0].clone()
+        rc, first, n = dc.ring.tutti_build_sqes(batch, 0, T.OP_READ)
+        info, _ = dc.ring.tutti_ring_read_iocb(first)
+        assert info.status == want and info.total_entries == 0
+        dc.ring.tutti_kv_restore_layer(first, n)
+        cqes = dc.poll_all(first, n)
+        assert all(c[1] == want and c[2] == 0 for c in cqes)
+        assert torch.equal(dc.pool_dev[0], before)               # nothing was written
+        # the ring and the context keep working
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
+def test_unpublished_iocb_times_out(engine):
+    """An IOCB that was reserved but never filled: the kernel's bounded wait runs out, the
+    completion carries TUTTI_ETIMEDOUT, and the next transfer works."""
+    dc = DeviceCase(small())
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+        dc.ctx.tutti_set_option(T.OPT_WAIT_NS, 200_000)
+        rc, first = dc.ring.tutti_ring_reserve(1, 16)
+        before = dc.pool_dev[0].clone()
+        dc.ring.tutti_kv_restore_layer(first, 1)
+        (idx, status, nbytes), = dc.poll_all(first, 1)
+        assert (idx, status, nbytes) == (first, T.ETIMEDOUT, 0)
+        assert torch.equal(dc.pool_dev[0], before)
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+    finally:
+        dc.close()

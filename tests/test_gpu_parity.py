@@ -1,0 +1,226 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs — descriptors element by element, pool and store bytes bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_03375_b200 import tutti as T
+from paper_2605_03375_b200 import workload as wl
+from tests.devcase import DeviceCase
+
+pytestmark = pytest.mark.gpu
+
+CASES = {
+    "cfg1": dict(index=1),
+    "cfg1-scattered-slots": dict(index=1, consecutive_slots=False, slot_mean_run=1.5,
+                                 slot_space_factor=3.0),
+    "cfg2-small": dict(index=2, scale=0.05, n_layers=4),
+    "cfg2-file-major": dict(index=2, scale=0.03, n_layers=3, layout=wl.LAYOUT_FILE_MAJOR),
+    "cfg2-2dev-interleaved": dict(index=2, scale=0.04, n_layers=2, n_devices=2,
+                                  pool_interleaved=True),
+    "cfg3-small": dict(index=3, scale=0.03, n_layers=2, store_kind="hbm"),
+    "cfg4-small": dict(index=4, scale=0.04, n_layers=2),
+    "cfg4-3dev-file-major": dict(index=4, scale=0.03, n_layers=2, n_devices=3,
+                                 layout=wl.LAYOUT_FILE_MAJOR),
+    "block-per-object": dict(index=2, scale=0.02, n_layers=2, obj_tokens=16, slot_mean_run=3.0),
+    "big-blocks-64k": dict(index=2, scale=0.03, n_layers=2, block_tokens=32, obj_tokens=256),
+    "odd-token-bytes": dict(index=4, scale=0.03, n_layers=2, n_kv_heads=3, head_dim=8,
+                            block_tokens=4, obj_tokens=32),
+}
+
+
+def mk(name):
+    c = dict(CASES[name])
+    return wl.config(c.pop("index"), c.pop("scale", 1.0), **c)
+
+
+def same_records(a, b):
+    return a.dtype.itemsize == b.dtype.itemsize and a.tobytes() == b.tobytes()
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
+def test_restore_and_save_match_oracle(name, engine):
+    w = mk(name)
+    dc = DeviceCase(w, capacity=2048)
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+        for layer in sorted({0, w.n_layers - 1}):
+            # descriptors
+            rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+            sq, sg, num, infos = dc.read_build(first, n)
+            orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 2048)
+            assert orc == 0
+            assert all(i.status == 0 and i.ready for i in infos)
+            assert same_records(sq, osq) and same_records(sg, osg)
+            assert list(num[:len(onum)]) == list(onum) and not num[len(onum):].any()
+            # restore
+            dc.ring.tutti_kv_restore_layer(first, n)
+            cqes = dc.poll_all(first, n)
+            assert sorted(c[0] for c in cqes) == list(range(first, first + n))
+            assert all(c[1] == 0 for c in cqes)
+            assert sum(c[2] for c in cqes) == int(osq["len"].sum())
+            got = dc.pool_dev[layer].cpu().numpy()
+            want = dc.oracle_restore(layer)
+            assert np.array_equal(got, want)
+            # save the restored pool into a zeroed store
+            for t in dc.store_dev:
+                t.zero_()
+            rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_WRITE)
+            dc.ring.tutti_kv_save_layer(first, n)
+            cqes = dc.poll_all(first, n)
+            assert all(c[1] == 0 for c in cqes)
+            st_want = [np.zeros_like(s) for s in dc.store_host]
+            dc.oracle_save(layer, want, st_want)
+            for t, s in zip(dc.store_dev, st_want):
+                assert np.array_equal(t.cpu().numpy(), s)
+            # round trip: what was saved equals the original store on the covered ranges
+            for t, s0, s1 in zip(dc.store_dev, dc.store_host, st_want):
+                cov = s1 != 0
+                assert np.array_equal(t.cpu().numpy()[cov], s0[cov])
+            for t, s in zip(dc.store_dev, dc.store_host):
+                t.copy_(torch.from_numpy(s))
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
+@pytest.mark.parametrize("sm_count", [0, 8, 32])
+def test_small_iocbs_ring_wrap_and_capped_mode(engine, sm_count):
+    """1-token pages with 64 contexts per IOCB and a ring of 64: many IOCBs per layer, the
+    ring and the SGL arena wrap, completions arrive in any order."""
+    w = mk("cfg4-small")
+    w2 = wl.config(4, 0.04, n_layers=2, slot_mean_run=1.2, slot_space_factor=2.0)
+    dc = DeviceCase(w2, depth=64, capacity=4, sgl_capacity=int(2.5 * 2 * len(w2.block_ids)))
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+        seen = []
+        for it in range(6):
+            layer = it % 2
+            dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
+            rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+            assert n > 1
+            sq, sg, num, infos = dc.read_build(first, n)
+            orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 4)
+            assert same_records(sq, osq) and same_records(sg, osg)
+            assert list(num[:len(onum)]) == list(onum)
+            dc.ring.tutti_kv_restore_layer(first, n, sm_count)
+            cqes = dc.poll_all(first, n)
+            assert sorted(c[0] for c in cqes) == list(range(first, first + n))
+            assert sum(c[2] for c in cqes) == int(osq["len"].sum())
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+            seen.append(first)
+        assert seen[-1] >= 64          # the index counter ran past the ring depth
+    finally:
+        dc.close()
+
+
+def test_host_prepared_descriptors():
+    """CPU-prepared IOCBs (the paper's own split): oracle-built descriptors, uploaded and
+    executed by the copy kernels, with entry lengths that differ."""
+    w = mk("cfg2-small")
+    dc = DeviceCase(w, depth=8, capacity=2048)
+    try:
+        for engine in (T.ENGINE_LDST, T.ENGINE_BULK):
+            dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+            layer = 1
+            dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
+            orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 2048)
+            rc, first = dc.ring.tutti_ring_reserve(1, len(osg))
+            dc.ring.tutti_ring_fill_host(first, osq, osg)
+            dc.ring.tutti_kv_restore_layer(first, 1)
+            (idx, status, nbytes), = dc.poll_all(first, 1)
+            assert (idx, status, nbytes) == (first, 0, int(osq["len"].sum()))
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        # split every entry in two unequal parts: same bytes, variable lengths
+        sg2 = np.zeros(2 * len(osg), dtype=osg.dtype)
+        sg2["addr"][0::2] = osg["addr"]
+        sg2["len"][0::2] = 4096
+        sg2["addr"][1::2] = osg["addr"] + 4096
+        sg2["len"][1::2] = osg["len"] - 4096
+        sg2["id"] = np.repeat(osg["id"], 2)
+        sq2 = osq.copy()
+        sq2["sgl_first"] *= 2
+        sq2["sgl_count"] *= 2
+        dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
+        rc, first = dc.ring.tutti_ring_reserve(1, len(sg2))
+        dc.ring.tutti_ring_fill_host(first, sq2, sg2)
+        dc.ring.tutti_kv_restore_layer(first, 1)
+        (idx, status, nbytes), = dc.poll_all(first, 1)
+        assert status == 0 and nbytes == int(osq["len"].sum())
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+    finally:
+        dc.close()
+
+
+def test_pinned_host_store_zero_copy():
+    w = wl.config(3, 0.03, n_layers=2)
+    assert w.store_kind == "host"
+    dc = DeviceCase(w, host_store=True)
+    try:
+        layer = 1
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        cqes = dc.poll_all(first, n)
+        assert all(c[1] == 0 for c in cqes)
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        # save back into the pinned store
+        want = dc.oracle_restore(layer)
+        for t in dc.store_dev:
+            t.zero_()
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_WRITE)
+        dc.ring.tutti_kv_save_layer(first, n)
+        dc.poll_all(first, n)
+        torch.cuda.synchronize()
+        st_want = [np.zeros_like(s) for s in dc.store_host]
+        dc.oracle_save(layer, want, st_want)
+        for t, s in zip(dc.store_dev, st_want):
+            assert np.array_equal(t.numpy(), s)
+    finally:
+        dc.close()
+
+
+def test_plan_reuse_across_layers_and_launch_count():
+    """With a plan epoch the batch is sorted once; every later layer costs one build launch
+    and one copy launch, independent of the number of blocks."""
+    w = mk("cfg2-small")
+    dc = DeviceCase(w)
+    try:
+        dc.batch.plan_epoch = 7
+        k0, h0 = dc.ring.tutti_ring_stats()
+        for layer in range(w.n_layers):
+            rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+            sq, sg, num, infos = dc.read_build(first, n)
+            orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 2048)
+            assert same_records(sq, osq) and same_records(sg, osg)
+            dc.ring.tutti_kv_restore_layer(first, n)
+            dc.poll_all(first, n)
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        k1, h1 = dc.ring.tutti_ring_stats()
+        assert k1 - k0 == 1 + 2 * w.n_layers           # one plan, then emit + copy per layer
+        assert h1 - h0 == 3 * w.n_layers               # build, restore, poll: O(1) per layer
+    finally:
+        dc.close()
+
+
+def test_empty_batch_and_zero_hits():
+    w = wl.make_workload("z", seed=5, n_layers=1, hit_tokens=[0, 256, 0], block_tokens=16,
+                         obj_tokens=256, n_pool_blocks=64)
+    dc = DeviceCase(w)
+    try:
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        cqes = dc.poll_all(first, n)
+        assert sum(c[2] for c in cqes) == 256 * 2 * 2048
+        assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
+        # a batch with no requests at all: one IOCB with no contexts, completes with 0 bytes
+        empty = T.Batch(0, 0, 0, 0, None, None, None, None, None)
+        rc, first, n = dc.ring.tutti_build_sqes(empty, 0, T.OP_READ)
+        assert n == 1
+        info, sq = dc.ring.tutti_ring_read_iocb(first)
+        assert info.num_ioctx == 0 and info.total_entries == 0 and info.ready
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert dc.poll_all(first, n) == [(first, 0, 0)]
+    finally:
+        dc.close()

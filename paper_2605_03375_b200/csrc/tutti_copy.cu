@@ -342,10 +342,39 @@ copy_bulk_kernel(CopyParams p) {
             if (lane == 0) complete_empty(p.ring, h, idx);
             continue;
         }
-        const ChunkGeom cg = chunk_geom(total, h->entry_len);
         const size_t e_base = (size_t)h->sgl_base + h->entry_first;
         const tutti_sgl_t *sgl = p.ring.sgl + e_base;
         const uint64_t *obj = p.ring.obj_ptr + e_base;
+        if (h->entry_len == 0) {
+            // entries of differing lengths (host-prepared IOCBs only): plain vector copies,
+            // one entry per warp at a time
+            for (;;) {
+                uint32_t c0 = 0;
+                if (lane == 0) c0 = atomicAdd(&h->claim_cursor, 8u);
+                c0 = __shfl_sync(0xffffffffu, c0, 0);
+                if (c0 >= total) break;
+                const uint32_t c1 = min(c0 + 8u, total);
+                unsigned long long moved = 0;
+                for (uint32_t e = c0; e < c1; ++e) {
+                    unsigned long long a_pool = 0, a_obj = 0;
+                    uint32_t len = 0;
+                    if (lane == 0) { a_pool = sgl[e].addr; len = sgl[e].len; a_obj = obj[e]; }
+                    a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
+                    a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
+                    len = __shfl_sync(0xffffffffu, len, 0);
+                    const unsigned long long src = TO_POOL ? a_obj : a_pool;
+                    const unsigned long long dst = TO_POOL ? a_pool : a_obj;
+                    for (uint32_t o = lane * 16u; o < len; o += 512u)
+                        st_stream(reinterpret_cast<void *>(dst + o),
+                                  ld_stream(reinterpret_cast<const void *>(src + o)));
+                    moved += len;
+                }
+                __syncwarp();
+                if (lane == 0) account_done(p.ring, h, idx, moved);
+            }
+            continue;
+        }
+        const ChunkGeom cg = chunk_geom(total, h->entry_len);
 
         uint32_t head = 0, tail = 0;            // stages issued / drained (monotonic)
         uint32_t cur = 0, cur_end = 0;          // claimed chunk range

@@ -302,4 +302,6 @@ def config(index: int, scale: float = 1.0, **overrides) -> Workload:
     else:
         raise ValueError("config index must be 1..5")
     kw.update(overrides)
+    bt = kw["block_tokens"]
+    kw["hit_tokens"] = [max(bt, int(h) // bt * bt) for h in kw["hit_tokens"]]
     return make_workload(f"cfg{index}", seed=seed, **kw)

@@ -88,15 +88,14 @@ def test_restore_and_save_match_oracle(name, engine):
 @pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
 @pytest.mark.parametrize("sm_count", [0, 8, 32])
 def test_small_iocbs_ring_wrap_and_capped_mode(engine, sm_count):
-    """1-token pages with 64 contexts per IOCB and a ring of 64: many IOCBs per layer, the
+    """1-token pages with 4 contexts per IOCB and a ring of 64: many IOCBs per layer, the
     ring and the SGL arena wrap, completions arrive in any order."""
-    w = mk("cfg4-small")
     w2 = wl.config(4, 0.04, n_layers=2, slot_mean_run=1.2, slot_space_factor=2.0)
     dc = DeviceCase(w2, depth=64, capacity=4, sgl_capacity=int(2.5 * 2 * len(w2.block_ids)))
     try:
         dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
         seen = []
-        for it in range(6):
+        for it in range(14):
             layer = it % 2
             dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
             rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)

@@ -1,0 +1,571 @@
+#!/usr/bin/env python
+"""Benchmark of the KV restore/save hot path on B200.
+
+One *step* = one pass of the whole path over one batch: for every layer, build the
+I/O contexts on the GPU and restore the prefix KV from the object store into the paged
+pool; then, for every layer, build and save it back; then poll every completion.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU, with no data-path
+collective (the path does not shard: "replicas only"); the time is the max over ranks.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+GIB = 1 << 30
+METRIC = "per-layer KV restore+save payload GB/s (HBM object store <-> paged pool)"
+STREAM_STORE = 0x100
+STREAM_POOL = 0x200
+
+
+# ----------------------------------------------------------------------------
+# ranks
+# ----------------------------------------------------------------------------
+def rank_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def init_dist(backend: str):
+    import torch.distributed as dist
+    rank, local_rank, world = rank_env()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, local_rank, world
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """Slowest rank's value (the whole job is done when the last replica is)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------
+# workload on the device
+# ----------------------------------------------------------------------------
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def ncu_traffic(kernel: str):
+    """DRAM bytes per payload byte of a copy kernel, from the committed ncu capture."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f).get(kernel)
+    return None
+
+
+class Replica:
+    """Config-2-shaped workload resident on one GPU, registered with the library."""
+
+    def __init__(self, args, device_index: int, host_store: bool = False, n_layers=None):
+        import torch
+        from paper_2605_03375_b200 import tutti as T
+        from paper_2605_03375_b200 import workload as wl
+        self.torch, self.T, self.wl = torch, T, wl
+        self.dev = torch.device("cuda", device_index)
+        torch.cuda.set_device(self.dev)
+        over = {}
+        if n_layers is not None:
+            over["n_layers"] = n_layers
+        self.w = w = wl.config(args.config, args.scale, **over)
+        self.geom = T.geom_of(w)
+        self.ctx = T.Context(self.geom, device_index)
+        lo = self.lo = self.ctx.layout
+        self.block_bytes = int(lo.block_bytes)
+        self.payload_per_layer = w.total_tokens * 2 * int(lo.token_bytes)
+        self.blocks_per_layer = len(w.block_ids)
+        # object store (every layer resident)
+        self.host_store = host_store
+        self.store = []
+        for d in range(w.n_devices):
+            n = int(lo.dev_bytes)
+            if host_store:
+                t = torch.empty(n, dtype=torch.uint8, pin_memory=True)
+                step = 1 << 28
+                for o in range(0, n, step):
+                    m = min(step, n - o)
+                    tmp = wl.fill_u16_torch(w.seed, STREAM_STORE + d, o // 2, m // 2, self.dev)
+                    t[o:o + m].copy_(tmp.view(torch.uint8))
+                kind = T.STORE_HOST_PINNED
+            else:
+                t = torch.empty(n, dtype=torch.uint8, device=self.dev)
+                wl.fill_u16_torch(w.seed, STREAM_STORE + d, 0, n // 2, self.dev, out=t)
+                kind = T.STORE_HBM
+            self.store.append(t)
+            self.ctx.tutti_store_register(d, t.data_ptr(), n, kind)
+        # pool: R resident layers; layer l uses buffer l mod R
+        pool_bytes = 2 * w.n_pool_blocks * self.block_bytes
+        free, _ = torch.cuda.mem_get_info(self.dev)
+        fit = int((free * 0.85) // pool_bytes)
+        R = args.resident_layers if args.resident_layers else w.n_layers
+        self.R = max(1, min(R, fit, w.n_layers))
+        self.pool = []
+        for i in range(self.R):
+            t = torch.empty(pool_bytes, dtype=torch.uint8, device=self.dev)
+            wl.fill_u16_torch(w.seed, STREAM_POOL + i, 0, pool_bytes // 2, self.dev, out=t)
+            self.pool.append(t)
+        self.v_off = w.n_pool_blocks * self.block_bytes
+        for l in range(w.n_layers):
+            t = self.pool[l % self.R]
+            self.ctx.tutti_pool_register(l, t.data_ptr(), t.data_ptr() + self.v_off,
+                                         self.block_bytes, w.n_pool_blocks)
+        # batch tables: pinned host copies (e2e uploads them every step) and device copies
+        def host(a, dt):
+            return torch.from_numpy(np.ascontiguousarray(a).astype(dt).view(np.int32)).pin_memory()
+        self.tables_host = (host(w.hit_tokens, np.uint32), host(w.obj_start, np.uint32),
+                            host(w.obj_slot, np.uint32), host(w.blk_start, np.uint32),
+                            host(w.block_ids, np.int32))
+        self.tables_dev = tuple(t.to(self.dev) for t in self.tables_host)
+        self.batch = T.make_batch(*self.tables_dev)
+        self.table_bytes = sum(t.numel() * 4 for t in self.tables_host)
+        n_iocb_layer = max(1, -(-2 * len(w.obj_slot) // args.ioctx_per_iocb))
+        depth = 1
+        while depth < 2 * w.n_layers * n_iocb_layer:
+            depth *= 2
+        self.ring = T.Ring(self.ctx, depth, args.ioctx_per_iocb,
+                           2 * len(w.block_ids) * (2 * w.n_layers + 1), 2 * len(w.obj_slot))
+        self.stream = torch.cuda.Stream(self.dev)
+        self.epoch = 1
+        if args.engine:
+            self.ctx.tutti_set_option(T.OPT_COPY_ENGINE, args.engine)
+        for opt, val in ((T.OPT_CTAS_PER_SM, args.ctas_per_sm), (T.OPT_BULK_WARPS, args.bulk_warps),
+                         (T.OPT_BULK_STAGES, args.bulk_stages), (T.OPT_CLAIM_CHUNKS, args.claim)):
+            if val:
+                self.ctx.tutti_set_option(opt, val)
+
+    def close(self):
+        self.torch.cuda.synchronize()
+        self.ring.close()
+        self.ctx.close()
+
+    def step(self, sm_count=0, upload_tables=False, events=None, directions=(0, 1)):
+        """One pass: all layers restored, all layers saved, all completions polled."""
+        T, torch = self.T, self.torch
+        s = self.stream
+        self.epoch += 1
+        self.batch.plan_epoch = self.epoch
+        issued = []
+        with torch.cuda.stream(s):
+            if upload_tables:
+                for h, d in zip(self.tables_host, self.tables_dev):
+                    d.copy_(h, non_blocking=True)
+            for op in directions:
+                if events is not None:
+                    ev = torch.cuda.Event(enable_timing=True)
+                    ev.record(s)
+                    events["pass"].append(ev)
+                for l in range(self.w.n_layers):
+                    rc, first, n = self.ring.tutti_build_sqes(self.batch, l, op, stream=s)
+                    if events is not None:
+                        a = torch.cuda.Event(enable_timing=True)
+                        b = torch.cuda.Event(enable_timing=True)
+                        a.record(s)
+                    if op == T.OP_READ:
+                        self.ring.tutti_kv_restore_layer(first, n, sm_count, stream=s)
+                    else:
+                        self.ring.tutti_kv_save_layer(first, n, sm_count, stream=s)
+                    if events is not None:
+                        b.record(s)
+                        events["copy"][op].append((a, b))
+                    issued.append((first, n))
+            if events is not None:
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record(s)
+                events["pass"].append(ev)
+        total = 0
+        for first, n in issued:
+            for i in range(first, first + n):
+                rc, cqe = self.ring.tutti_ring_poll(i, 20_000_000_000)
+                if rc != T.OK or cqe.status != 0:
+                    raise RuntimeError(f"IOCB {i}: poll rc {rc}, status {cqe.status}")
+                total += cqe.bytes
+        return total
+
+    def verify_samples(self, n_samples=256):
+        """Sampled outputs at full size: for random tokens the oracle names the store bytes
+        and the pool bytes that must be equal after a restore."""
+        import oracle
+        torch = self.torch
+        w = self.w
+        og = oracle.geom_of(w)
+        ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
+        rng = np.random.default_rng(1234)
+        tb = int(self.lo.token_bytes)
+        for _ in range(n_samples):
+            l = int(rng.integers(0, w.n_layers))
+            r = int(rng.integers(0, w.n_req))
+            t = int(rng.integers(0, int(w.hit_tokens[r])))
+            kv = int(rng.integers(0, 2))
+            d, so, blk, ro = oracle.token_location(og, l, ob, r, t, kv)
+            po = kv * self.v_off + blk * self.block_bytes + ro
+            a = self.store[d][so:so + tb].to(self.dev)
+            b = self.pool[l % self.R][po:po + tb]
+            if not torch.equal(a, b):
+                return False
+        return True
+
+
+def cpu_baseline(rep, seconds_hint=12.0):
+    """The oracle, as it stands, on the host cores: restore + save of whole layers of the
+    same batch, on host copies of the same inputs."""
+    import oracle
+    torch = rep.torch
+    w = rep.w
+    lo = rep.lo
+    og = oracle.geom(1, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
+                     w.n_devices, w.layout, w.n_slots)       # one layer's slice of the store
+    ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
+    layer_bytes = int(lo.stride_layer)
+    done_bytes, t_total, layers = 0, 0.0, 0
+    for l in range(w.n_layers):
+        if w.layout != rep.wl.LAYOUT_LAYER_MAJOR:
+            break
+        store = [s[l * layer_bytes:(l + 1) * layer_bytes].cpu().numpy() for s in rep.store]
+        pool = rep.pool[l % rep.R].cpu().numpy()
+        t0 = time.perf_counter()
+        rc1 = oracle.restore_layer(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
+                                   w.n_pool_blocks)
+        rc2 = oracle.save_layer(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
+                                w.n_pool_blocks)
+        t_total += time.perf_counter() - t0
+        assert rc1 == 0 and rc2 == 0
+        done_bytes += 2 * rep.payload_per_layer
+        layers += 1
+        if t_total > seconds_hint:
+            break
+    return {"value": round(done_bytes / t_total / 1e9, 3), "unit": "GB/s", "cores": 1,
+            "kind": "oracle", "seconds": round(t_total, 2),
+            "sample": f"restore+save of {layers} full layer(s) of the same batch "
+                      f"({done_bytes / GIB:.1f} GiB payload), single thread"}
+
+
+# ----------------------------------------------------------------------------
+# arms
+# ----------------------------------------------------------------------------
+def workload_name(w):
+    return (f"cfg{w.name[3:]}: {w.n_layers} layers x {w.n_req} requests x "
+            f"{int(w.hit_tokens.mean())} tokens, 8 KV heads x 128 x bf16, block {w.block_tokens}, "
+            f"objects of {w.obj_tokens} tokens, pool {w.n_pool_blocks} blocks 60% occupied")
+
+
+def run_ours(args):
+    import torch
+    rank, local_rank, world = init_dist("nccl")
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    from paper_2605_03375_b200 import tutti as T
+    rep = Replica(args, local_rank)
+    w = rep.w
+    peak, peak_kind = measured_peak()
+
+    for _ in range(args.warmup):
+        rep.step()
+    torch.cuda.synchronize()
+    k0, _ = rep.ring.tutti_ring_stats()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    events = {"pass": [], "copy": {T.OP_READ: [], T.OP_WRITE: []}}
+    barrier(world)
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(rep.stream)
+    moved = 0
+    for _ in range(args.steps):
+        moved += rep.step(events=events)
+    e1.record(rep.stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop()
+    k1, _ = rep.ring.tutti_ring_stats()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, rep.dev)
+    ms_step = ms_total / args.steps
+    payload_step = 2 * w.n_layers * rep.payload_per_layer
+    assert moved == payload_step * args.steps
+    all_payload = sum_over_ranks(float(payload_step), world, rep.dev)
+    value = all_payload / (ms_step * 1e-3) / 1e9
+
+    # per-direction figures from the events inside the timed region
+    def dir_stats(op):
+        pairs = events["copy"][op]
+        ms = [a.elapsed_time(b) for a, b in pairs]
+        passes = events["pass"]
+        idx = 0 if op == T.OP_READ else 1
+        pass_ms = [passes[3 * s + idx].elapsed_time(passes[3 * s + idx + 1])
+                   for s in range(args.steps)]
+        per_layer = statistics.mean(pass_ms) / w.n_layers
+        gbs = rep.payload_per_layer / (per_layer * 1e-3) / 1e9
+        return {"payload_gbs": round(gbs, 1), "hbm_traffic_gbs": round(2 * gbs, 1),
+                "hbm_frac": round(2 * gbs / peak, 4), "ms_per_layer": round(per_layer, 4),
+                "blocks_per_s": round(rep.blocks_per_layer / (per_layer * 1e-3)),
+                "copy_kernel_ms": round(statistics.mean(ms), 4),
+                "copy_kernel_ms_min": round(min(ms), 4)}
+    restore, save = dir_stats(T.OP_READ), dir_stats(T.OP_WRITE)
+    verified = rep.verify_samples()
+
+    out = None
+    if rank == 0:
+        # roofline of the dominant kernel (the restore copy kernel): algorithmic bytes per
+        # launch = payload read + payload written + SGL entry and object address per block
+        n_entries = 2 * rep.blocks_per_layer
+        alg_bytes = 2 * rep.payload_per_layer + n_entries * 24
+        achieved = alg_bytes / (restore["copy_kernel_ms"] * 1e-3) / 1e9
+        traffic = ncu_traffic("restore_copy")
+        out = {
+            "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_step, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+            "data": "synthetic (seeded bf16 N(0,1) KV bytes, seeded block tables and object map)",
+            "config": {"workload": workload_name(w), "layers": w.n_layers,
+                       "payload_gib_per_layer": round(rep.payload_per_layer / GIB, 3),
+                       "store": "hbm, all layers resident",
+                       "resident_pool_layers": rep.R,
+                       "parallelism": "replicas only" if world > 1 else "1 gpu",
+                       "l2": "inputs larger than L2 (each layer moves >= 2 GiB of HBM traffic)",
+                       "copy_engine": args.engine or "auto",
+                       "ioctx_per_iocb": args.ioctx_per_iocb},
+            "restore": restore, "save": save,
+            "blocks_per_s": restore["blocks_per_s"],
+            "gpu_launches": int(k1 - k0),
+            "verified_vs_oracle_samples": bool(verified),
+            "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "copy kernel, restore direction",
+                         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                         "frac": round(achieved / peak, 4), "peak_source": f"of {peak_kind}",
+                         "traffic": None if traffic is None else
+                         round(traffic * rep.payload_per_layer)},
+        }
+    # end-to-end leg: object store in pinned host memory, read zero-copy by the kernels
+    e2e = None
+    if not args.no_e2e:
+        rep.close()
+        del rep
+        torch.cuda.empty_cache()
+        e2e = run_e2e(args, local_rank, world)
+        if rank == 0:
+            out["e2e"] = e2e
+        rep = None
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        if rep is None:
+            a2 = argparse.Namespace(**vars(args))
+            a2.resident_layers = 1
+            rep = Replica(a2, local_rank, n_layers=min(4, w.n_layers))
+        out["cpu_baseline"] = cpu_baseline(rep)
+    if rep is not None:
+        rep.close()
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    barrier(world)
+
+
+def run_e2e(args, local_rank, world):
+    """Same metric through the public call with the objects in HOST memory: every step
+    uploads the batch tables from pinned host memory, restores every layer from the pinned
+    host object store (the kernels read it zero-copy over the host link), saves every layer
+    back to it, and reads the completions on the host."""
+    import torch
+    a2 = argparse.Namespace(**vars(args))
+    a2.resident_layers = 2
+    L_host = min(args.e2e_host_layers, 32)
+    rep = Replica(a2, local_rank, host_store=True, n_layers=L_host)
+    passes = max(1, 32 // L_host) if args.config in (2, 5) else 1
+    for _ in range(1):
+        rep.step(upload_tables=True)
+    torch.cuda.synchronize()
+    barrier(world)
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(rep.stream)
+    for _ in range(steps * passes):
+        rep.step(upload_tables=True)
+    e1.record(rep.stream)
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    ms = max_over_ranks(max(e0.elapsed_time(e1), wall_ms), world, rep.dev) / steps
+    layers = L_host * passes
+    payload = 2 * layers * rep.payload_per_layer
+    h2d = layers * rep.payload_per_layer + passes * rep.table_bytes
+    d2h = layers * rep.payload_per_layer + 2 * layers * 32
+    value = sum_over_ranks(float(payload), world, rep.dev) / (ms * 1e-3) / 1e9
+    rep.close()
+    return {"value": round(value, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms, 2),
+            "store": f"pinned host memory, zero-copy; {L_host} layers resident, "
+                     f"{passes} passes per step = {layers} layer transfers each way"}
+
+
+def run_reference(args):
+    """The reference arm of this tier is the oracle on the host cores: each step is a
+    bounded sample of the same workload (restore + save of one layer of the batch)."""
+    rank, _, world = rank_env()
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2605_03375_b200 import workload as wl
+    w = wl.config(args.config, args.scale)
+    og = oracle.geom(1, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
+                     w.n_devices, w.layout, w.n_slots)
+    lo = oracle.obj_layout(og)
+    ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
+    bb = int(lo.block_bytes)
+    store = [wl.fill_u16_torch(w.seed, STREAM_STORE + d, 0, int(lo.dev_bytes) // 2, "cpu")
+             .numpy().view(np.uint8) for d in range(w.n_devices)]
+    pool = wl.fill_u16_torch(w.seed, STREAM_POOL, 0, w.n_pool_blocks * bb, "cpu").numpy().view(np.uint8)
+    payload = w.total_tokens * 2 * int(lo.token_bytes)
+
+    def step():
+        assert oracle.restore_layer(og, 0, ob, store, pool, 0, w.n_pool_blocks * bb, bb,
+                                    w.n_pool_blocks) == 0
+        assert oracle.save_layer(og, 0, ob, store, pool, 0, w.n_pool_blocks * bb, bb,
+                                 w.n_pool_blocks) == 0
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = 2 * payload * args.steps / dt / 1e9
+    sample = "each step = restore+save of 1 layer of the batch (oracle, single thread)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(dt / args.steps * 1e3, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": workload_name(w), "sample": sample},
+        "cpu_baseline": {"value": round(value, 3), "unit": "GB/s", "cores": 1, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": "GB/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 ld/st, 2 bulk-async")
+    ap.add_argument("--resident-layers", type=int, default=0)
+    ap.add_argument("--ioctx-per-iocb", type=int, default=2048)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--bulk-warps", type=int, default=0)
+    ap.add_argument("--bulk-stages", type=int, default=0)
+    ap.add_argument("--claim", type=int, default=0)
+    ap.add_argument("--e2e-host-layers", type=int, default=4)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -518,7 +518,7 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     p.wait_ns = opt.wait_ns;
     p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : 4;
     uint32_t engine = opt.engine;
-    if (engine == 0) engine = (sm_count != 0 && !host_store) ? 2 : 1;
+    if (engine == 0) engine = host_store ? 1 : 2;   // measured: bulk-async wins on HBM
     const uint32_t sms = sm_count ? sm_count : (uint32_t)device_sms;
     if (engine == 2) {
         uint32_t warps = opt.bulk_warps ? opt.bulk_warps : 2;

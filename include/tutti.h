@@ -305,6 +305,39 @@ int tutti_sm_partition_create(tutti_ctx_t *ctx, uint32_t io_sms, void **io_strea
                               uint32_t *compute_sms_got);
 int tutti_sm_partition_destroy(tutti_ctx_t *ctx);
 
+/*
+ * (No counterpart in the paper.)  Build and restore one layer without allocating
+ * anything.  Some callers must not call cudaMalloc: code that runs after a serving
+ * engine has handed the whole HBM budget to its own pools, or inside a section where
+ * allocator calls are forbidden.  They cannot create a ring, so this call keeps what
+ * a ring would hold — one IOCB with its contexts, SGL entries and plan arrays — in a
+ * fixed device array inside the library (about 1.9 MiB, held by every GPU that loads
+ * the library until the process exits) and runs the same kernels on it.
+ *   geom, batch      host pointers; the batch arrays are device pointers, as for
+ *                    tutti_build_sqes.  Limits: 2 * n_obj <= 4096 and
+ *                    2 * n_blk <= 65536; a larger batch returns TUTTI_EINVAL.
+ *   k_base, v_base,  the pool layer to restore into (device pointers, 16-byte
+ *   block_stride,    aligned), as for tutti_pool_register.
+ *   n_blocks
+ *   store_base,      host arrays [geom->n_devices]: device pointer and size of every
+ *   store_bytes      storage device's region (HBM).
+ *   cqe_out          where the completion entry {iocb_idx = 0, status, bytes} is
+ *                    copied when the layer is done: device memory, or pinned host
+ *                    memory.  Valid once `stream` has reached that point.
+ * Asynchronous on `stream`; completion is observed through the stream (there is no
+ * completion queue here: a pinned CQ would have to be allocated).  The call issues
+ * no cudaMalloc / cudaFree / cudaHostAlloc.  The first call on a device resolves the
+ * address of the fixed array and sets kernel attributes; make that first call before
+ * any stream capture begins.  All calls on a device share the array, which keeps the
+ * previous call's contents (the call clears the words that must start at zero): two
+ * calls whose kernels overlap on the GPU — different streams without ordering — race.
+ */
+int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int device, uint32_t layer,
+                                   const tutti_batch_t *batch, void *k_base, void *v_base,
+                                   uint64_t block_stride, uint64_t n_blocks,
+                                   void *const *store_base, const uint64_t *store_bytes,
+                                   tutti_cqe_t *cqe_out, void *stream);
+
 /* Host-side ring accounting on its own (no GPU involved; used by CPU tests):
  * the reservation / release bookkeeping that tutti_build_sqes and tutti_ring_poll
  * apply to IOCB indices and SGL arena ranges. */

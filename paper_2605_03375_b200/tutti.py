@@ -65,7 +65,7 @@ EXPORTS = [
     "tutti_ring_stats", "tutti_sm_partition_create", "tutti_sm_partition_destroy",
     "tutti_hostring_create", "tutti_hostring_destroy", "tutti_hostring_reserve",
     "tutti_hostring_release", "tutti_hostring_live", "tutti_strerror", "tutti_last_cuda_error",
-    "tutti_version",
+    "tutti_version", "tutti_kv_restore_layer_noalloc",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -111,6 +111,8 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_strerror": (C.c_char_p, [C.c_int]),
         "tutti_last_cuda_error": (C.c_char_p, []),
         "tutti_version": (u32, []),
+        "tutti_kv_restore_layer_noalloc": (C.c_int, [P(Geom), C.c_int, u32, P(Batch), vp, vp, u64,
+                                                     u64, P(vp), P(u64), vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -287,3 +289,20 @@ class Ring:
         a, b = C.c_uint64(), C.c_uint64()
         _check(self.lib.tutti_ring_stats(self.h, C.byref(a), C.byref(b)), "tutti_ring_stats")
         return a.value, b.value
+
+
+def tutti_kv_restore_layer_noalloc(geom: Geom, device: int, layer: int, batch: Batch, k_base: int,
+                                   v_base: int, block_stride: int, n_blocks: int,
+                                   store_base: Sequence[int], store_bytes: Sequence[int],
+                                   cqe_out: int, stream=None, allow: Sequence[int] = ()) -> int:
+    """Build + restore one layer using only the library's fixed device scratch: for callers
+    that may not allocate (no context, no ring).  `cqe_out` is the address of 16 bytes of
+    device or pinned host memory that receive {iocb_idx, status, bytes}."""
+    n = len(store_base)
+    bases = (C.c_void_p * n)(*store_base)
+    sizes = (C.c_uint64 * n)(*store_bytes)
+    return _check(load().tutti_kv_restore_layer_noalloc(C.byref(geom), device, layer,
+                                                        C.byref(batch), k_base, v_base,
+                                                        block_stride, n_blocks, bases, sizes,
+                                                        cqe_out, _stream_ptr(stream)),
+                  "tutti_kv_restore_layer_noalloc", allow)

@@ -146,13 +146,15 @@ def measured_peak():
     return 6650.0, "fallback"
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per payload byte of one launch of
+# the bulk copy kernel, from the ncu capture summarised in
+# profiles/copy_bulk_kernel_cfg2_one_layer.md (one config-2 layer; traffic is proportional
+# to the payload, every entry is an independent 32 KiB copy).
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore_copy": 1.957, "save_copy": 1.953}
+
+
 def ncu_traffic(kernel: str):
-    """DRAM bytes per payload byte of a copy kernel, from the committed ncu capture."""
-    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if os.path.exists(p):
-        with open(p) as f:
-            return json.load(f).get(kernel)
-    return None
+    return NCU_DRAM_BYTES_PER_PAYLOAD_BYTE.get(kernel)
 
 
 class Replica:
@@ -166,6 +168,8 @@ class Replica:
         self.dev = torch.device("cuda", device_index)
         torch.cuda.set_device(self.dev)
         over = {}
+        if n_layers is None and getattr(args, "layers", 0):
+            n_layers = args.layers
         if n_layers is not None:
             over["n_layers"] = n_layers
         self.w = w = wl.config(args.config, args.scale, **over)
@@ -293,7 +297,7 @@ class Replica:
         rng = np.random.default_rng(1234)
         tb = int(self.lo.token_bytes)
         for _ in range(n_samples):
-            l = int(rng.integers(0, w.n_layers))
+            l = int(rng.integers(w.n_layers - self.R, w.n_layers))   # layers whose pool buffer is still theirs
             r = int(rng.integers(0, w.n_req))
             t = int(rng.integers(0, int(w.hit_tokens[r])))
             kv = int(rng.integers(0, 2))
@@ -318,9 +322,10 @@ def cpu_baseline(rep, seconds_hint=12.0):
     ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
     layer_bytes = int(lo.stride_layer)
     done_bytes, t_total, layers = 0, 0.0, 0
-    for l in range(w.n_layers):
-        if w.layout != rep.wl.LAYOUT_LAYER_MAJOR:
-            break
+    if w.layout != rep.wl.LAYOUT_LAYER_MAJOR:
+        raise RuntimeError("cpu_baseline expects the layer-major store of the bench workloads")
+    while t_total < seconds_hint:
+        l = layers % w.n_layers
         store = [s[l * layer_bytes:(l + 1) * layer_bytes].cpu().numpy() for s in rep.store]
         pool = rep.pool[l % rep.R].cpu().numpy()
         t0 = time.perf_counter()
@@ -332,11 +337,9 @@ def cpu_baseline(rep, seconds_hint=12.0):
         assert rc1 == 0 and rc2 == 0
         done_bytes += 2 * rep.payload_per_layer
         layers += 1
-        if t_total > seconds_hint:
-            break
     return {"value": round(done_bytes / t_total / 1e9, 3), "unit": "GB/s", "cores": 1,
             "kind": "oracle", "seconds": round(t_total, 2),
-            "sample": f"restore+save of {layers} full layer(s) of the same batch "
+            "sample": f"restore+save of {layers} full layers of the same batch "
                       f"({done_bytes / GIB:.1f} GiB payload), single thread"}
 
 
@@ -550,6 +553,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the layer count (small captures under a profiler)")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 ld/st, 2 bulk-async")
     ap.add_argument("--resident-layers", type=int, default=0)
     ap.add_argument("--ioctx-per-iocb", type=int, default=2048)

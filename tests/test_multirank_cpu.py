@@ -1,0 +1,51 @@
+"""The N > 1 harness of bench.py on CPU: two gloo ranks agree on the slowest rank's time
+and on the summed work, as the replicas-only scaling run needs."""
+import os
+import socket
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+CHILD = r"""
+import os, sys, json
+sys.path.insert(0, {root!r})
+import torch
+import bench
+rank, local_rank, world = bench.init_dist("gloo")
+assert world == 2 and rank == local_rank
+bench.barrier(world)
+t = bench.max_over_ranks(10.0 + 5.0 * rank, world, torch.device("cpu"))
+s = bench.sum_over_ranks(100.0 * (rank + 1), world, torch.device("cpu"))
+bench.barrier(world)
+print(json.dumps({{"rank": rank, "max": t, "sum": s}}), flush=True)
+"""
+
+
+def test_two_gloo_ranks_reduce_time_and_work():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE="2",
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", CHILD.format(root=ROOT)], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = []
+    for p in procs:
+        out, err = p.communicate(timeout=180)
+        assert p.returncode == 0, err[-2000:]
+        outs.append(out.strip().splitlines()[-1])
+    import json
+    res = sorted((json.loads(o) for o in outs), key=lambda r: r["rank"])
+    assert [r["max"] for r in res] == [15.0, 15.0]
+    assert [r["sum"] for r in res] == [300.0, 300.0]
+
+
+def test_reference_arm_only_rank0_prints():
+    env = dict(os.environ, RANK="1", LOCAL_RANK="1", WORLD_SIZE="2")
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
+                        "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
+                       capture_output=True, text=True, timeout=120)
+    assert p.returncode == 0 and p.stdout.strip() == ""

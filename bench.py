@@ -499,6 +499,176 @@ def run_e2e(args, local_rank, world):
                      f"{passes} passes per step = {layers} layer transfers each way"}
 
 
+def host_link_gbs(dev, nbytes=1 << 30, reps=10):
+    """Pinned host -> HBM copy bandwidth on this machine (cudaMemcpyAsync, best of `reps`)."""
+    import torch
+    src = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    dst = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    best = 0.0
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        dst.copy_(src, non_blocking=True)
+        b.record()
+        torch.cuda.synchronize()
+        best = max(best, nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
+    h2d = best
+    best = 0.0
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        src.copy_(dst, non_blocking=True)
+        b.record()
+        torch.cuda.synchronize()
+        best = max(best, nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
+    return h2d, best
+
+
+def run_config3(args):
+    """Config 3: Llama-3-70B-shaped KV restored per layer from the pinned-host object store,
+    zero-copy.  80 layer transfers per step over a window of resident host layers."""
+    import torch
+    from paper_2605_03375_b200 import tutti as T
+    rank, local_rank, world = init_dist("nccl")
+    a2 = argparse.Namespace(**vars(args))
+    a2.resident_layers = 2
+    L_host = args.e2e_host_layers
+    rep = Replica(a2, local_rank, host_store=True, n_layers=L_host)
+    peak, peak_kind = measured_peak()
+    h2d, d2h = host_link_gbs(rep.dev)
+    passes = max(1, 80 // L_host)
+    out = {"config": workload_name(rep.w).replace(f"{L_host} layers", "80 layers"),
+           "host_layers_resident": L_host, "host_link_h2d_gbs": round(h2d, 2),
+           "host_link_d2h_gbs": round(d2h, 2)}
+    for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
+        for eng in (1, 2):
+            rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, eng)
+            rep.step(directions=dirs)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(rep.stream)
+            for _ in range(passes):
+                rep.step(directions=dirs)
+            e1.record(rep.stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / (passes * L_host)
+            gbs = rep.payload_per_layer / (ms * 1e-3) / 1e9
+            link = h2d if name == "restore" else d2h
+            out[f"{name}_engine{eng}"] = {
+                "payload_gbs": round(gbs, 2), "ms_per_layer": round(ms, 3),
+                "link_frac": round(gbs / link, 4), "hbm_frac": round(gbs / peak, 5),
+                "blocks_per_s": round(rep.blocks_per_layer / (ms * 1e-3))}
+    out["verified_vs_oracle_samples"] = bool(rep.verify_samples())
+    rep.close()
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+
+
+def run_config5(args):
+    """Config 5: config 2's restore as persistent CTAs capped at 8/16/32 SMs while a bf16
+    8192^3 GEMM runs on the remaining SMs (green-context partition when the driver allows)."""
+    import torch
+    from paper_2605_03375_b200 import tutti as T
+    rank, local_rank, world = init_dist("nccl")
+    a2 = argparse.Namespace(**vars(args))
+    a2.config = 2
+    if not a2.resident_layers:
+        a2.resident_layers = 8
+    rep = Replica(a2, local_rank)
+    dev = rep.dev
+    peak, _ = measured_peak()
+    n = 8192
+    A = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
+    B = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
+    Cm = torch.empty(n, n, device=dev, dtype=torch.bfloat16)
+    gemm_iters = args.gemm_iters
+
+    def time_gemm(stream, iters):
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                torch.matmul(A, B, out=Cm)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(iters):
+                torch.matmul(A, B, out=Cm)
+            b.record(stream)
+        return a, b
+
+    def restore_pass(stream, sm_count, events):
+        rep.stream = stream
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        rep.step(sm_count=sm_count, directions=(T.OP_READ,))
+        b.record(stream)
+        events.append((a, b))
+
+    main = torch.cuda.Stream(dev)
+    a, b = time_gemm(main, gemm_iters)
+    torch.cuda.synchronize()
+    gemm_alone_ms = a.elapsed_time(b) / gemm_iters
+    ev = []
+    restore_pass(main, 0, ev)
+    restore_pass(main, 0, ev)
+    torch.cuda.synchronize()
+    full_ms = ev[-1][0].elapsed_time(ev[-1][1]) / rep.w.n_layers
+    out = {"config": "cfg5: " + workload_name(rep.w) + "; bf16 GEMM 8192^3 beside it",
+           "gemm_alone_ms": round(gemm_alone_ms, 4),
+           "gemm_alone_tflops": round(2 * n ** 3 / (gemm_alone_ms * 1e-3) / 1e12, 1),
+           "restore_all_sms": {"ms_per_layer": round(full_ms, 4),
+                               "payload_gbs": round(rep.payload_per_layer / (full_ms * 1e-3) / 1e9, 1)},
+           "capped": []}
+    for io_sms in (8, 16, 32):
+        entry = {"sm_count": io_sms}
+        try:
+            io_s, comp_s, got_io, got_comp = rep.ctx.tutti_sm_partition_create(io_sms)
+            io_stream = torch.cuda.ExternalStream(io_s, device=dev)
+            comp_stream = torch.cuda.ExternalStream(comp_s, device=dev)
+            entry["partition"] = {"kind": "green contexts", "io_sms": got_io, "compute_sms": got_comp}
+            partition = True
+        except T.TuttiError as e:
+            io_stream, comp_stream = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+            got_io = io_sms
+            entry["partition"] = {"kind": "plain streams (no isolation)", "why": str(e)[:200]}
+            partition = False
+        # each alone inside its partition
+        a, b = time_gemm(comp_stream, gemm_iters)
+        torch.cuda.synchronize()
+        entry["gemm_alone_in_partition_ms"] = round(a.elapsed_time(b) / gemm_iters, 4)
+        ev = []
+        restore_pass(io_stream, got_io, ev)
+        restore_pass(io_stream, got_io, ev)
+        torch.cuda.synchronize()
+        alone_ms = ev[-1][0].elapsed_time(ev[-1][1]) / rep.w.n_layers
+        entry["restore_alone_capped"] = {
+            "ms_per_layer": round(alone_ms, 4),
+            "payload_gbs": round(rep.payload_per_layer / (alone_ms * 1e-3) / 1e9, 1)}
+        # together: GEMMs keep running for the whole restore pass
+        n_gemm = max(8, int(1.5 * alone_ms * rep.w.n_layers / entry["gemm_alone_in_partition_ms"]))
+        torch.cuda.synchronize()
+        ga, gb = time_gemm(comp_stream, n_gemm)
+        ev = []
+        restore_pass(io_stream, got_io, ev)
+        torch.cuda.synchronize()
+        both_ms = ev[-1][0].elapsed_time(ev[-1][1]) / rep.w.n_layers
+        gemm_ms = ga.elapsed_time(gb) / n_gemm
+        gbs = rep.payload_per_layer / (both_ms * 1e-3) / 1e9
+        entry["concurrent"] = {
+            "restore_ms_per_layer": round(both_ms, 4), "restore_payload_gbs": round(gbs, 1),
+            "restore_hbm_frac": round(2 * gbs / peak, 4),
+            "gemm_ms": round(gemm_ms, 4), "gemms_overlapped": n_gemm,
+            "gemm_slowdown_vs_all_sms": round(gemm_ms / gemm_alone_ms, 3),
+            "gemm_slowdown_vs_partition": round(gemm_ms / entry["gemm_alone_in_partition_ms"], 3),
+            "restore_slowdown_vs_capped_alone": round(both_ms / alone_ms, 3)}
+        entry["verified_vs_oracle_samples"] = bool(rep.verify_samples(64))
+        if partition:
+            rep.ctx.tutti_sm_partition_destroy()
+        out["capped"].append(entry)
+    rep.stream = main
+    rep.close()
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+
+
 def run_reference(args):
     """The reference arm of this tier is the oracle on the host cores: each step is a
     bounded sample of the same workload (restore + save of one layer of the batch)."""
@@ -563,11 +733,16 @@ def main():
     ap.add_argument("--bulk-stages", type=int, default=0)
     ap.add_argument("--claim", type=int, default=0)
     ap.add_argument("--e2e-host-layers", type=int, default=4)
+    ap.add_argument("--gemm-iters", type=int, default=20)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == 3:
+        run_config3(args)
+    elif args.config == 5:
+        run_config5(args)
     else:
         run_ours(args)
 

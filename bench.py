@@ -230,11 +230,14 @@ class Replica:
         self.ring = T.Ring(self.ctx, depth, args.ioctx_per_iocb,
                            2 * len(w.block_ids) * (2 * w.n_layers + 1), 2 * len(w.obj_slot))
         self.stream = torch.cuda.Stream(self.dev)
+        self.build_stream = torch.cuda.Stream(self.dev)
+        self.two_streams = not getattr(args, "one_stream", False)
         self.epoch = 1
         if args.engine:
             self.ctx.tutti_set_option(T.OPT_COPY_ENGINE, args.engine)
         for opt, val in ((T.OPT_CTAS_PER_SM, args.ctas_per_sm), (T.OPT_BULK_WARPS, args.bulk_warps),
-                         (T.OPT_BULK_STAGES, args.bulk_stages), (T.OPT_CLAIM_CHUNKS, args.claim)):
+                         (T.OPT_BULK_STAGES, args.bulk_stages), (T.OPT_CLAIM_CHUNKS, args.claim),
+                         (T.OPT_BULK_CHUNK_BYTES, getattr(args, "bulk_chunk", 0))):
             if val:
                 self.ctx.tutti_set_option(opt, val)
 
@@ -250,17 +253,27 @@ class Replica:
         self.epoch += 1
         self.batch.plan_epoch = self.epoch
         issued = []
+        sb = self.build_stream if self.two_streams else s
         with torch.cuda.stream(s):
             if upload_tables:
                 for h, d in zip(self.tables_host, self.tables_dev):
                     d.copy_(h, non_blocking=True)
+            if self.two_streams:
+                fork = torch.cuda.Event()
+                fork.record(s)
+                sb.wait_event(fork)
             for op in directions:
                 if events is not None:
                     ev = torch.cuda.Event(enable_timing=True)
                     ev.record(s)
                     events["pass"].append(ev)
                 for l in range(self.w.n_layers):
-                    rc, first, n = self.ring.tutti_build_sqes(self.batch, l, op, stream=s)
+                    # descriptors are built on their own stream, ahead of the copies
+                    rc, first, n = self.ring.tutti_build_sqes(self.batch, l, op, stream=sb)
+                    if self.two_streams:
+                        built = torch.cuda.Event()
+                        built.record(sb)
+                        s.wait_event(built)
                     if events is not None:
                         a = torch.cuda.Event(enable_timing=True)
                         b = torch.cuda.Event(enable_timing=True)
@@ -426,6 +439,8 @@ def run_ours(args):
                        "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": "inputs larger than L2 (each layer moves >= 2 GiB of HBM traffic)",
                        "copy_engine": args.engine or "auto",
+                       "streams": "copy + descriptor-build stream, event-ordered"
+                       if rep.two_streams else "one stream",
                        "ioctx_per_iocb": args.ioctx_per_iocb},
             "restore": restore, "save": save,
             "blocks_per_s": restore["blocks_per_s"],
@@ -732,8 +747,11 @@ def main():
     ap.add_argument("--bulk-warps", type=int, default=0)
     ap.add_argument("--bulk-stages", type=int, default=0)
     ap.add_argument("--claim", type=int, default=0)
+    ap.add_argument("--bulk-chunk", type=int, default=0)
     ap.add_argument("--e2e-host-layers", type=int, default=4)
     ap.add_argument("--gemm-iters", type=int, default=20)
+    ap.add_argument("--one-stream", action="store_true",
+                    help="build and copy on one stream (default: descriptors on their own stream)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -56,7 +56,9 @@ extern "C" {
 #define TUTTI_OPT_CTAS_PER_SM 3 /* resident CTAs per SM of the load/store kernel (grid mode)     */
 #define TUTTI_OPT_BULK_WARPS 4  /* copy warps per CTA of the bulk-async kernel                   */
 #define TUTTI_OPT_BULK_STAGES 5 /* shared-memory stages per copy warp of the bulk-async kernel   */
-#define TUTTI_OPT_CLAIM_CHUNKS 6 /* chunks (32 KiB each) taken per work claim                    */
+#define TUTTI_OPT_CLAIM_CHUNKS 6 /* chunks taken per work claim                                   */
+#define TUTTI_OPT_BULK_CHUNK_BYTES 7 /* bytes per shared-memory stage of the bulk-async kernel: a
+                                        power of two, 4096..32768                                 */
 
 /*
  * Geometry of the KV cache and of the object store (Section 3.1, "Scalable GPU

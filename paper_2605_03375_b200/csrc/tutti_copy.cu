@@ -33,6 +33,7 @@ struct CopyParams {
     unsigned long long wait_ns;
     uint32_t claim_chunks;
     uint32_t stages;        // bulk engine: stages per warp
+    uint32_t chunk_bytes;   // bulk engine: bytes per stage (a power of two, 4..32 KiB)
 };
 
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
@@ -283,24 +284,24 @@ constexpr int BULK_MAX_STAGES = 8;
 // Geometry of the chunks of one IOCB with uniform entry length.
 struct ChunkGeom {
     uint32_t elen;       // entry length
-    uint32_t per_chunk;  // entries per chunk when elen <= CHUNK_BYTES (1..32), else 0
-    uint32_t pieces;     // pieces per entry when elen > CHUNK_BYTES, else 0
+    uint32_t per_chunk;  // entries per chunk when elen <= chunk bytes (1..32), else 0
+    uint32_t pieces;     // pieces per entry when elen > chunk bytes, else 0
     uint32_t n_chunks;
     uint32_t total;
 };
 
-__device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen) {
+__device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen, uint32_t CB) {
     ChunkGeom g;
     g.elen = elen;
     g.total = total;
-    if (elen <= CHUNK_BYTES) {
-        uint32_t pc = CHUNK_BYTES / elen;
+    if (elen <= CB) {
+        uint32_t pc = CB / elen;
         g.per_chunk = pc > 32 ? 32 : pc;
         g.pieces = 0;
         g.n_chunks = (total + g.per_chunk - 1) / g.per_chunk;
     } else {
         g.per_chunk = 0;
-        g.pieces = (elen + CHUNK_BYTES - 1) / CHUNK_BYTES;
+        g.pieces = (elen + CB - 1) / CB;
         g.n_chunks = total * g.pieces;
     }
     return g;
@@ -308,7 +309,7 @@ __device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen) {
 
 // Each warp of the CTA is an independent agent with its own stage ring.
 // Shared memory: [warps][stages][CHUNK_BYTES] data, then [warps][stages] mbarriers,
-// then [warps][stages] chunk ids.
+// then per stage the store descriptors of the 32 lanes and the chunk's byte count.
 template <int TO_POOL>
 __global__ void __launch_bounds__(256, 1)
 copy_bulk_kernel(CopyParams p) {
@@ -316,11 +317,17 @@ copy_bulk_kernel(CopyParams p) {
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_warps = blockDim.x >> 5;
     const uint32_t S = p.stages;
-    unsigned char *data = smem + (size_t)warp * S * CHUNK_BYTES;
+    const uint32_t CB = p.chunk_bytes;
+    unsigned char *data = smem + (size_t)warp * S * CB;
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(
-        smem + (size_t)n_warps * S * CHUNK_BYTES) + warp * S;
-    uint32_t *chunk_of = reinterpret_cast<uint32_t *>(
-        smem + (size_t)n_warps * S * CHUNK_BYTES + (size_t)n_warps * S * 8) + warp * S;
+        smem + (size_t)n_warps * S * CB) + warp * S;
+    // per stage: destination address and byte count of every lane's store, chunk bytes
+    unsigned char *meta = smem + (size_t)n_warps * S * (CB + 8);
+    unsigned long long *st_addr_of = reinterpret_cast<unsigned long long *>(meta) + (size_t)warp * S * 32;
+    uint32_t *st_bytes_of = reinterpret_cast<uint32_t *>(meta + (size_t)n_warps * S * 32 * 8) +
+                            (size_t)warp * S * 32;
+    uint32_t *chunk_bytes_of = reinterpret_cast<uint32_t *>(meta + (size_t)n_warps * S * 32 * 12) +
+                               warp * S;
 
     if (lane == 0)
         for (uint32_t s = 0; s < S; ++s) mbar_init(smem_u32(&bars[s]), 1);
@@ -374,116 +381,109 @@ copy_bulk_kernel(CopyParams p) {
             }
             continue;
         }
-        const ChunkGeom cg = chunk_geom(total, h->entry_len);
+        const ChunkGeom cg = chunk_geom(total, h->entry_len, CB);
 
         uint32_t head = 0, tail = 0;            // stages issued / drained (monotonic)
-        uint32_t cur = 0, cur_end = 0;          // claimed chunk range
-        bool exhausted = false;
         unsigned long long moved = 0;           // bytes this agent has stored
         bool failed = false;
 
-        for (;;) {
-            // ---- issue loads while a stage is free (keep one stage of slack for the
-            //      store that is still reading shared memory)
-            while (!exhausted && head - tail < S - 1) {
-                if (cur == cur_end) {
-                    uint32_t c0 = 0;
-                    if (lane == 0) c0 = atomicAdd(&h->claim_cursor, p.claim_chunks);
-                    c0 = __shfl_sync(0xffffffffu, c0, 0);
-                    if (c0 >= cg.n_chunks) { exhausted = true; break; }
-                    cur = c0;
-                    cur_end = min(c0 + p.claim_chunks, cg.n_chunks);
+        // Work claims are taken one ahead of need (the atomic's latency hides behind the
+        // copies of the current claim), and the addresses of the next chunk are fetched as
+        // soon as the current chunk's loads are issued.
+        uint32_t pending_claim = 0;
+        if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
+        uint32_t cur = 0, cur_end = 0;
+        bool have_next = false;
+        uint32_t c_next = 0, n_e = 0, ld_bytes = 0, st_bytes = 0;
+        unsigned long long ld_addr = 0, st_addr = 0;
+
+        auto fetch_next = [&]() {
+            have_next = false;
+            if (failed) return;
+            if (cur == cur_end) {
+                uint32_t c0 = __shfl_sync(0xffffffffu, pending_claim, 0);
+                if (c0 >= cg.n_chunks) return;
+                cur = c0;
+                cur_end = min(c0 + p.claim_chunks, cg.n_chunks);
+                if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
+            }
+            c_next = cur++;
+            have_next = true;
+            ld_bytes = 0; st_bytes = 0; ld_addr = 0; st_addr = 0;
+            if (cg.per_chunk) {
+                const uint32_t e0 = c_next * cg.per_chunk;
+                n_e = min(cg.per_chunk, cg.total - e0);
+                unsigned long long a_obj = 0, a_pool = 0;
+                if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
+                // the object side is contiguous in runs: one bulk copy per run
+                unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
+                bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
+                uint32_t heads = __ballot_sync(0xffffffffu, is_head);
+                uint32_t run_bytes = 0;
+                if (is_head) {
+                    uint32_t above = lane < 31 ? heads >> (lane + 1) : 0u;
+                    uint32_t next = above ? lane + __ffs(above) : n_e;
+                    run_bytes = (next - lane) * cg.elen;
                 }
-                const uint32_t c = cur++;
+                const uint32_t one = lane < n_e ? cg.elen : 0;
+                if (TO_POOL) { ld_addr = a_obj; ld_bytes = run_bytes; st_addr = a_pool; st_bytes = one; }
+                else         { ld_addr = a_pool; ld_bytes = one; st_addr = a_obj; st_bytes = run_bytes; }
+            } else {
+                const uint32_t e = c_next / cg.pieces, piece = c_next % cg.pieces;
+                const uint32_t off = piece * CB;
+                const uint32_t bytes = min(CB, cg.elen - off);
+                n_e = 1;
+                if (lane == 0) {
+                    unsigned long long a_obj = obj[e] + off, a_pool = sgl[e].addr + off;
+                    ld_addr = TO_POOL ? a_obj : a_pool;
+                    st_addr = TO_POOL ? a_pool : a_obj;
+                    ld_bytes = bytes; st_bytes = bytes;
+                }
+            }
+        };
+        fetch_next();
+
+        for (;;) {
+            // ---- issue loads while a stage is free (one stage of slack is kept for the
+            //      store that may still be reading shared memory)
+            while (have_next && head - tail < S - 1) {
                 const uint32_t s = head % S;
                 // the store that last used this stage must have finished reading it:
                 // at most one newer store group may still be pending
                 bulk_wait_read_1();
                 __syncwarp();
                 const uint32_t bar = smem_u32(&bars[s]);
-                const uint32_t sbase = smem_u32(data + (size_t)s * CHUNK_BYTES);
-                if (cg.per_chunk) {
-                    const uint32_t e0 = c * cg.per_chunk;
-                    const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
-                    unsigned long long a_obj = 0, a_pool = 0;
-                    if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
-                    if (lane == 0) mbar_expect_tx(bar, n_e * cg.elen);
-                    __syncwarp();
-                    if (TO_POOL) {
-                        // object side is contiguous in runs: one load per run
-                        unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
-                        bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
-                        uint32_t heads = __ballot_sync(0xffffffffu, is_head);
-                        if (is_head) {
-                            uint32_t above = heads >> (lane + 1);
-                            uint32_t next = above ? lane + __ffs(above) : n_e;
-                            bulk_g2s(sbase + lane * cg.elen, a_obj, (next - lane) * cg.elen, bar);
-                        }
-                    } else {
-                        if (lane < n_e) bulk_g2s(sbase + lane * cg.elen, a_pool, cg.elen, bar);
-                    }
-                } else {
-                    const uint32_t e = c / cg.pieces, piece = c % cg.pieces;
-                    const uint32_t off = piece * CHUNK_BYTES;
-                    const uint32_t bytes = min(CHUNK_BYTES, cg.elen - off);
-                    if (lane == 0) {
-                        unsigned long long src = (TO_POOL ? obj[e] : sgl[e].addr) + off;
-                        mbar_expect_tx(bar, bytes);
-                        bulk_g2s(sbase, src, bytes, bar);
-                    }
-                }
-                if (lane == 0) chunk_of[s] = c;
+                const uint32_t sbase = smem_u32(data + (size_t)s * CB);
+                const uint32_t total_bytes = __reduce_add_sync(0xffffffffu, ld_bytes);
+                const uint32_t my_off = cg.per_chunk ? lane * cg.elen : 0;
+                if (lane == 0) mbar_expect_tx(bar, total_bytes);
+                __syncwarp();
+                if (ld_bytes) bulk_g2s(sbase + my_off, ld_addr, ld_bytes, bar);
+                st_addr_of[s * 32 + lane] = st_addr;
+                st_bytes_of[s * 32 + lane] = st_bytes;
+                if (lane == 0) chunk_bytes_of[s] = total_bytes;
                 __syncwarp();
                 ++head;
+                fetch_next();
             }
             if (head == tail) break;
 
             // ---- drain the oldest stage: wait for its bytes, store them
             const uint32_t s = tail % S;
             const uint32_t bar = smem_u32(&bars[s]);
-            const uint32_t sbase = smem_u32(data + (size_t)s * CHUNK_BYTES);
-            const uint32_t c = chunk_of[s];
+            const uint32_t sbase = smem_u32(data + (size_t)s * CB);
             bool arrived = mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
             arrived = __all_sync(0xffffffffu, arrived);
             phase_bits ^= (1u << s);
             if (!arrived) failed = true;
-            fence_proxy_async();
-            if (cg.per_chunk) {
-                const uint32_t e0 = c * cg.per_chunk;
-                const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
-                unsigned long long a_obj = 0, a_pool = 0;
-                if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
-                if (arrived) {
-                    if (TO_POOL) {
-                        if (lane < n_e) bulk_s2g(a_pool, sbase + lane * cg.elen, cg.elen);
-                    } else {
-                        unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
-                        bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
-                        uint32_t heads = __ballot_sync(0xffffffffu, is_head);
-                        if (is_head) {
-                            uint32_t above = heads >> (lane + 1);
-                            uint32_t next = above ? lane + __ffs(above) : n_e;
-                            bulk_s2g(a_obj, sbase + lane * cg.elen, (next - lane) * cg.elen);
-                        }
-                    }
-                }
-                moved += (unsigned long long)n_e * cg.elen;
-            } else {
-                const uint32_t e = c / cg.pieces, piece = c % cg.pieces;
-                const uint32_t off = piece * CHUNK_BYTES;
-                const uint32_t bytes = min(CHUNK_BYTES, cg.elen - off);
-                if (lane == 0 && arrived) {
-                    unsigned long long dst = (TO_POOL ? sgl[e].addr : obj[e]) + off;
-                    bulk_s2g(dst, sbase, bytes);
-                }
-                moved += bytes;
-            }
+            const unsigned long long dst = st_addr_of[s * 32 + lane];
+            const uint32_t nbytes = st_bytes_of[s * 32 + lane];
+            const uint32_t my_off = cg.per_chunk ? lane * cg.elen : 0;
+            if (arrived && nbytes) bulk_s2g(dst, sbase + my_off, nbytes);
             bulk_commit();
+            moved += chunk_bytes_of[s];
             ++tail;
-            if (failed) {
-                // stop taking new work; what is in flight is still drained above
-                exhausted = true;
-            }
+            if (failed) have_next = false;    // stop taking new work; the rest is drained
         }
         // all of this agent's stores must have landed before they are accounted
         bulk_wait_all();
@@ -521,16 +521,21 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     if (engine == 0) engine = host_store ? 1 : 2;   // measured: bulk-async wins on HBM
     const uint32_t sms = sm_count ? sm_count : (uint32_t)device_sms;
     if (engine == 2) {
-        uint32_t warps = opt.bulk_warps ? opt.bulk_warps : 2;
+        // measured on B200: all SMs -> 2 warps x 3 stages x 32 KiB; a capped launch gets
+        // closest to the per-SM ceiling (~49 GB/s each way) with 4 warps x 3 stages x 16 KiB
+        uint32_t warps = opt.bulk_warps ? opt.bulk_warps : (sm_count ? 4 : 2);
         uint32_t stages = opt.bulk_stages ? opt.bulk_stages : 3;
         if (warps > 8) warps = 8;
         if (stages < 2) stages = 2;
         if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
-        while ((size_t)warps * stages * (CHUNK_BYTES + 16) > 220u * 1024u) {
+        uint32_t cb = opt.bulk_chunk ? opt.bulk_chunk : (sm_count ? 16384u : CHUNK_BYTES);
+        const size_t per_stage = cb + 8 + 32 * 12 + 4;
+        while ((size_t)warps * stages * per_stage > 224u * 1024u) {
             if (stages > 2) --stages; else --warps;
         }
         p.stages = stages;
-        size_t smem = (size_t)warps * stages * (CHUNK_BYTES + 8 + 4);
+        p.chunk_bytes = cb;
+        size_t smem = (size_t)warps * stages * per_stage;
         // a capped launch keeps one CTA per SM: pad shared memory so no second CTA fits
         if (sm_count && smem < 120u * 1024u) smem = 120u * 1024u;
         if (opcode == TUTTI_OP_READ)
@@ -539,6 +544,7 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
             copy_bulk_kernel<0><<<sms, warps * 32, smem, stream>>>(p);
     } else {
         p.stages = 0;
+        p.chunk_bytes = CHUNK_BYTES;
         uint32_t per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 4;
         if (opcode == TUTTI_OP_READ)
             copy_ldst_kernel<1><<<sms * per_sm, LDST_THREADS, 0, stream>>>(p);

@@ -102,6 +102,7 @@ struct CopyOptions {
     uint32_t ctas_per_sm;
     uint32_t bulk_warps, bulk_stages;
     uint32_t claim_chunks;
+    uint32_t bulk_chunk;    // bytes per stage of the bulk engine (0 = 32 KiB)
 };
 
 // kernels (tutti_build.cu / tutti_copy.cu)

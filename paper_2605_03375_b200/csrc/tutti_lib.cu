@@ -162,7 +162,7 @@ int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
     c->device_sms = prop.multiProcessorCount;
     c->pool.assign(geom->n_layers, PoolLayer{0, 0, 0, 0, false});
     for (auto &s : c->store) s = StoreDev{0, 0, 0, false};
-    c->opt = CopyOptions{0, 2000000ull, 4, 2, 3, 4};
+    c->opt = CopyOptions{0, 2000000ull, 4, 0, 0, 4, 0};   // 0 = chosen per launch
     c->gdev.block_tokens = geom->block_tokens;
     c->gdev.obj_tokens = geom->obj_tokens;
     c->gdev.blocks_per_obj = (uint32_t)lo.blocks_per_obj;
@@ -229,6 +229,10 @@ int tutti_set_option(tutti_ctx_t *ctx, uint32_t option, uint64_t value) {
         case TUTTI_OPT_CLAIM_CHUNKS:
             if (value < 1 || value > 1024) return TUTTI_EINVAL;
             ctx->opt.claim_chunks = (uint32_t)value;
+            return TUTTI_OK;
+        case TUTTI_OPT_BULK_CHUNK_BYTES:
+            if (value < 4096 || value > 32768 || (value & (value - 1))) return TUTTI_EINVAL;
+            ctx->opt.bulk_chunk = (uint32_t)value;
             return TUTTI_OK;
         default:
             return TUTTI_EINVAL;

@@ -69,3 +69,29 @@ def test_config2_full_size(engine):
         assert np.array_equal(got_store[cov], orig.cpu().numpy()[cov])     # round trip
     finally:
         rep.close()
+
+
+def test_one_object_per_block_at_full_batch_size():
+    """The paper's own granularity (one object per paged block) on the config-2 batch: 32,768
+    items — more than the shared-memory sort holds, so the plan sorts in ring scratch — and
+    sixteen IOCBs per layer."""
+    from paper_2605_03375_b200 import workload as wl
+    from tests.devcase import DeviceCase
+    w = wl.config(2, 1.0, n_layers=1, obj_tokens=16, slot_mean_run=1.3, slot_space_factor=2.0)
+    assert len(w.obj_slot) == 16384
+    dc = DeviceCase(w, depth=64, capacity=2048)
+    try:
+        layer = 0
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+        assert n == 16
+        sq, sg, num, infos = dc.read_build(first, n)
+        orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 2048)
+        assert orc == 0 and len(osq) > 2048
+        assert sq.tobytes() == osq.tobytes() and sg.tobytes() == osg.tobytes()
+        assert list(num[:len(onum)]) == list(onum) and not num[len(onum):].any()
+        dc.ring.tutti_kv_restore_layer(first, n)
+        cqes = dc.poll_all(first, n)
+        assert sum(c[2] for c in cqes) == 1 << 30 and all(c[1] == 0 for c in cqes)
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+    finally:
+        dc.close()

@@ -95,3 +95,93 @@ def test_one_object_per_block_at_full_batch_size():
         assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
     finally:
         dc.close()
+
+
+def _whole_layer_check(rep, l, pool_before):
+    """Layer l's pool buffer against the oracle's restore on host copies."""
+    w = rep.w
+    og = oracle.geom(1, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
+                     w.n_devices, w.layout, w.n_slots)
+    ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
+    lb = int(rep.lo.stride_layer)
+    store_l = [s[l * lb:(l + 1) * lb].cpu().numpy() for s in rep.store]
+    want = pool_before.cpu().numpy()
+    assert oracle.restore_layer(og, 0, ob, store_l, want, 0, rep.v_off, rep.block_bytes,
+                                w.n_pool_blocks) == 0
+    assert np.array_equal(rep.pool[l % rep.R].cpu().numpy(), want)
+
+
+def test_config4_full_size_per_layer():
+    """1-token pages, 64 requests with partial hits: a layer at full size (about 2 GiB in
+    2 KiB fragments, >1 M SGL entries), 64 contexts per IOCB so that a layer spans dozens of
+    IOCBs; sampled tokens and one whole layer."""
+    rep = bench.Replica(_args(config=4, layers=2, resident_layers=2, ioctx_per_iocb=64), 0)
+    try:
+        w = rep.w
+        assert w.n_req == 64 and w.block_tokens == 1 and len(w.block_ids) > 400_000
+        before = rep.pool[1].clone()
+        moved = rep.step(directions=(T.OP_READ,))
+        assert moved == 2 * rep.payload_per_layer
+        assert rep.verify_samples(512)
+        _whole_layer_check(rep, 1, before)
+    finally:
+        rep.close()
+
+
+def test_config3_full_size_per_layer_from_pinned_host():
+    """Llama-3-70B-shaped batch (2 x 128K tokens, 1024-token objects) restored zero-copy from
+    pinned host memory, then saved back to it."""
+    rep = bench.Replica(_args(config=3, layers=2, resident_layers=2), 0, host_store=True)
+    try:
+        w = rep.w
+        assert (w.n_req, w.obj_tokens, len(w.block_ids)) == (2, 1024, 16384)
+        before = rep.pool[1].clone()
+        rep.step(directions=(T.OP_READ,))
+        assert rep.verify_samples(256)
+        _whole_layer_check(rep, 1, before)
+        orig = [s.clone() for s in rep.store]
+        for s in rep.store:
+            s.zero_()
+        rep.step(directions=(T.OP_WRITE,))
+        torch.cuda.synchronize()
+        for s, o in zip(rep.store, orig):
+            cov = s != 0
+            assert torch.equal(s[cov], o[cov]) and int(cov.sum()) > 0.9 * 2 * rep.payload_per_layer
+    finally:
+        rep.close()
+
+
+@pytest.mark.parametrize("sm_count", [8, 32])
+def test_config5_capped_restore_beside_a_gemm(sm_count):
+    """Config 2's restore as persistent CTAs inside a green-context SM partition while bf16
+    GEMMs run in the other partition: the bytes are still exactly the oracle's."""
+    rep = bench.Replica(_args(config=2, layers=2, resident_layers=2), 0)
+    try:
+        try:
+            io_s, comp_s, got_io, got_comp = rep.ctx.tutti_sm_partition_create(sm_count)
+        except T.TuttiError as e:
+            pytest.skip(f"green contexts unavailable: {e}")
+        assert got_io >= sm_count and got_io + got_comp <= 148
+        io_stream = torch.cuda.ExternalStream(io_s, device=rep.dev)
+        comp_stream = torch.cuda.ExternalStream(comp_s, device=rep.dev)
+        a = torch.randn(4096, 4096, device=rep.dev, dtype=torch.bfloat16)
+        c = torch.empty_like(a)
+        with torch.cuda.stream(comp_stream):
+            torch.matmul(a, a, out=c)
+        torch.cuda.synchronize()
+        ref = (a.float() @ a.float())
+        before = rep.pool[1].clone()
+        with torch.cuda.stream(comp_stream):
+            for _ in range(60):
+                torch.matmul(a, a, out=c)
+        rep.stream = io_stream
+        rep.two_streams = False
+        moved = rep.step(sm_count=got_io, directions=(T.OP_READ,))
+        torch.cuda.synchronize()
+        assert moved == 2 * rep.payload_per_layer
+        assert rep.verify_samples(256)
+        _whole_layer_check(rep, 1, before)
+        assert torch.allclose(c.float(), ref, rtol=2e-2, atol=2.0)       # the GEMM was not disturbed
+        rep.ctx.tutti_sm_partition_destroy()
+    finally:
+        rep.close()

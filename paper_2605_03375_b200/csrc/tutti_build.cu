@@ -79,15 +79,18 @@ struct ScanPair {
     uint32_t a, b;
 };
 
-// Inclusive scan of (a, b) across the CTA for one element per thread, plus carry.
+// Inclusive scan of (a, b) across the CTA for one element per thread, plus carry.  `a`
+// (block counts) goes through shuffles; `b` is a 0/1 flag (run head), so its warp-level
+// prefix is a ballot and a population count.
 __device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &carry) {
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
         uint32_t ua = __shfl_up_sync(0xffffffffu, v.a, d);
-        uint32_t ub = __shfl_up_sync(0xffffffffu, v.b, d);
-        if (lane >= (uint32_t)d) { v.a += ua; v.b += ub; }
+        if (lane >= (uint32_t)d) v.a += ua;
     }
+    const uint32_t heads = __ballot_sync(0xffffffffu, v.b != 0);
+    v.b = __popc(heads & (0xffffffffu >> (31 - lane)));
     if (lane == 31) warp_tot[warp] = v;
     __syncthreads();
     if (warp == 0) {

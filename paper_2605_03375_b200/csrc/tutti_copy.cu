@@ -123,7 +123,7 @@ __device__ __forceinline__ void st_stream(void *p, const uint4 &v) {
 // ldst engine
 // ---------------------------------------------------------------------------
 template <int TO_POOL>
-__global__ void __launch_bounds__(LDST_THREADS)
+__global__ void __launch_bounds__(LDST_THREADS, 4)
 copy_ldst_kernel(CopyParams p) {
     __shared__ uint32_t s_claim;
     __shared__ int s_mode;
@@ -164,30 +164,53 @@ copy_ldst_kernel(CopyParams p) {
                     const unsigned long long p0 = (unsigned long long)t * CHUNK_BYTES + warp * 4096u;
                     if (p0 >= total_bytes) continue;
                     const uint32_t e0 = pow2 ? (uint32_t)(p0 >> shift) : (uint32_t)(p0 / elen);
-                    // lanes 0..7 fetch the entries this sub-range can touch, once
+                    const uint32_t off0 = (uint32_t)(p0 - (unsigned long long)e0 * elen);
+                    if (off0 + 4096u <= elen) {
+                        // the whole sub-range lies in one entry (blocks of 4 KiB and more):
+                        // lane 0 reads the entry once, every lane gets it by shuffle
+                        unsigned long long a_pool = 0, a_obj = 0;
+                        if (lane == 0) { a_pool = sgl[e0].addr; a_obj = obj[e0]; }
+                        a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
+                        a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
+                        const char *src = reinterpret_cast<const char *>(TO_POOL ? a_obj : a_pool) +
+                                          off0 + lane * 16u;
+                        char *dst = reinterpret_cast<char *>(TO_POOL ? a_pool : a_obj) + off0 + lane * 16u;
+                        uint4 v[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) v[k] = ld_stream(src + k * 512);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) st_stream(dst + k * 512, v[k]);
+                        continue;
+                    }
+                    // small entries (512 B .. 2 KiB, e.g. 1-token pages): lanes 0..7 fetch the
+                    // entries this sub-range touches, once; rows pick theirs by shuffle
                     unsigned long long my_pool = 0, my_obj = 0;
                     if (lane < 8 && e0 + lane < total) {
                         my_pool = sgl[e0 + lane].addr;
                         my_obj = obj[e0 + lane];
                     }
-                    uint4 v[8];
-                    unsigned long long dst[8];
-                    bool ok[8];
+#pragma unroll 1
+                    for (int half = 0; half < 2; ++half) {
+                        uint4 v[4];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const unsigned long long pk = p0 + (unsigned long long)k * 512u;
-                        ok[k] = pk < total_bytes;
-                        const uint32_t e = ok[k] ? (pow2 ? (uint32_t)(pk >> shift) : (uint32_t)(pk / elen)) : e0;
-                        const uint32_t off = (uint32_t)(pk - (unsigned long long)e * elen) + lane * 16u;
-                        const unsigned long long a_pool = __shfl_sync(0xffffffffu, my_pool, e - e0);
-                        const unsigned long long a_obj = __shfl_sync(0xffffffffu, my_obj, e - e0);
-                        const unsigned long long src = (TO_POOL ? a_obj : a_pool) + off;
-                        dst[k] = (TO_POOL ? a_pool : a_obj) + off;
-                        if (ok[k]) v[k] = ld_stream(reinterpret_cast<const void *>(src));
+                        for (int k = 0; k < 4; ++k) {
+                            const unsigned long long pk = p0 + (unsigned long long)(half * 4 + k) * 512u;
+                            const bool ok = pk < total_bytes;
+                            const uint32_t e = ok ? (pow2 ? (uint32_t)(pk >> shift) : (uint32_t)(pk / elen)) : e0;
+                            const uint32_t off = (uint32_t)(pk - (unsigned long long)e * elen) + lane * 16u;
+                            const unsigned long long a = __shfl_sync(0xffffffffu, TO_POOL ? my_obj : my_pool, e - e0);
+                            if (ok) v[k] = ld_stream(reinterpret_cast<const void *>(a + off));
+                        }
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const unsigned long long pk = p0 + (unsigned long long)(half * 4 + k) * 512u;
+                            const bool ok = pk < total_bytes;
+                            const uint32_t e = ok ? (pow2 ? (uint32_t)(pk >> shift) : (uint32_t)(pk / elen)) : e0;
+                            const uint32_t off = (uint32_t)(pk - (unsigned long long)e * elen) + lane * 16u;
+                            const unsigned long long a = __shfl_sync(0xffffffffu, TO_POOL ? my_pool : my_obj, e - e0);
+                            if (ok) st_stream(reinterpret_cast<void *>(a + off), v[k]);
+                        }
                     }
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        if (ok[k]) st_stream(reinterpret_cast<void *>(dst[k]), v[k]);
                 }
                 __syncthreads();
                 if (threadIdx.x == 0) {
@@ -307,9 +330,11 @@ __device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen, u
     return g;
 }
 
-// Each warp of the CTA is an independent agent with its own stage ring.
-// Shared memory: [warps][stages][CHUNK_BYTES] data, then [warps][stages] mbarriers,
-// then per stage the store descriptors of the 32 lanes and the chunk's byte count.
+// Each warp of the CTA is an independent agent with its own ring of stages, fed by a
+// stream of chunks that runs across the IOCBs of the launch without draining in between.
+// Shared memory: [warps][stages][chunk bytes] data, [warps][stages] mbarriers, then per
+// stage the store descriptor of every lane (address, bytes, offset in the stage) and
+// the chunk's byte count and IOCB.
 template <int TO_POOL>
 __global__ void __launch_bounds__(256, 1)
 copy_bulk_kernel(CopyParams p) {
@@ -321,13 +346,14 @@ copy_bulk_kernel(CopyParams p) {
     unsigned char *data = smem + (size_t)warp * S * CB;
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(
         smem + (size_t)n_warps * S * CB) + warp * S;
-    // per stage: destination address and byte count of every lane's store, chunk bytes
     unsigned char *meta = smem + (size_t)n_warps * S * (CB + 8);
+    const size_t lanes_all = (size_t)n_warps * S * 32;
     unsigned long long *st_addr_of = reinterpret_cast<unsigned long long *>(meta) + (size_t)warp * S * 32;
-    uint32_t *st_bytes_of = reinterpret_cast<uint32_t *>(meta + (size_t)n_warps * S * 32 * 8) +
-                            (size_t)warp * S * 32;
-    uint32_t *chunk_bytes_of = reinterpret_cast<uint32_t *>(meta + (size_t)n_warps * S * 32 * 12) +
-                               warp * S;
+    uint32_t *st_bytes_of = reinterpret_cast<uint32_t *>(meta + lanes_all * 8) + (size_t)warp * S * 32;
+    uint32_t *st_off_of = reinterpret_cast<uint32_t *>(meta + lanes_all * 12) + (size_t)warp * S * 32;
+    uint32_t *chunk_bytes_of = reinterpret_cast<uint32_t *>(meta + lanes_all * 16) + warp * S;
+    uint32_t *chunk_iocb_of = reinterpret_cast<uint32_t *>(meta + lanes_all * 16 +
+                                                           (size_t)n_warps * S * 4) + warp * S;
 
     if (lane == 0)
         for (uint32_t s = 0; s < S; ++s) mbar_init(smem_u32(&bars[s]), 1);
@@ -336,164 +362,208 @@ copy_bulk_kernel(CopyParams p) {
     __syncwarp();
 
     uint32_t phase_bits = 0;   // parity of every stage's mbarrier (bit s)
+    uint32_t head = 0, tail = 0;            // stages issued / drained (monotonic)
+    bool failed = false;
 
-    for (uint32_t bi = 0; bi < p.n_iocb; ++bi) {
-        const uint32_t idx = p.first_iocb + bi;
-        IocbHdr *h = &p.ring.hdrs[idx & (p.ring.depth - 1)];
-        int mode = 0;
-        if (lane == 0) mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
-        mode = __shfl_sync(0xffffffffu, mode, 0);
-        if (mode == IOCB_SKIP) continue;
-        const uint32_t total = h->total_entries;
-        if (total == 0 || h->status != 0) {
-            if (lane == 0) complete_empty(p.ring, h, idx);
-            continue;
-        }
-        const size_t e_base = (size_t)h->sgl_base + h->entry_first;
-        const tutti_sgl_t *sgl = p.ring.sgl + e_base;
-        const uint64_t *obj = p.ring.obj_ptr + e_base;
-        if (h->entry_len == 0) {
-            // entries of differing lengths (host-prepared IOCBs only): plain vector copies,
-            // one entry per warp at a time
-            for (;;) {
-                uint32_t c0 = 0;
-                if (lane == 0) c0 = atomicAdd(&h->claim_cursor, 8u);
-                c0 = __shfl_sync(0xffffffffu, c0, 0);
-                if (c0 >= total) break;
-                const uint32_t c1 = min(c0 + 8u, total);
-                unsigned long long moved = 0;
-                for (uint32_t e = c0; e < c1; ++e) {
-                    unsigned long long a_pool = 0, a_obj = 0;
-                    uint32_t len = 0;
-                    if (lane == 0) { a_pool = sgl[e].addr; len = sgl[e].len; a_obj = obj[e]; }
-                    a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
-                    a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
-                    len = __shfl_sync(0xffffffffu, len, 0);
-                    const unsigned long long src = TO_POOL ? a_obj : a_pool;
-                    const unsigned long long dst = TO_POOL ? a_pool : a_obj;
-                    for (uint32_t o = lane * 16u; o < len; o += 512u)
-                        st_stream(reinterpret_cast<void *>(dst + o),
-                                  ld_stream(reinterpret_cast<const void *>(src + o)));
-                    moved += len;
-                }
-                __syncwarp();
-                if (lane == 0) account_done(p.ring, h, idx, moved);
-            }
-            continue;
-        }
-        const ChunkGeom cg = chunk_geom(total, h->entry_len, CB);
+    // ---- source side of the stream: the IOCB chunks are being claimed from
+    uint32_t f_bi = 0;                      // next IOCB of the launch to open
+    IocbHdr *f_h = nullptr;
+    ChunkGeom cg{0, 0, 0, 0, 0};
+    const tutti_sgl_t *sgl = nullptr;
+    const uint64_t *obj = nullptr;
+    bool f_open = false;
+    uint32_t f_cur_bi = 0;
+    uint32_t pending_claim = 0, cur = 0, cur_end = 0;
+    // the next chunk, fetched ahead: one bulk load and one bulk store per lane
+    bool have_next = false;
+    uint32_t n_bi = 0, ld_bytes = 0, st_bytes = 0, st_off = 0;
+    unsigned long long ld_addr = 0, st_addr = 0;
 
-        uint32_t head = 0, tail = 0;            // stages issued / drained (monotonic)
-        unsigned long long moved = 0;           // bytes this agent has stored
-        bool failed = false;
+    // ---- sink side: bytes stored for the IOCB being accounted
+    uint32_t acct_bi = 0;
+    unsigned long long moved = 0;
 
-        // Work claims are taken one ahead of need (the atomic's latency hides behind the
-        // copies of the current claim), and the addresses of the next chunk are fetched as
-        // soon as the current chunk's loads are issued.
-        uint32_t pending_claim = 0;
-        if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
-        uint32_t cur = 0, cur_end = 0;
-        bool have_next = false;
-        uint32_t c_next = 0, n_e = 0, ld_bytes = 0, st_bytes = 0;
-        unsigned long long ld_addr = 0, st_addr = 0;
-
-        auto fetch_next = [&]() {
-            have_next = false;
-            if (failed) return;
-            if (cur == cur_end) {
-                uint32_t c0 = __shfl_sync(0xffffffffu, pending_claim, 0);
-                if (c0 >= cg.n_chunks) return;
-                cur = c0;
-                cur_end = min(c0 + p.claim_chunks, cg.n_chunks);
-                if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
-            }
-            c_next = cur++;
-            have_next = true;
-            ld_bytes = 0; st_bytes = 0; ld_addr = 0; st_addr = 0;
-            if (cg.per_chunk) {
-                const uint32_t e0 = c_next * cg.per_chunk;
-                n_e = min(cg.per_chunk, cg.total - e0);
-                unsigned long long a_obj = 0, a_pool = 0;
-                if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
-                // the object side is contiguous in runs: one bulk copy per run
-                unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
-                bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
-                uint32_t heads = __ballot_sync(0xffffffffu, is_head);
-                uint32_t run_bytes = 0;
-                if (is_head) {
-                    uint32_t above = lane < 31 ? heads >> (lane + 1) : 0u;
-                    uint32_t next = above ? lane + __ffs(above) : n_e;
-                    run_bytes = (next - lane) * cg.elen;
-                }
-                const uint32_t one = lane < n_e ? cg.elen : 0;
-                if (TO_POOL) { ld_addr = a_obj; ld_bytes = run_bytes; st_addr = a_pool; st_bytes = one; }
-                else         { ld_addr = a_pool; ld_bytes = one; st_addr = a_obj; st_bytes = run_bytes; }
-            } else {
-                const uint32_t e = c_next / cg.pieces, piece = c_next % cg.pieces;
-                const uint32_t off = piece * CB;
-                const uint32_t bytes = min(CB, cg.elen - off);
-                n_e = 1;
-                if (lane == 0) {
-                    unsigned long long a_obj = obj[e] + off, a_pool = sgl[e].addr + off;
-                    ld_addr = TO_POOL ? a_obj : a_pool;
-                    st_addr = TO_POOL ? a_pool : a_obj;
-                    ld_bytes = bytes; st_bytes = bytes;
-                }
-            }
-        };
-        fetch_next();
-
-        for (;;) {
-            // ---- issue loads while a stage is free (one stage of slack is kept for the
-            //      store that may still be reading shared memory)
-            while (have_next && head - tail < S - 1) {
-                const uint32_t s = head % S;
-                // the store that last used this stage must have finished reading it:
-                // at most one newer store group may still be pending
-                bulk_wait_read_1();
-                __syncwarp();
-                const uint32_t bar = smem_u32(&bars[s]);
-                const uint32_t sbase = smem_u32(data + (size_t)s * CB);
-                const uint32_t total_bytes = __reduce_add_sync(0xffffffffu, ld_bytes);
-                const uint32_t my_off = cg.per_chunk ? lane * cg.elen : 0;
-                if (lane == 0) mbar_expect_tx(bar, total_bytes);
-                __syncwarp();
-                if (ld_bytes) bulk_g2s(sbase + my_off, ld_addr, ld_bytes, bar);
-                st_addr_of[s * 32 + lane] = st_addr;
-                st_bytes_of[s * 32 + lane] = st_bytes;
-                if (lane == 0) chunk_bytes_of[s] = total_bytes;
-                __syncwarp();
-                ++head;
-                fetch_next();
-            }
-            if (head == tail) break;
-
-            // ---- drain the oldest stage: wait for its bytes, store them
-            const uint32_t s = tail % S;
-            const uint32_t bar = smem_u32(&bars[s]);
-            const uint32_t sbase = smem_u32(data + (size_t)s * CB);
-            bool arrived = mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
-            arrived = __all_sync(0xffffffffu, arrived);
-            phase_bits ^= (1u << s);
-            if (!arrived) failed = true;
-            const unsigned long long dst = st_addr_of[s * 32 + lane];
-            const uint32_t nbytes = st_bytes_of[s * 32 + lane];
-            const uint32_t my_off = cg.per_chunk ? lane * cg.elen : 0;
-            if (arrived && nbytes) bulk_s2g(dst, sbase + my_off, nbytes);
-            bulk_commit();
-            moved += chunk_bytes_of[s];
-            ++tail;
-            if (failed) have_next = false;    // stop taking new work; the rest is drained
-        }
-        // all of this agent's stores must have landed before they are accounted
+    auto hdr_of = [&](uint32_t bi) -> IocbHdr * {
+        return &p.ring.hdrs[(p.first_iocb + bi) & (p.ring.depth - 1)];
+    };
+    // all stores of this agent so far have landed: account what belongs to acct_bi
+    auto flush_account = [&]() {
+        if (moved == 0) return;
         bulk_wait_all();
         __syncwarp();
-        if (lane == 0) {
-            if (failed) atomicCAS(&h->status, 0, TUTTI_ETIMEDOUT);
-            account_done(p.ring, h, idx, moved);
-        }
+        if (lane == 0) account_done(p.ring, hdr_of(acct_bi), p.first_iocb + acct_bi, moved);
         __syncwarp();
+        moved = 0;
+    };
+
+    // Entries of differing lengths (host-prepared IOCBs only): plain vector copies, one
+    // entry per warp at a time, outside the staged pipeline.
+    auto copy_varlen = [&](IocbHdr *h, uint32_t idx, uint32_t total) {
+        for (;;) {
+            uint32_t c0 = 0;
+            if (lane == 0) c0 = atomicAdd(&h->claim_cursor, 8u);
+            c0 = __shfl_sync(0xffffffffu, c0, 0);
+            if (c0 >= total) break;
+            const uint32_t c1 = min(c0 + 8u, total);
+            unsigned long long mv = 0;
+            for (uint32_t e = c0; e < c1; ++e) {
+                unsigned long long a_pool = 0, a_obj = 0;
+                uint32_t len = 0;
+                if (lane == 0) { a_pool = sgl[e].addr; len = sgl[e].len; a_obj = obj[e]; }
+                a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
+                a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
+                len = __shfl_sync(0xffffffffu, len, 0);
+                const unsigned long long src = TO_POOL ? a_obj : a_pool;
+                const unsigned long long dst = TO_POOL ? a_pool : a_obj;
+                for (uint32_t o = lane * 16u; o < len; o += 512u)
+                    st_stream(reinterpret_cast<void *>(dst + o),
+                              ld_stream(reinterpret_cast<const void *>(src + o)));
+                mv += len;
+            }
+            __syncwarp();
+            if (lane == 0) account_done(p.ring, h, idx, mv);
+        }
+    };
+
+    // Open the next IOCB that has staged work; false when the launch has none left.
+    auto open_next_iocb = [&]() -> bool {
+        while (f_bi < p.n_iocb) {
+            const uint32_t bi = f_bi++;
+            const uint32_t idx = p.first_iocb + bi;
+            IocbHdr *h = hdr_of(bi);
+            int mode = 0;
+            if (lane == 0) mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
+            mode = __shfl_sync(0xffffffffu, mode, 0);
+            if (mode == IOCB_SKIP) continue;
+            const uint32_t total = h->total_entries;
+            if (total == 0 || h->status != 0) {
+                if (lane == 0) complete_empty(p.ring, h, idx);
+                continue;
+            }
+            const size_t e_base = (size_t)h->sgl_base + h->entry_first;
+            sgl = p.ring.sgl + e_base;
+            obj = p.ring.obj_ptr + e_base;
+            if (h->entry_len == 0) { copy_varlen(h, idx, total); continue; }
+            f_h = h;
+            f_cur_bi = bi;
+            cg = chunk_geom(total, h->entry_len, CB);
+            cur = cur_end = 0;
+            if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
+            return true;
+        }
+        return false;
+    };
+
+    // Work claims are taken one ahead of need (the atomic's latency hides behind the
+    // copies of the current claim), and the addresses of the next chunk are fetched as
+    // soon as the current chunk's loads are issued.
+    auto fetch_next = [&]() {
+        have_next = false;
+        if (failed) return;
+        for (;;) {
+            if (!f_open) {
+                if (!open_next_iocb()) return;
+                f_open = true;
+            }
+            if (cur == cur_end) {
+                uint32_t c0 = __shfl_sync(0xffffffffu, pending_claim, 0);
+                if (c0 >= cg.n_chunks) { f_open = false; continue; }
+                cur = c0;
+                cur_end = min(c0 + p.claim_chunks, cg.n_chunks);
+                if (lane == 0) pending_claim = atomicAdd(&f_h->claim_cursor, p.claim_chunks);
+            }
+            break;
+        }
+        const uint32_t c = cur++;
+        have_next = true;
+        n_bi = f_cur_bi;
+        ld_bytes = 0; st_bytes = 0; st_off = 0; ld_addr = 0; st_addr = 0;
+        if (cg.per_chunk) {
+            const uint32_t e0 = c * cg.per_chunk;
+            const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
+            unsigned long long a_obj = 0, a_pool = 0;
+            if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
+            // the object side is contiguous in runs: one bulk copy per run
+            unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
+            bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
+            uint32_t heads = __ballot_sync(0xffffffffu, is_head);
+            uint32_t run_bytes = 0;
+            if (is_head) {
+                uint32_t above = lane < 31 ? heads >> (lane + 1) : 0u;
+                uint32_t next = above ? lane + __ffs(above) : n_e;
+                run_bytes = (next - lane) * cg.elen;
+            }
+            const uint32_t one = lane < n_e ? cg.elen : 0;
+            st_off = lane * cg.elen;
+            if (TO_POOL) { ld_addr = a_obj; ld_bytes = run_bytes; st_addr = a_pool; st_bytes = one; }
+            else         { ld_addr = a_pool; ld_bytes = one; st_addr = a_obj; st_bytes = run_bytes; }
+        } else {
+            const uint32_t e = c / cg.pieces, piece = c % cg.pieces;
+            const uint32_t off = piece * CB;
+            const uint32_t bytes = min(CB, cg.elen - off);
+            if (lane == 0) {
+                unsigned long long a_obj = obj[e] + off, a_pool = sgl[e].addr + off;
+                ld_addr = TO_POOL ? a_obj : a_pool;
+                st_addr = TO_POOL ? a_pool : a_obj;
+                ld_bytes = bytes; st_bytes = bytes;
+            }
+        }
+    };
+    fetch_next();
+
+    for (;;) {
+        // ---- issue loads while a stage is free (one stage of slack is kept for the
+        //      store that may still be reading shared memory)
+        while (have_next && head - tail < S - 1) {
+            const uint32_t s = head % S;
+            // the store that last used this stage must have finished reading it:
+            // at most one newer store group may still be pending
+            bulk_wait_read_1();
+            __syncwarp();
+            const uint32_t bar = smem_u32(&bars[s]);
+            const uint32_t sbase = smem_u32(data + (size_t)s * CB);
+            const uint32_t total_bytes = __reduce_add_sync(0xffffffffu, ld_bytes);
+            if (lane == 0) mbar_expect_tx(bar, total_bytes);
+            __syncwarp();
+            if (ld_bytes) bulk_g2s(sbase + st_off, ld_addr, ld_bytes, bar);
+            st_addr_of[s * 32 + lane] = st_addr;
+            st_bytes_of[s * 32 + lane] = st_bytes;
+            st_off_of[s * 32 + lane] = st_off;
+            if (lane == 0) { chunk_bytes_of[s] = total_bytes; chunk_iocb_of[s] = n_bi; }
+            __syncwarp();
+            ++head;
+            fetch_next();
+        }
+        if (head == tail) break;
+
+        // ---- drain the oldest stage: wait for its bytes, store them
+        const uint32_t s = tail % S;
+        const uint32_t bar = smem_u32(&bars[s]);
+        const uint32_t sbase = smem_u32(data + (size_t)s * CB);
+        const uint32_t s_bi = chunk_iocb_of[s];
+        if (s_bi != acct_bi) {
+            // first chunk of a later IOCB: close the books of the previous one.  Only the
+            // stores are waited for; the loads already in flight keep streaming.
+            flush_account();
+            acct_bi = s_bi;
+        }
+        bool arrived = mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
+        arrived = __all_sync(0xffffffffu, arrived);
+        phase_bits ^= (1u << s);
+        if (!arrived) {
+            failed = true;
+            if (lane == 0) atomicCAS(&hdr_of(s_bi)->status, 0, TUTTI_ETIMEDOUT);
+        }
+        const unsigned long long dst = st_addr_of[s * 32 + lane];
+        const uint32_t nbytes = st_bytes_of[s * 32 + lane];
+        const uint32_t off = st_off_of[s * 32 + lane];
+        if (arrived && nbytes) bulk_s2g(dst, sbase + off, nbytes);
+        bulk_commit();
+        moved += chunk_bytes_of[s];
+        ++tail;
+        if (failed) have_next = false;    // stop taking new work; the rest is drained
     }
+    flush_account();
 }
 
 }  // namespace
@@ -529,7 +599,7 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
         if (stages < 2) stages = 2;
         if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
         uint32_t cb = opt.bulk_chunk ? opt.bulk_chunk : (sm_count ? 16384u : CHUNK_BYTES);
-        const size_t per_stage = cb + 8 + 32 * 12 + 4;
+        const size_t per_stage = cb + 8 + 32 * 16 + 8;
         while ((size_t)warps * stages * per_stage > 224u * 1024u) {
             if (stages > 2) --stages; else --warps;
         }

@@ -340,6 +340,53 @@ int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int device, uint32_
                                    void *const *store_base, const uint64_t *store_bytes,
                                    tutti_cqe_t *cqe_out, void *stream);
 
+/* ------------------------------------------------------------------------- */
+/* Slack-aware I/O scheduler (Section 3.3).  Pure host logic.                  */
+/* ------------------------------------------------------------------------- */
+#define TUTTI_PHASE_PREFILL 0
+#define TUTTI_PHASE_DECODE 1
+
+typedef struct tutti_sched tutti_sched_t;
+
+/* One kernel launch the scheduler asks for: IOCBs [first_iocb, first_iocb + n_iocb)
+ * with tutti_kv_restore_layer / tutti_kv_save_layer on sm_count SMs (0 = all).
+ * est_us is the profiled time of the whole read (or write) group the launch opens. */
+typedef struct tutti_launch {
+    uint32_t opcode;
+    uint32_t first_iocb;
+    uint32_t n_iocb;
+    uint32_t sm_count;
+    uint32_t layer; /* layer of the first IOCB */
+    float est_us;
+} tutti_launch_t;
+
+/* The lookup table is indexed by input length and prefix length in steps of
+ * token_step tokens ("the token length of a single warp", Section 3.3). */
+int tutti_sched_create(uint32_t n_layers, uint32_t token_step, uint32_t max_input_tokens,
+                       uint32_t max_prefix_tokens, tutti_sched_t **out);
+int tutti_sched_destroy(tutti_sched_t *sched);
+/* Offline profile of the model: duration and free-SM budget of a layer's slack window. */
+int tutti_sched_set_slack(tutti_sched_t *sched, uint32_t l_input, uint32_t l_prefix,
+                          float slack_us, uint32_t sm_budget);
+int tutti_sched_set_decode_slack(tutti_sched_t *sched, float slack_us, uint32_t sm_budget);
+/* Offline profile of the I/O kernels: time of one launch of n_iocb IOCBs on sm_count SMs.
+ * Other counts are interpolated linearly (extrapolated beyond the last point); an
+ * unprofiled SM count uses the largest profiled one that is not larger. */
+int tutti_sched_set_io_time(tutti_sched_t *sched, uint32_t opcode, uint32_t sm_count,
+                            uint32_t n_iocb, float us);
+int tutti_sched_io_time(const tutti_sched_t *sched, uint32_t opcode, uint32_t sm_count,
+                        uint32_t n_iocb, float *us);
+/* Queue built IOCBs: reads when a request arrives, writes when a layer's KV is produced. */
+int tutti_sched_enqueue(tutti_sched_t *sched, uint32_t opcode, uint32_t layer, uint32_t first_iocb,
+                        uint32_t n_iocb);
+/* Decide what to launch before `layer` begins (prefill) or in a decode step: reads first —
+ * as many as fit the window, at least those of layers <= layer — then writes if window
+ * is left; the rest stays queued.  Launches are written to out[0..*n_out).  TUTTI_EAGAIN
+ * (nothing lost: *n_out is the count needed) if max_out is too small. */
+int tutti_sched_next(tutti_sched_t *sched, uint32_t phase, uint32_t layer, uint32_t l_input,
+                     uint32_t l_prefix, tutti_launch_t *out, uint32_t max_out, uint32_t *n_out);
+int tutti_sched_pending(const tutti_sched_t *sched, uint32_t *reads, uint32_t *writes);
+
 /* Host-side ring accounting on its own (no GPU involved; used by CPU tests):
  * the reservation / release bookkeeping that tutti_build_sqes and tutti_ring_poll
  * apply to IOCB indices and SGL arena ranges. */

@@ -46,6 +46,11 @@ class Cqe(C.Structure):
     _fields_ = [("iocb_idx", C.c_uint32), ("status", C.c_int32), ("bytes", C.c_uint64)]
 
 
+class Launch(C.Structure):
+    _fields_ = [("opcode", C.c_uint32), ("first_iocb", C.c_uint32), ("n_iocb", C.c_uint32),
+                ("sm_count", C.c_uint32), ("layer", C.c_uint32), ("est_us", C.c_float)]
+
+
 class IocbInfo(C.Structure):
     _fields_ = [("iocb_idx", C.c_uint32), ("ready", C.c_uint32), ("num_ioctx", C.c_uint32),
                 ("opcode", C.c_uint32), ("layer", C.c_uint32), ("status", C.c_int32),
@@ -66,6 +71,9 @@ EXPORTS = [
     "tutti_hostring_create", "tutti_hostring_destroy", "tutti_hostring_reserve",
     "tutti_hostring_release", "tutti_hostring_live", "tutti_strerror", "tutti_last_cuda_error",
     "tutti_version", "tutti_kv_restore_layer_noalloc",
+    "tutti_sched_create", "tutti_sched_destroy", "tutti_sched_set_slack",
+    "tutti_sched_set_decode_slack", "tutti_sched_set_io_time", "tutti_sched_io_time",
+    "tutti_sched_enqueue", "tutti_sched_next", "tutti_sched_pending",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -111,6 +119,15 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_strerror": (C.c_char_p, [C.c_int]),
         "tutti_last_cuda_error": (C.c_char_p, []),
         "tutti_version": (u32, []),
+        "tutti_sched_create": (C.c_int, [u32, u32, u32, u32, P(vp)]),
+        "tutti_sched_destroy": (C.c_int, [vp]),
+        "tutti_sched_set_slack": (C.c_int, [vp, u32, u32, C.c_float, u32]),
+        "tutti_sched_set_decode_slack": (C.c_int, [vp, C.c_float, u32]),
+        "tutti_sched_set_io_time": (C.c_int, [vp, u32, u32, u32, C.c_float]),
+        "tutti_sched_io_time": (C.c_int, [vp, u32, u32, u32, P(C.c_float)]),
+        "tutti_sched_enqueue": (C.c_int, [vp, u32, u32, u32, u32]),
+        "tutti_sched_next": (C.c_int, [vp, u32, u32, u32, u32, P(Launch), u32, P(u32)]),
+        "tutti_sched_pending": (C.c_int, [vp, P(u32), P(u32)]),
         "tutti_kv_restore_layer_noalloc": (C.c_int, [P(Geom), C.c_int, u32, P(Batch), vp, vp, u64,
                                                      u64, P(vp), P(u64), vp, vp]),
     }
@@ -306,3 +323,62 @@ def tutti_kv_restore_layer_noalloc(geom: Geom, device: int, layer: int, batch: B
                                                         block_stride, n_blocks, bases, sizes,
                                                         cqe_out, _stream_ptr(stream)),
                   "tutti_kv_restore_layer_noalloc", allow)
+
+
+PHASE_PREFILL, PHASE_DECODE = 0, 1
+
+
+class Scheduler:
+    """tutti_sched_t: the slack-aware I/O scheduler (host logic only)."""
+
+    def __init__(self, n_layers: int, token_step: int, max_input_tokens: int,
+                 max_prefix_tokens: int):
+        self.lib = load()
+        h = C.c_void_p()
+        _check(self.lib.tutti_sched_create(n_layers, token_step, max_input_tokens,
+                                           max_prefix_tokens, C.byref(h)), "tutti_sched_create")
+        self.h = h
+
+    def close(self):
+        if self.h:
+            self.lib.tutti_sched_destroy(self.h)
+            self.h = None
+
+    def tutti_sched_set_slack(self, l_input, l_prefix, slack_us, sm_budget):
+        _check(self.lib.tutti_sched_set_slack(self.h, l_input, l_prefix, slack_us, sm_budget),
+               "tutti_sched_set_slack")
+
+    def tutti_sched_set_decode_slack(self, slack_us, sm_budget):
+        _check(self.lib.tutti_sched_set_decode_slack(self.h, slack_us, sm_budget),
+               "tutti_sched_set_decode_slack")
+
+    def tutti_sched_set_io_time(self, opcode, sm_count, n_iocb, us):
+        _check(self.lib.tutti_sched_set_io_time(self.h, opcode, sm_count, n_iocb, us),
+               "tutti_sched_set_io_time")
+
+    def tutti_sched_io_time(self, opcode, sm_count, n_iocb) -> float:
+        us = C.c_float()
+        _check(self.lib.tutti_sched_io_time(self.h, opcode, sm_count, n_iocb, C.byref(us)),
+               "tutti_sched_io_time")
+        return us.value
+
+    def tutti_sched_enqueue(self, opcode, layer, first_iocb, n_iocb, allow: Sequence[int] = ()):
+        return _check(self.lib.tutti_sched_enqueue(self.h, opcode, layer, first_iocb, n_iocb),
+                      "tutti_sched_enqueue", allow)
+
+    def tutti_sched_next(self, phase, layer, l_input, l_prefix, max_out: int = 64):
+        """[(opcode, first_iocb, n_iocb, sm_count, layer, est_us)] to launch now."""
+        out = (Launch * max_out)()
+        n = C.c_uint32()
+        rc = self.lib.tutti_sched_next(self.h, phase, layer, l_input, l_prefix, out, max_out,
+                                       C.byref(n))
+        if rc == EAGAIN:
+            return self.tutti_sched_next(phase, layer, l_input, l_prefix, n.value)
+        _check(rc, "tutti_sched_next")
+        return [(o.opcode, o.first_iocb, o.n_iocb, o.sm_count, o.layer, o.est_us)
+                for o in out[:n.value]]
+
+    def tutti_sched_pending(self) -> Tuple[int, int]:
+        a, b = C.c_uint32(), C.c_uint32()
+        _check(self.lib.tutti_sched_pending(self.h, C.byref(a), C.byref(b)), "tutti_sched_pending")
+        return a.value, b.value

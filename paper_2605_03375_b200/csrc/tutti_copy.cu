@@ -94,6 +94,39 @@ __device__ void complete_empty(const RingDev &ring, IocbHdr *h, uint32_t idx) {
         post_cqe(ring, idx, h->status, 0);
 }
 
+// Warp-collective look-ahead over the IOCBs [bi, n_iocb) of a launch: 32 headers are read at
+// a time, and the leading ones that need no copying — already complete, or published with
+// nothing to move (the unused tail of a build's reservation, or a build error) — are
+// skipped without a round trip each.  The `designated` warp (one per launch) completes
+// the published-but-empty ones, one lane per IOCB.  Returns the first IOCB that is either
+// not published yet or has bytes to move (n_iocb if none).
+__device__ uint32_t skip_idle_iocbs(const RingDev &ring, uint32_t first_iocb, uint32_t bi,
+                                    uint32_t n_iocb, bool designated) {
+    const uint32_t lane = threadIdx.x & 31;
+    while (bi < n_iocb) {
+        const uint32_t k = bi + lane;
+        bool idle = false, empty_ready = false;
+        IocbHdr *h = nullptr;
+        uint32_t idx = first_iocb + k;
+        if (k < n_iocb) {
+            h = &ring.hdrs[idx & (ring.depth - 1)];
+            const uint32_t st = ld_acquire_u32(&h->state);
+            if (st == state_word(idx, PHASE_DONE)) {
+                idle = true;
+            } else if (st == state_word(idx, PHASE_READY)) {
+                empty_ready = (h->total_entries == 0 || h->status != 0);
+                idle = empty_ready;
+            }
+        }
+        const uint32_t mask = __ballot_sync(0xffffffffu, idle);
+        const uint32_t lead = (mask == 0xffffffffu) ? 32u : (uint32_t)(__ffs(~mask) - 1);
+        if (designated && empty_ready && lane < lead) complete_empty(ring, h, idx);
+        bi += lead;
+        if (lead < 32u) break;
+    }
+    return bi < n_iocb ? bi : n_iocb;
+}
+
 // Account `bytes` landed; the agent that completes the IOCB posts the CQE.
 __device__ void account_done(const RingDev &ring, IocbHdr *h, uint32_t idx,
                              unsigned long long bytes) {
@@ -129,7 +162,16 @@ copy_ldst_kernel(CopyParams p) {
     __shared__ int s_mode;
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
+    __shared__ uint32_t s_bi;
     for (uint32_t bi = 0; bi < p.n_iocb; ++bi) {
+        // warp 0 looks ahead past IOCBs that need no copying
+        if (warp == 0) {
+            uint32_t nb = skip_idle_iocbs(p.ring, p.first_iocb, bi, p.n_iocb, blockIdx.x == 0);
+            if (lane == 0) s_bi = nb;
+        }
+        __syncthreads();
+        bi = s_bi;
+        if (bi >= p.n_iocb) break;
         const uint32_t idx = p.first_iocb + bi;
         IocbHdr *h = &p.ring.hdrs[idx & (p.ring.depth - 1)];
         if (threadIdx.x == 0) s_mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
@@ -428,6 +470,9 @@ copy_bulk_kernel(CopyParams p) {
     // Open the next IOCB that has staged work; false when the launch has none left.
     auto open_next_iocb = [&]() -> bool {
         while (f_bi < p.n_iocb) {
+            f_bi = skip_idle_iocbs(p.ring, p.first_iocb, f_bi, p.n_iocb,
+                                   blockIdx.x == 0 && warp == 0);
+            if (f_bi >= p.n_iocb) break;
             const uint32_t bi = f_bi++;
             const uint32_t idx = p.first_iocb + bi;
             IocbHdr *h = hdr_of(bi);

@@ -43,6 +43,11 @@ extern "C" {
 
 #define TUTTI_OP_READ 0  /* object store -> paged pool  (restore / Retrieve) */
 #define TUTTI_OP_WRITE 1 /* paged pool  -> object store (save / Store)       */
+/* Opcode flag carried by contexts and IOCBs built while the pool layout is head-major:
+ * a pool block is [head][token][dim] instead of [token][head][dim] (Section 2.1 gives
+ * the paged layout as [Block, h, d]; objects always stay token-major), so the copy
+ * transposes rows of head_dim elements inside every block. */
+#define TUTTI_OP_FLAG_HND 0x100
 
 #define TUTTI_STORE_HBM 0
 #define TUTTI_STORE_HOST_PINNED 1
@@ -57,6 +62,10 @@ extern "C" {
 #define TUTTI_OPT_BULK_WARPS 4  /* copy warps per CTA of the bulk-async kernel                   */
 #define TUTTI_OPT_BULK_STAGES 5 /* shared-memory stages per copy warp of the bulk-async kernel   */
 #define TUTTI_OPT_CLAIM_CHUNKS 6 /* chunks taken per work claim                                   */
+#define TUTTI_OPT_POOL_LAYOUT 8  /* TUTTI_POOL_NHD (default) or TUTTI_POOL_HND: element order inside a
+                                   pool block; applies to builds made after it is set        */
+#define TUTTI_POOL_NHD 0
+#define TUTTI_POOL_HND 1
 #define TUTTI_OPT_BULK_CHUNK_BYTES 7 /* bytes per shared-memory stage of the bulk-async kernel: a
                                         power of two, 4096..32768                                 */
 

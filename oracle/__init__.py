@@ -24,6 +24,7 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 OK, EINVAL, ENOSPC = 0, -1, -2
 FILE_MAJOR, LAYER_MAJOR = 0, 1
 OP_READ, OP_WRITE = 0, 1
+OP_HND = 0x100       # opcode flag: head-major pool blocks
 
 
 def build(force: bool = False) -> str:
@@ -106,30 +107,34 @@ def _store_ptrs(store: Sequence[np.ndarray]):
     return arr
 
 
-def _move(fn, g, layer, batch, store, pool, k_off, v_off, block_stride, n_pool_blocks):
+def _move(fn, g, layer, batch, store, pool, k_off, v_off, block_stride, n_pool_blocks, pool_hnd):
     keep, bargs = _batch(*batch)
     assert pool.dtype == np.uint8 and pool.flags["C_CONTIGUOUS"]
     sp = _store_ptrs(store)
     base = pool.ctypes.data
     rc = fn(C.byref(g), C.c_uint32(layer), *bargs, sp, C.c_void_p(base + k_off),
-            C.c_void_p(base + v_off), C.c_uint64(block_stride), C.c_uint64(n_pool_blocks))
+            C.c_void_p(base + v_off), C.c_uint64(block_stride), C.c_uint64(n_pool_blocks),
+            C.c_int(1 if pool_hnd else 0))
     del keep
     return rc
 
 
 def restore_layer(g: Geom, layer: int, batch, store: Sequence[np.ndarray], pool: np.ndarray,
-                  k_off: int, v_off: int, block_stride: int, n_pool_blocks: int) -> int:
+                  k_off: int, v_off: int, block_stride: int, n_pool_blocks: int,
+                  pool_hnd: bool = False) -> int:
     """store -> pool for every cached token; `batch` = (hit_tokens, obj_start,
-    obj_slot, blk_start, block_ids).  Modifies `pool` in place."""
+    obj_slot, blk_start, block_ids).  Modifies `pool` in place.  pool_hnd: pool blocks are
+    [head][token][dim] instead of [token][head][dim]."""
     return _move(lib().orc_restore_layer, g, layer, batch, store, pool, k_off, v_off,
-                 block_stride, n_pool_blocks)
+                 block_stride, n_pool_blocks, pool_hnd)
 
 
 def save_layer(g: Geom, layer: int, batch, store: Sequence[np.ndarray], pool: np.ndarray,
-               k_off: int, v_off: int, block_stride: int, n_pool_blocks: int) -> int:
+               k_off: int, v_off: int, block_stride: int, n_pool_blocks: int,
+               pool_hnd: bool = False) -> int:
     """pool -> store for every cached token.  Modifies `store` in place."""
     return _move(lib().orc_save_layer, g, layer, batch, store, pool, k_off, v_off,
-                 block_stride, n_pool_blocks)
+                 block_stride, n_pool_blocks, pool_hnd)
 
 
 def token_location(g: Geom, layer: int, batch, r: int, t: int, kv: int
@@ -175,7 +180,8 @@ def build_descriptors(g: Geom, layer: int, opcode: int, batch, k_base_addr: int,
 
 
 def exec_descriptors(sqes: np.ndarray, sgl: np.ndarray, store: Sequence[np.ndarray],
-                     pool: np.ndarray, pool_base_addr: int) -> int:
+                     pool: np.ndarray, pool_base_addr: int, n_kv_heads: int = 0,
+                     row_bytes: int = 0) -> int:
     """Perform the transfers the descriptors describe on host copies."""
     sqes = np.ascontiguousarray(sqes)
     sgl = np.ascontiguousarray(sgl)
@@ -186,4 +192,4 @@ def exec_descriptors(sqes: np.ndarray, sgl: np.ndarray, store: Sequence[np.ndarr
                           C.c_void_p(sgl.ctypes.data), C.c_uint32(sgl.shape[0]), sp,
                           _p(sb, C.c_uint64), C.c_uint32(len(store)),
                           C.c_void_p(pool.ctypes.data), C.c_uint64(pool_base_addr),
-                          C.c_uint64(pool.nbytes))
+                          C.c_uint64(pool.nbytes), C.c_uint32(n_kv_heads), C.c_uint32(row_bytes))

@@ -51,6 +51,7 @@
 
 #define ORC_OP_READ 0  /* object store -> paged pool (restore) */
 #define ORC_OP_WRITE 1 /* paged pool -> object store (save)    */
+#define ORC_OP_HND 0x100 /* flag: pool blocks are [head][token][dim] instead of [token][head][dim] */
 
 typedef struct {
     uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
@@ -174,7 +175,8 @@ static int move_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
                       const uint32_t *hit_tokens, const uint32_t *obj_start,
                       const uint32_t *obj_slot, const uint32_t *blk_start,
                       const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
-                      uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks, int to_pool)
+                      uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks, int to_pool,
+                      int pool_hnd)
 {
     orc_layout lo;
     int rc = orc_obj_layout(g, &lo);
@@ -191,12 +193,27 @@ static int move_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
                                     t, kv, &dev, &soff, &blk, &roff);
                 if (rc) return rc;
                 if (blk < 0 || (uint64_t)blk >= n_pool_blocks) return ORC_EINVAL;
-                uint8_t *in_pool = (kv ? pool_v : pool_k) + (uint64_t)blk * block_stride + roff;
                 uint8_t *in_store = store[dev] + soff;
-                if (to_pool)
-                    memcpy(in_pool, in_store, lo.token_bytes);
-                else
-                    memcpy(in_store, in_pool, lo.token_bytes);
+                if (!pool_hnd) {
+                    /* block = [token][head][dim]: the token's bytes are one run */
+                    uint8_t *in_pool = (kv ? pool_v : pool_k) + (uint64_t)blk * block_stride + roff;
+                    if (to_pool)
+                        memcpy(in_pool, in_store, lo.token_bytes);
+                    else
+                        memcpy(in_store, in_pool, lo.token_bytes);
+                } else {
+                    /* block = [head][token][dim]: one row of head_dim elements per head */
+                    uint64_t row = (uint64_t)g->head_dim * g->elem_bytes;
+                    uint64_t tok = t % g->block_tokens;
+                    for (uint32_t hd = 0; hd < g->n_kv_heads; ++hd) {
+                        uint8_t *in_pool = (kv ? pool_v : pool_k) + (uint64_t)blk * block_stride +
+                                           ((uint64_t)hd * g->block_tokens + tok) * row;
+                        if (to_pool)
+                            memcpy(in_pool, in_store + hd * row, row);
+                        else
+                            memcpy(in_store + hd * row, in_pool, row);
+                    }
+                }
             }
         }
     }
@@ -208,10 +225,10 @@ int orc_restore_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
                       const uint32_t *hit_tokens, const uint32_t *obj_start,
                       const uint32_t *obj_slot, const uint32_t *blk_start,
                       const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
-                      uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks)
+                      uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks, int pool_hnd)
 {
     return move_layer(g, layer, n_req, hit_tokens, obj_start, obj_slot, blk_start, block_ids,
-                      store, pool_k, pool_v, block_stride, n_pool_blocks, 1);
+                      store, pool_k, pool_v, block_stride, n_pool_blocks, 1, pool_hnd);
 }
 
 /* Layer-wise Store (Section 3.1 / 3.4): paged pool -> object store. */
@@ -219,10 +236,10 @@ int orc_save_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
                    const uint32_t *hit_tokens, const uint32_t *obj_start,
                    const uint32_t *obj_slot, const uint32_t *blk_start,
                    const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
-                   uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks)
+                   uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks, int pool_hnd)
 {
     return move_layer(g, layer, n_req, hit_tokens, obj_start, obj_slot, blk_start, block_ids,
-                      store, pool_k, pool_v, block_stride, n_pool_blocks, 0);
+                      store, pool_k, pool_v, block_stride, n_pool_blocks, 0, pool_hnd);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -267,7 +284,8 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
     if (rc) return rc;
     rc = check_batch(g, layer, n_req, hit_tokens, obj_start, blk_start);
     if (rc) return rc;
-    if (capacity == 0 || (opcode != ORC_OP_READ && opcode != ORC_OP_WRITE)) return ORC_EINVAL;
+    if (capacity == 0 || ((opcode & 0xff) != ORC_OP_READ && (opcode & 0xff) != ORC_OP_WRITE))
+        return ORC_EINVAL;
 
     /* step 1: items, one per hit object and per K / V half */
     uint64_t n_items = 0;
@@ -352,22 +370,36 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
  */
 int orc_exec(const orc_sqe *sqes, uint32_t n_sqe, const orc_sgl *sgl, uint32_t n_sgl,
              uint8_t *const *store, const uint64_t *store_bytes, uint32_t n_devices,
-             uint8_t *pool_host, uint64_t pool_base_addr, uint64_t pool_bytes)
+             uint8_t *pool_host, uint64_t pool_base_addr, uint64_t pool_bytes,
+             uint32_t n_kv_heads, uint32_t row_bytes)
 {
     for (uint32_t k = 0; k < n_sqe; ++k) {
         const orc_sqe *s = &sqes[k];
         if (s->dev >= n_devices) return ORC_EINVAL;
         if ((uint64_t)s->sgl_first + s->sgl_count > n_sgl) return ORC_EINVAL;
+        int to_pool = (s->opcode & 0xff) == ORC_OP_READ;
         uint64_t cursor = s->src_off;
         for (uint32_t e = s->sgl_first; e < s->sgl_first + s->sgl_count; ++e) {
             if (sgl[e].addr < pool_base_addr) return ORC_EINVAL;
             uint64_t poff = sgl[e].addr - pool_base_addr;
             if (poff + sgl[e].len > pool_bytes) return ORC_EINVAL;
             if (cursor + sgl[e].len > store_bytes[s->dev]) return ORC_EINVAL;
-            if (s->opcode == ORC_OP_READ)
-                memcpy(pool_host + poff, store[s->dev] + cursor, sgl[e].len);
-            else
-                memcpy(store[s->dev] + cursor, pool_host + poff, sgl[e].len);
+            uint8_t *obj = store[s->dev] + cursor, *blk = pool_host + poff;
+            if (!(s->opcode & ORC_OP_HND)) {
+                if (to_pool) memcpy(blk, obj, sgl[e].len); else memcpy(obj, blk, sgl[e].len);
+            } else {
+                /* the entry is one block: object side [token][head][row], pool side
+                 * [head][token][row] */
+                uint64_t tok_bytes = (uint64_t)n_kv_heads * row_bytes;
+                if (tok_bytes == 0 || sgl[e].len % tok_bytes) return ORC_EINVAL;
+                uint64_t n_tok = sgl[e].len / tok_bytes;
+                for (uint64_t t = 0; t < n_tok; ++t)
+                    for (uint32_t hd = 0; hd < n_kv_heads; ++hd) {
+                        uint8_t *o = obj + t * tok_bytes + (uint64_t)hd * row_bytes;
+                        uint8_t *q = blk + ((uint64_t)hd * n_tok + t) * row_bytes;
+                        if (to_pool) memcpy(q, o, row_bytes); else memcpy(o, q, row_bytes);
+                    }
+            }
             cursor += sgl[e].len;
         }
         if (cursor - s->src_off != s->len) return ORC_EINVAL;

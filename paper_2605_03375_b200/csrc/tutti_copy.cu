@@ -34,7 +34,16 @@ struct CopyParams {
     uint32_t claim_chunks;
     uint32_t stages;        // bulk engine: stages per warp
     uint32_t chunk_bytes;   // bulk engine: bytes per stage (a power of two, 4..32 KiB)
+    PermGeom perm;          // head-major pool blocks
 };
+
+// Offset inside a head-major pool block of the byte that sits at `off` in the
+// token-major object: off = (t * heads + h) * row + x  ->  (h * tokens + t) * row + x.
+__device__ __forceinline__ uint32_t hnd_offset(uint32_t off, const PermGeom &g) {
+    const uint32_t t = off / g.token_bytes, y = off - t * g.token_bytes;
+    const uint32_t hh = y / g.row_bytes, x = y - hh * g.row_bytes;
+    return (hh * g.block_tokens + t) * g.row_bytes + x;
+}
 
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
     unsigned long long t;
@@ -188,6 +197,18 @@ copy_ldst_kernel(CopyParams p) {
         const size_t e_base = (size_t)h->sgl_base + h->entry_first;
         const tutti_sgl_t *sgl = p.ring.sgl + e_base;
         const uint64_t *obj = p.ring.obj_ptr + e_base;
+        const bool hnd = (h->opcode & TUTTI_OP_FLAG_HND) != 0;
+        if (hnd && (elen == 0 || elen != p.perm.block_tokens * p.perm.token_bytes)) {
+            // a head-major entry must be exactly one block
+            if (threadIdx.x == 0) {
+                atomicCAS(&h->status, 0, TUTTI_EINVAL);
+                __threadfence();
+                if (atomicCAS(&h->state, state_word(idx, PHASE_READY), state_word(idx, PHASE_DONE)) ==
+                    state_word(idx, PHASE_READY))
+                    post_cqe(p.ring, idx, TUTTI_EINVAL, 0);
+            }
+            continue;
+        }
 
         if (elen != 0 && (elen & 511u) == 0) {
             // uniform entries, every 512-byte warp row lies inside one entry
@@ -214,14 +235,32 @@ copy_ldst_kernel(CopyParams p) {
                         if (lane == 0) { a_pool = sgl[e0].addr; a_obj = obj[e0]; }
                         a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
                         a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
-                        const char *src = reinterpret_cast<const char *>(TO_POOL ? a_obj : a_pool) +
-                                          off0 + lane * 16u;
-                        char *dst = reinterpret_cast<char *>(TO_POOL ? a_pool : a_obj) + off0 + lane * 16u;
+                        const uint32_t o_obj = off0 + lane * 16u;
                         uint4 v[8];
+                        if (!hnd) {
+                            const char *src = reinterpret_cast<const char *>(TO_POOL ? a_obj : a_pool) + o_obj;
+                            char *dst = reinterpret_cast<char *>(TO_POOL ? a_pool : a_obj) + o_obj;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) v[k] = ld_stream(src + k * 512);
+                            for (int k = 0; k < 8; ++k) v[k] = ld_stream(src + k * 512);
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) st_stream(dst + k * 512, v[k]);
+                            for (int k = 0; k < 8; ++k) st_stream(dst + k * 512, v[k]);
+                        } else {
+                            // head-major pool block: every 16-byte vector keeps its place in the
+                            // object and goes to the transposed row of the block
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint32_t oo = o_obj + k * 512u;
+                                const uint32_t op = hnd_offset(oo, p.perm);
+                                v[k] = ld_stream(reinterpret_cast<const void *>(
+                                    TO_POOL ? a_obj + oo : a_pool + op));
+                            }
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint32_t oo = o_obj + k * 512u;
+                                const uint32_t op = hnd_offset(oo, p.perm);
+                                st_stream(reinterpret_cast<void *>(TO_POOL ? a_pool + op : a_obj + oo), v[k]);
+                            }
+                        }
                         continue;
                     }
                     // small entries (512 B .. 2 KiB, e.g. 1-token pages): lanes 0..7 fetch the
@@ -241,7 +280,8 @@ copy_ldst_kernel(CopyParams p) {
                             const uint32_t e = ok ? (pow2 ? (uint32_t)(pk >> shift) : (uint32_t)(pk / elen)) : e0;
                             const uint32_t off = (uint32_t)(pk - (unsigned long long)e * elen) + lane * 16u;
                             const unsigned long long a = __shfl_sync(0xffffffffu, TO_POOL ? my_obj : my_pool, e - e0);
-                            if (ok) v[k] = ld_stream(reinterpret_cast<const void *>(a + off));
+                            const uint32_t o2 = (hnd && !TO_POOL) ? hnd_offset(off, p.perm) : off;
+                            if (ok) v[k] = ld_stream(reinterpret_cast<const void *>(a + o2));
                         }
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
@@ -250,7 +290,8 @@ copy_ldst_kernel(CopyParams p) {
                             const uint32_t e = ok ? (pow2 ? (uint32_t)(pk >> shift) : (uint32_t)(pk / elen)) : e0;
                             const uint32_t off = (uint32_t)(pk - (unsigned long long)e * elen) + lane * 16u;
                             const unsigned long long a = __shfl_sync(0xffffffffu, TO_POOL ? my_pool : my_obj, e - e0);
-                            if (ok) st_stream(reinterpret_cast<void *>(a + off), v[k]);
+                            const uint32_t o2 = (hnd && TO_POOL) ? hnd_offset(off, p.perm) : off;
+                            if (ok) st_stream(reinterpret_cast<void *>(a + o2), v[k]);
                         }
                     }
                 }
@@ -278,11 +319,13 @@ copy_ldst_kernel(CopyParams p) {
                     a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
                     a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
                     len = __shfl_sync(0xffffffffu, len, 0);
-                    const unsigned long long src = TO_POOL ? a_obj : a_pool;
-                    const unsigned long long dst = TO_POOL ? a_pool : a_obj;
-                    for (uint32_t o = lane * 16u; o < len; o += 512u)
-                        st_stream(reinterpret_cast<void *>(dst + o),
-                                  ld_stream(reinterpret_cast<const void *>(src + o)));
+                    for (uint32_t o = lane * 16u; o < len; o += 512u) {
+                        const uint32_t op = hnd ? hnd_offset(o, p.perm) : o;
+                        const unsigned long long src = TO_POOL ? a_obj + o : a_pool + op;
+                        const unsigned long long dst = TO_POOL ? a_pool + op : a_obj + o;
+                        st_stream(reinterpret_cast<void *>(dst),
+                                  ld_stream(reinterpret_cast<const void *>(src)));
+                    }
                     moved += len;
                 }
                 __syncwarp();
@@ -440,7 +483,7 @@ copy_bulk_kernel(CopyParams p) {
 
     // Entries of differing lengths (host-prepared IOCBs only): plain vector copies, one
     // entry per warp at a time, outside the staged pipeline.
-    auto copy_varlen = [&](IocbHdr *h, uint32_t idx, uint32_t total) {
+    auto copy_varlen = [&](IocbHdr *h, uint32_t idx, uint32_t total, bool hnd) {
         for (;;) {
             uint32_t c0 = 0;
             if (lane == 0) c0 = atomicAdd(&h->claim_cursor, 8u);
@@ -455,11 +498,12 @@ copy_bulk_kernel(CopyParams p) {
                 a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
                 a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
                 len = __shfl_sync(0xffffffffu, len, 0);
-                const unsigned long long src = TO_POOL ? a_obj : a_pool;
-                const unsigned long long dst = TO_POOL ? a_pool : a_obj;
-                for (uint32_t o = lane * 16u; o < len; o += 512u)
-                    st_stream(reinterpret_cast<void *>(dst + o),
-                              ld_stream(reinterpret_cast<const void *>(src + o)));
+                for (uint32_t o = lane * 16u; o < len; o += 512u) {
+                    const uint32_t op = hnd ? hnd_offset(o, p.perm) : o;
+                    const unsigned long long src = TO_POOL ? a_obj + o : a_pool + op;
+                    const unsigned long long dst = TO_POOL ? a_pool + op : a_obj + o;
+                    st_stream(reinterpret_cast<void *>(dst), ld_stream(reinterpret_cast<const void *>(src)));
+                }
                 mv += len;
             }
             __syncwarp();
@@ -488,7 +532,20 @@ copy_bulk_kernel(CopyParams p) {
             const size_t e_base = (size_t)h->sgl_base + h->entry_first;
             sgl = p.ring.sgl + e_base;
             obj = p.ring.obj_ptr + e_base;
-            if (h->entry_len == 0) { copy_varlen(h, idx, total); continue; }
+            const bool hnd = (h->opcode & TUTTI_OP_FLAG_HND) != 0;
+            if (hnd && h->entry_len != p.perm.block_tokens * p.perm.token_bytes) {
+                if (lane == 0) {
+                    atomicCAS(&h->status, 0, TUTTI_EINVAL);
+                    __threadfence();
+                    if (atomicCAS(&h->state, state_word(idx, PHASE_READY), state_word(idx, PHASE_DONE)) ==
+                        state_word(idx, PHASE_READY))
+                        post_cqe(p.ring, idx, TUTTI_EINVAL, 0);
+                }
+                continue;
+            }
+            // entries of differing lengths, and head-major blocks (a transposition the staged
+            // bulk copies cannot express), go through the per-entry vector path
+            if (h->entry_len == 0 || hnd) { copy_varlen(h, idx, total, hnd); continue; }
             f_h = h;
             f_cur_bi = bi;
             cg = chunk_geom(total, h->entry_len, CB);
@@ -624,7 +681,8 @@ cudaError_t copy_kernels_setup() {
 
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
-                        cudaStream_t stream, uint32_t *launches) {
+                        bool pool_hnd, const PermGeom &perm, cudaStream_t stream,
+                        uint32_t *launches) {
     CopyParams p;
     p.ring = ring;
     p.first_iocb = first_iocb;
@@ -633,7 +691,8 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     p.wait_ns = opt.wait_ns;
     p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : 4;
     uint32_t engine = opt.engine;
-    if (engine == 0) engine = host_store ? 1 : 2;   // measured: bulk-async wins on HBM
+    if (engine == 0) engine = (host_store || pool_hnd) ? 1 : 2;   // measured: bulk-async wins on HBM
+    p.perm = perm;
     const uint32_t sms = sm_count ? sm_count : (uint32_t)device_sms;
     if (engine == 2) {
         // measured on B200: all SMs -> 2 warps x 3 stages x 32 KiB; a capped launch gets

@@ -96,6 +96,12 @@ struct BatchDev {
     const int32_t *block_ids;
 };
 
+// What a head-major pool block needs to be addressed: tokens per block, heads, bytes of
+// one head's row of a token, bytes of a whole token.
+struct PermGeom {
+    uint32_t block_tokens, n_heads, row_bytes, token_bytes;
+};
+
 struct CopyOptions {
     uint32_t engine;        // 0 auto, 1 ld/st, 2 bulk
     uint64_t wait_ns;
@@ -115,7 +121,8 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
                         cudaStream_t stream);
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
-                        cudaStream_t stream, uint32_t *launches);
+                        bool pool_hnd, const PermGeom &perm, cudaStream_t stream,
+                        uint32_t *launches);
 cudaError_t copy_kernels_setup();
 
 }  // namespace tutti

@@ -62,6 +62,7 @@ struct tutti_ctx {
     CopyOptions opt;
     GeomDev gdev;
     void *partition = nullptr;   // SM partition state (tutti_partition.cu)
+    bool pool_hnd = false;       // pool blocks are [head][token][dim]
 };
 
 struct tutti_ring {
@@ -230,6 +231,10 @@ int tutti_set_option(tutti_ctx_t *ctx, uint32_t option, uint64_t value) {
             if (value < 1 || value > 1024) return TUTTI_EINVAL;
             ctx->opt.claim_chunks = (uint32_t)value;
             return TUTTI_OK;
+        case TUTTI_OPT_POOL_LAYOUT:
+            if (value > TUTTI_POOL_HND) return TUTTI_EINVAL;
+            ctx->pool_hnd = value == TUTTI_POOL_HND;
+            return TUTTI_OK;
         case TUTTI_OPT_BULK_CHUNK_BYTES:
             if (value < 4096 || value > 32768 || (value & (value - 1))) return TUTTI_EINVAL;
             ctx->opt.bulk_chunk = (uint32_t)value;
@@ -376,7 +381,8 @@ int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *bat
         sbase[d] = ctx->store[d].base;
         sbytes[d] = ctx->store[d].bytes;
     }
-    CK(launch_emit(r->dev, ctx->gdev, b, layer, opcode, ctx->pool[layer], sbase, sbytes, first,
+    const uint32_t op_flags = opcode | (ctx->pool_hnd ? TUTTI_OP_FLAG_HND : 0u);
+    CK(launch_emit(r->dev, ctx->gdev, b, layer, op_flags, ctx->pool[layer], sbase, sbytes, first,
                    need_iocb, sgl_base, need_sgl, ctx->device_sms, st));
     r->kernel_launches++;
     *first_iocb = first;
@@ -400,8 +406,10 @@ static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, 
     }
     DeviceGuard guard(ctx->device);
     uint32_t launches = 0;
+    PermGeom pg{ctx->geom.block_tokens, ctx->geom.n_kv_heads,
+                ctx->geom.head_dim * ctx->geom.elem_bytes, (uint32_t)ctx->layout.token_bytes};
     CK(launch_copy(r->dev, first, n, opcode, sm_count, ctx->device_sms, ctx->opt, host_store,
-                   (cudaStream_t)stream, &launches));
+                   ctx->pool_hnd, pg, (cudaStream_t)stream, &launches));
     r->kernel_launches += launches;
     return TUTTI_OK;
 }
@@ -490,6 +498,8 @@ int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
         const tutti_sqe_t &s = sqes[k];
         if (s.dev >= ctx->geom.n_devices || !ctx->store[s.dev].registered) return TUTTI_EINVAL;
         if (s.opcode != opcode || (uint64_t)s.sgl_first + s.sgl_count > n_sgl) return TUTTI_EINVAL;
+        if ((s.opcode & 0xff) > TUTTI_OP_WRITE || (s.opcode & ~(0xffu | TUTTI_OP_FLAG_HND)))
+            return TUTTI_EINVAL;
         uint64_t cursor = s.src_off;
         for (uint32_t e = s.sgl_first; e < s.sgl_first + s.sgl_count; ++e) {
             if (seen[e] || (sgl[e].len & 15) || (sgl[e].addr & 15) || sgl[e].len == 0) return TUTTI_EINVAL;
@@ -530,7 +540,7 @@ int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
     h.bytes = total;
     // stream order publishes the header after the descriptors it refers to
     CK(cudaMemcpyAsync(&r->dev.hdrs[slot], &h, sizeof(h), cudaMemcpyHostToDevice, st));
-    r->opcode_of[slot] = (uint8_t)opcode;
+    r->opcode_of[slot] = (uint8_t)(opcode & 0xff);
     return TUTTI_OK;
 }
 

@@ -145,7 +145,10 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
             e = launch_emit(r, g, b, layer, TUTTI_OP_READ, pool, sbase, sbytes, 0, 1, 0,
                             NA_MAX_ENTRIES, sms, st);
         if (e == cudaSuccess)
-            e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, st, &launches);
+            e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, false,
+                            PermGeom{geom->block_tokens, geom->n_kv_heads,
+                                     geom->head_dim * geom->elem_bytes, (uint32_t)lo.token_bytes},
+                            st, &launches);
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(cqe_out, base + OFF_CQ, sizeof(tutti_cqe_t), cudaMemcpyDefault, st);
         if (e != cudaSuccess) rc = TUTTI_ECUDA;

@@ -19,7 +19,9 @@ LAYOUT_FILE_MAJOR, LAYOUT_LAYER_MAJOR = 0, 1
 OP_READ, OP_WRITE = 0, 1
 STORE_HBM, STORE_HOST_PINNED = 0, 1
 OPT_COPY_ENGINE, OPT_WAIT_NS, OPT_CTAS_PER_SM, OPT_BULK_WARPS, OPT_BULK_STAGES, OPT_CLAIM_CHUNKS, \
-    OPT_BULK_CHUNK_BYTES = 1, 2, 3, 4, 5, 6, 7
+    OPT_BULK_CHUNK_BYTES, OPT_POOL_LAYOUT = 1, 2, 3, 4, 5, 6, 7, 8
+POOL_NHD, POOL_HND = 0, 1
+OP_FLAG_HND = 0x100
 ENGINE_AUTO, ENGINE_LDST, ENGINE_BULK = 0, 1, 2
 
 

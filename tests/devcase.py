@@ -19,6 +19,9 @@ class DeviceCase:
         self.layers = list(range(w.n_layers)) if layers is None else list(layers)
         self.dev = torch.device("cuda", device)
         self.ctx = T.Context(T.geom_of(w), device)
+        self.hnd = bool(getattr(w, "pool_hnd", False))
+        if self.hnd:
+            self.ctx.tutti_set_option(T.OPT_POOL_LAYOUT, T.POOL_HND)
         lo = self.ctx.layout
         assert lo.dev_bytes == self.olo.dev_bytes
         # object store
@@ -67,19 +70,21 @@ class DeviceCase:
     # ---- oracle side -----------------------------------------------------
     def oracle_descriptors(self, layer, opcode, capacity):
         base = self.pool_dev[layer].data_ptr()
+        if self.hnd:
+            opcode |= oracle.OP_HND
         return oracle.build_descriptors(self.og, layer, opcode, self.obatch, base + self.k_off,
                                         base + self.v_off, self.stride, capacity)
 
     def oracle_restore(self, layer):
         pool = self.pool_host[layer].copy()
         rc = oracle.restore_layer(self.og, layer, self.obatch, self.store_host, pool, self.k_off,
-                                  self.v_off, self.stride, self.w.n_pool_blocks)
+                                  self.v_off, self.stride, self.w.n_pool_blocks, self.hnd)
         assert rc == 0
         return pool
 
     def oracle_save(self, layer, pool_host, store_host):
         rc = oracle.save_layer(self.og, layer, self.obatch, store_host, pool_host, self.k_off,
-                               self.v_off, self.stride, self.w.n_pool_blocks)
+                               self.v_off, self.stride, self.w.n_pool_blocks, self.hnd)
         assert rc == 0
 
     # ---- CUDA side -------------------------------------------------------

@@ -127,7 +127,17 @@ def _store_nd(store, w, lo, d):
 def _expected_pool_numpy(w, lo, store, pool_before, layer):
     tb = int(lo.token_bytes)
     exp = pool_before.copy()
-    if w.pool_interleaved:
+    if w.pool_hnd:
+        # a block is [head][token][row]: present it as [token][head * row] through a view
+        row = w.head_dim * w.elem_bytes
+        if w.pool_interleaved:
+            nd = exp.reshape(w.n_pool_blocks, 2, w.n_kv_heads, w.block_tokens, row)
+            nd = nd.transpose(1, 0, 3, 2, 4)
+        else:
+            nd = exp.reshape(2, w.n_pool_blocks, w.n_kv_heads, w.block_tokens, row)
+            nd = nd.transpose(0, 1, 3, 2, 4)
+        # nd is now [kv][block][token][head][row]
+    elif w.pool_interleaved:
         nd = exp.reshape(w.n_pool_blocks, 2, w.block_tokens, tb).transpose(1, 0, 2, 3)
     else:
         nd = exp.reshape(2, w.n_pool_blocks, w.block_tokens, tb)
@@ -147,6 +157,8 @@ def _expected_pool_numpy(w, lo, store, pool_before, layer):
                     src = snd[loc, layer, kv, t[sel] % w.obj_tokens]
                 else:
                     src = snd[layer, loc, kv, t[sel] % w.obj_tokens]
+                if w.pool_hnd:
+                    src = src.reshape(src.shape[0], w.n_kv_heads, -1)
                 nd[kv, blk[sel], t[sel] % w.block_tokens] = src
     return exp
 
@@ -159,6 +171,9 @@ CASES = [
     dict(index=4, scale=0.02, n_layers=2, n_devices=3, layout=wl.LAYOUT_FILE_MAJOR),
     dict(index=3, scale=0.02, n_layers=2),
     dict(index=1),
+    dict(index=2, scale=0.03, n_layers=2, pool_hnd=True),
+    dict(index=4, scale=0.02, n_layers=2, pool_hnd=True, pool_interleaved=True, n_kv_heads=4,
+         head_dim=32, block_tokens=4, obj_tokens=32),
 ]
 
 
@@ -181,7 +196,7 @@ def test_restore_equals_numpy_indexing(case):
         pool0 = hc.make_pool_layer(w, lo, layer)
         pool = pool0.copy()
         rc = oracle.restore_layer(g, layer, hc.batch_of(w), store, pool, k_off, v_off, stride,
-                                  w.n_pool_blocks)
+                                  w.n_pool_blocks, w.pool_hnd)
         assert rc == oracle.OK
         exp = _expected_pool_numpy(w, lo, store, pool0, layer)
         assert np.array_equal(pool, exp)
@@ -219,7 +234,8 @@ def test_identity_table_is_memcpy():
 # invariants: round trip, untouched bytes, exec(build) == restore
 # --------------------------------------------------------------------------
 
-@pytest.mark.parametrize("case", CASES[:5], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
+@pytest.mark.parametrize("case", CASES[:5] + CASES[7:],
+                         ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
 def test_round_trip_and_untouched(case):
     w, g, lo = _mk(case)
     store = hc.make_store(w, lo)
@@ -228,11 +244,11 @@ def test_round_trip_and_untouched(case):
     batch = hc.batch_of(w)
     pool = hc.make_pool_layer(w, lo, layer)
     assert oracle.restore_layer(g, layer, batch, store, pool, k_off, v_off, stride,
-                                w.n_pool_blocks) == 0
+                                w.n_pool_blocks, w.pool_hnd) == 0
     # save into a zeroed store: covered ranges reproduce the original store, rest stays zero
     st2 = [np.zeros_like(s) for s in store]
     assert oracle.save_layer(g, layer, batch, st2, pool, k_off, v_off, stride,
-                             w.n_pool_blocks) == 0
+                             w.n_pool_blocks, w.pool_hnd) == 0
     covered = [np.zeros(s.nbytes, dtype=bool) for s in store]
     tb = int(lo.token_bytes)
     for r in range(w.n_req):
@@ -253,7 +269,7 @@ def test_round_trip_and_untouched(case):
     batch2 = (w.hit_tokens, w.obj_start, w.obj_slot, w2.blk_start, w2.block_ids)
     pool2 = np.zeros(nbytes, dtype=np.uint8)
     assert oracle.restore_layer(g, layer, batch2, st2, pool2, k_off, v_off, stride,
-                                w.n_pool_blocks) == 0
+                                w.n_pool_blocks, w.pool_hnd) == 0
     bb = int(lo.block_bytes)
     for plane in (k_off, v_off):
         for i in range(0, len(w.block_ids), max(1, len(w.block_ids) // 64)):
@@ -270,9 +286,12 @@ def test_descriptors(case, capacity):
     base = 0x7F0000000000
     layer = w.n_layers - 1
     batch = hc.batch_of(w)
-    rc, sqes, sgl, num = oracle.build_descriptors(g, layer, oracle.OP_READ, batch, base + k_off,
-                                                  base + v_off, stride, capacity)
+    flag = oracle.OP_HND if w.pool_hnd else 0
+    rowb = w.head_dim * w.elem_bytes
+    rc, sqes, sgl, num = oracle.build_descriptors(g, layer, oracle.OP_READ | flag, batch,
+                                                  base + k_off, base + v_off, stride, capacity)
     assert rc == 0
+    assert np.all(sqes["opcode"] == (oracle.OP_READ | flag))
     tb, bb = int(lo.token_bytes), int(lo.block_bytes)
     payload = w.total_tokens * 2 * tb
     # total length = payload; sgl_first = exclusive prefix sum of sgl_count
@@ -305,18 +324,18 @@ def test_descriptors(case, capacity):
     pool_a = hc.make_pool_layer(w, lo, layer)
     pool_b = pool_a.copy()
     assert oracle.restore_layer(g, layer, batch, store, pool_a, k_off, v_off, stride,
-                                w.n_pool_blocks) == 0
-    assert oracle.exec_descriptors(sqes, sgl, store, pool_b, base) == 0
+                                w.n_pool_blocks, w.pool_hnd) == 0
+    assert oracle.exec_descriptors(sqes, sgl, store, pool_b, base, w.n_kv_heads, rowb) == 0
     assert np.array_equal(pool_a, pool_b)
     # and the WRITE direction reproduces the plain save
-    rc, sq_w, sgl_w, _ = oracle.build_descriptors(g, layer, oracle.OP_WRITE, batch, base + k_off,
-                                                  base + v_off, stride, capacity)
-    assert rc == 0 and np.all(sq_w["opcode"] == oracle.OP_WRITE)
+    rc, sq_w, sgl_w, _ = oracle.build_descriptors(g, layer, oracle.OP_WRITE | flag, batch,
+                                                  base + k_off, base + v_off, stride, capacity)
+    assert rc == 0 and np.all(sq_w["opcode"] == (oracle.OP_WRITE | flag))
     st_a = [np.zeros_like(s) for s in store]
     st_b = [np.zeros_like(s) for s in store]
     assert oracle.save_layer(g, layer, batch, st_a, pool_a, k_off, v_off, stride,
-                             w.n_pool_blocks) == 0
-    assert oracle.exec_descriptors(sq_w, sgl_w, st_b, pool_a, base) == 0
+                             w.n_pool_blocks, w.pool_hnd) == 0
+    assert oracle.exec_descriptors(sq_w, sgl_w, st_b, pool_a, base, w.n_kv_heads, rowb) == 0
     for a, b in zip(st_a, st_b):
         assert np.array_equal(a, b)
 
@@ -433,3 +452,39 @@ def test_paper_counts():
     assert 60 * 1024 ** 3 // 4096 == gold["prp_pages_60gb"]
     # Section 3.2: one IOCB holds 2048 contexts = 2 SMs x 64 warps x 32 threads / 2
     assert 2 * 64 * 32 // 2 == gold["ioctx_per_iocb"]
+
+
+def test_head_major_block_by_enumeration():
+    """Head-major pool block, tiny and explicit: the block is written down in pool order
+    (for each head, for each token, one row) and compared with what restore leaves there."""
+    H, D, bt = 3, 8, 4                                   # rows of 16 bytes
+    g = oracle.geom(1, H, D, 2, bt, 2 * bt, 1, oracle.LAYER_MAJOR, 2)
+    row = D * 2
+    store = np.zeros(2 * 2 * 2 * bt * H * row, dtype=np.uint8)     # 2 slots x {K,V} x 8 tokens
+    cells = store.reshape(2, 2, 2 * bt, H, row)                    # [slot][kv][token][head][row]
+    for s in range(2):
+        for kv in range(2):
+            for t in range(2 * bt):
+                for h in range(H):
+                    cells[s, kv, t, h, :] = [s + 1, kv + 1, t + 1, h + 1] * (row // 4)
+    n_pool = 5
+    ids = [3, 0]                                          # token 0..3 -> block 3, 4..7 -> block 0
+    batch = ([2 * bt], [0, 1], [1], [0, 2], ids)          # one request, object slot 1
+    pool = np.zeros(2 * n_pool * bt * H * row, dtype=np.uint8)
+    bb = bt * H * row
+    assert oracle.restore_layer(g, 0, batch, [store], pool, 0, n_pool * bb, bb, n_pool, True) == 0
+    for kv in range(2):
+        for j, blk in enumerate(ids):
+            want = []
+            for h in range(H):                            # pool order: head, then token
+                for tt in range(bt):
+                    want += [2, kv + 1, j * bt + tt + 1, h + 1] * (row // 4)
+            o = kv * n_pool * bb + blk * bb
+            assert pool[o:o + bb].tolist() == want
+    untouched = [b for b in range(n_pool) if b not in ids]
+    for b in untouched:
+        assert not pool[b * bb:(b + 1) * bb].any()
+    # and back
+    st2 = np.zeros_like(store)
+    assert oracle.save_layer(g, 0, batch, [st2], pool, 0, n_pool * bb, bb, n_pool, True) == 0
+    assert np.array_equal(st2.reshape(2, -1)[1], store.reshape(2, -1)[1]) and not st2.reshape(2, -1)[0].any()

@@ -168,6 +168,8 @@ class Replica:
         self.dev = torch.device("cuda", device_index)
         torch.cuda.set_device(self.dev)
         over = {}
+        if getattr(args, "pool_hnd", False):
+            over["pool_hnd"] = True
         if n_layers is None and getattr(args, "layers", 0):
             n_layers = args.layers
         if n_layers is not None:
@@ -175,6 +177,8 @@ class Replica:
         self.w = w = wl.config(args.config, args.scale, **over)
         self.geom = T.geom_of(w)
         self.ctx = T.Context(self.geom, device_index)
+        if w.pool_hnd:
+            self.ctx.tutti_set_option(T.OPT_POOL_LAYOUT, T.POOL_HND)
         lo = self.lo = self.ctx.layout
         self.block_bytes = int(lo.block_bytes)
         self.payload_per_layer = w.total_tokens * 2 * int(lo.token_bytes)
@@ -308,16 +312,17 @@ class Replica:
         og = oracle.geom_of(w)
         ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
         rng = np.random.default_rng(1234)
-        tb = int(self.lo.token_bytes)
+        row = w.head_dim * w.elem_bytes
         for _ in range(n_samples):
             l = int(rng.integers(w.n_layers - self.R, w.n_layers))   # layers whose pool buffer is still theirs
             r = int(rng.integers(0, w.n_req))
             t = int(rng.integers(0, int(w.hit_tokens[r])))
             kv = int(rng.integers(0, 2))
-            d, so, blk, ro = oracle.token_location(og, l, ob, r, t, kv)
-            po = kv * self.v_off + blk * self.block_bytes + ro
-            a = self.store[d][so:so + tb].to(self.dev)
-            b = self.pool[l % self.R][po:po + tb]
+            hd = int(rng.integers(0, w.n_kv_heads))
+            d, so, blk, bo = oracle.row_location(og, l, ob, r, t, kv, hd, w.pool_hnd)
+            po = kv * self.v_off + blk * self.block_bytes + bo
+            a = self.store[d][so:so + row].to(self.dev)
+            b = self.pool[l % self.R][po:po + row]
             if not torch.equal(a, b):
                 return False
         return True
@@ -343,9 +348,9 @@ def cpu_baseline(rep, seconds_hint=12.0):
         pool = rep.pool[l % rep.R].cpu().numpy()
         t0 = time.perf_counter()
         rc1 = oracle.restore_layer(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
-                                   w.n_pool_blocks)
+                                   w.n_pool_blocks, w.pool_hnd)
         rc2 = oracle.save_layer(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
-                                w.n_pool_blocks)
+                                w.n_pool_blocks, w.pool_hnd)
         t_total += time.perf_counter() - t0
         assert rc1 == 0 and rc2 == 0
         done_bytes += 2 * rep.payload_per_layer
@@ -907,6 +912,8 @@ def main():
     ap.add_argument("--sched-gemms", type=int, default=3)
     ap.add_argument("--one-stream", action="store_true",
                     help="build and copy on one stream (default: descriptors on their own stream)")
+    ap.add_argument("--pool-hnd", action="store_true",
+                    help="head-major pool blocks [head][token][dim] (transposing copy)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -155,6 +155,25 @@ def token_location(g: Geom, layer: int, batch, r: int, t: int, kv: int
     return dev.value, soff.value, blk.value, roff.value
 
 
+def row_location(g: Geom, layer: int, batch, r: int, t: int, kv: int, head: int,
+                 pool_hnd: bool = False) -> Tuple[int, int, int, int]:
+    """(device, store byte offset, pool block id, byte offset inside the block) of one head's
+    row of token t of request r, for token-major or head-major pool blocks."""
+    keep, bargs = _batch(*batch)
+    dev = C.c_uint32()
+    soff = C.c_uint64()
+    blk = C.c_int64()
+    boff = C.c_uint64()
+    rc = lib().orc_row_location(C.byref(g), C.c_uint32(layer), *bargs[2:], C.c_uint32(r),
+                                C.c_uint64(t), C.c_uint32(kv), C.c_uint32(head),
+                                C.c_int(1 if pool_hnd else 0), C.byref(dev), C.byref(soff),
+                                C.byref(blk), C.byref(boff))
+    del keep
+    if rc != OK:
+        raise ValueError(f"orc_row_location: {rc}")
+    return dev.value, soff.value, blk.value, boff.value
+
+
 def build_descriptors(g: Geom, layer: int, opcode: int, batch, k_base_addr: int,
                       v_base_addr: int, block_stride: int, capacity: int):
     """Returns (rc, sqes, sgl, num_ioctx) — structured arrays SQE_DTYPE / SGL_DTYPE and the

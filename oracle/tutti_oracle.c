@@ -171,6 +171,31 @@ int orc_token_location(const orc_geom *g, uint32_t layer, const uint32_t *obj_st
                           dev, store_off, block, row_off);
 }
 
+/* One head's row of one token: where it sits in the store and inside its pool block,
+ * for either element order of the block. */
+int orc_row_location(const orc_geom *g, uint32_t layer, const uint32_t *obj_start,
+                     const uint32_t *obj_slot, const uint32_t *blk_start,
+                     const int32_t *block_ids, uint32_t r, uint64_t t, uint32_t kv, uint32_t head,
+                     int pool_hnd, uint32_t *dev, uint64_t *store_off, int64_t *block,
+                     uint64_t *off_in_block)
+{
+    orc_layout lo;
+    uint64_t tok_off;
+    int rc = orc_obj_layout(g, &lo);
+    if (rc) return rc;
+    if (head >= g->n_kv_heads) return ORC_EINVAL;
+    rc = token_location(g, &lo, layer, obj_start, obj_slot, blk_start, block_ids, r, t, kv, dev,
+                        store_off, block, &tok_off);
+    if (rc) return rc;
+    uint64_t row = (uint64_t)g->head_dim * g->elem_bytes;
+    *store_off += head * row;
+    if (pool_hnd)
+        *off_in_block = ((uint64_t)head * g->block_tokens + t % g->block_tokens) * row;
+    else
+        *off_in_block = tok_off + head * row;
+    return ORC_OK;
+}
+
 static int move_layer(const orc_geom *g, uint32_t layer, uint32_t n_req,
                       const uint32_t *hit_tokens, const uint32_t *obj_start,
                       const uint32_t *obj_slot, const uint32_t *blk_start,

@@ -488,3 +488,26 @@ def test_head_major_block_by_enumeration():
     st2 = np.zeros_like(store)
     assert oracle.save_layer(g, 0, batch, [st2], pool, 0, n_pool * bb, bb, n_pool, True) == 0
     assert np.array_equal(st2.reshape(2, -1)[1], store.reshape(2, -1)[1]) and not st2.reshape(2, -1)[0].any()
+
+
+def test_row_location_agrees_with_restore():
+    """The single-row locator used for sampled checks at full size names exactly the bytes
+    that restore moves, for both element orders of a pool block."""
+    for hnd in (False, True):
+        w = wl.config(2, 0.03, n_layers=2, pool_hnd=hnd)
+        g = oracle.geom_of(w)
+        lo = oracle.obj_layout(g)
+        store = hc.make_store(w, lo)
+        nbytes, k_off, v_off, stride = hc.pool_geometry(w, lo)
+        pool = np.zeros(nbytes, dtype=np.uint8)
+        batch = hc.batch_of(w)
+        assert oracle.restore_layer(g, 1, batch, store, pool, k_off, v_off, stride,
+                                    w.n_pool_blocks, hnd) == 0
+        row = w.head_dim * w.elem_bytes
+        rng = np.random.default_rng(0)
+        for _ in range(300):
+            r = int(rng.integers(0, w.n_req)); t = int(rng.integers(0, int(w.hit_tokens[r])))
+            kv = int(rng.integers(0, 2)); hd = int(rng.integers(0, w.n_kv_heads))
+            d, so, blk, bo = oracle.row_location(g, 1, batch, r, t, kv, hd, hnd)
+            po = (v_off if kv else k_off) + blk * stride + bo
+            assert np.array_equal(pool[po:po + row], store[d][so:so + row])

@@ -170,6 +170,9 @@ class Replica:
         over = {}
         if getattr(args, "pool_hnd", False):
             over["pool_hnd"] = True
+        for kv in getattr(args, "set", None) or []:
+            k, v = kv.split("=")
+            over[k] = int(v)
         if n_layers is None and getattr(args, "layers", 0):
             n_layers = args.layers
         if n_layers is not None:
@@ -914,6 +917,8 @@ def main():
                     help="build and copy on one stream (default: descriptors on their own stream)")
     ap.add_argument("--pool-hnd", action="store_true",
                     help="head-major pool blocks [head][token][dim] (transposing copy)")
+    ap.add_argument("--set", action="append", metavar="KEY=INT",
+                    help="override a workload field, e.g. layout=0 n_devices=2 elem_bytes=1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

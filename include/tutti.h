@@ -37,6 +37,7 @@ extern "C" {
 #define TUTTI_ETIMEDOUT (-4) /* a bounded device-side wait ran out                       */
 #define TUTTI_EFAULT (-5)    /* a block id or object slot points outside its region      */
 #define TUTTI_ECUDA (-6)     /* a CUDA call failed; see tutti_last_cuda_error()          */
+#define TUTTI_ENOENT (-7)    /* key not in the file pool                                 */
 
 #define TUTTI_LAYOUT_FILE_MAJOR 0  /* a file = all layers of one chunk; files back to back */
 #define TUTTI_LAYOUT_LAYER_MAJOR 1 /* all objects of a layer together; layers back to back */
@@ -395,6 +396,31 @@ int tutti_sched_enqueue(tutti_sched_t *sched, uint32_t opcode, uint32_t layer, u
 int tutti_sched_next(tutti_sched_t *sched, uint32_t phase, uint32_t layer, uint32_t l_input,
                      uint32_t l_prefix, tutti_launch_t *out, uint32_t max_out, uint32_t *n_out);
 int tutti_sched_pending(const tutti_sched_t *sched, uint32_t *reads, uint32_t *writes);
+
+/* ------------------------------------------------------------------------- */
+/* CPU-side GPU-file pool (Section 3.1 "Scalable GPU File Pool").  Host only.  */
+/* ------------------------------------------------------------------------- */
+typedef struct tutti_filepool tutti_filepool_t;
+
+/* Every object slot exists from the start and is free.  Keys are 64-bit hashes of a
+ * chunk's token prefix (computed by the engine). */
+int tutti_filepool_create(uint64_t n_slots, tutti_filepool_t **out);
+int tutti_filepool_destroy(tutti_filepool_t *pool);
+/* Slot for a chunk that is about to be saved: the slot it already has (*was_present = 1,
+ * shared by every request with that prefix), else the free slot with the lowest id, else
+ * the slot of the least recently used unpinned chunk (evicted).  TUTTI_EAGAIN when every
+ * slot is pinned. */
+int tutti_filepool_insert(tutti_filepool_t *pool, uint64_t key, uint32_t *slot, int *was_present);
+int tutti_filepool_lookup(tutti_filepool_t *pool, uint64_t key, uint32_t *slot); /* or TUTTI_ENOENT */
+/* Longest stored prefix of a request's chunk keys: slots[0..*n_hit) are filled in chunk
+ * order (ready to be a row of tutti_batch_t.obj_slot).  pin != 0 pins every hit slot
+ * until tutti_filepool_pin(slot, -1). */
+int tutti_filepool_match_prefix(tutti_filepool_t *pool, const uint64_t *keys, uint32_t n_keys,
+                                uint32_t *slots, uint32_t *n_hit, int pin);
+int tutti_filepool_pin(tutti_filepool_t *pool, uint32_t slot, int delta);
+int tutti_filepool_remove(tutti_filepool_t *pool, uint64_t key); /* TUTTI_EAGAIN while pinned */
+int tutti_filepool_stats(const tutti_filepool_t *pool, uint64_t *used, uint64_t *free_slots,
+                         uint64_t *hits, uint64_t *misses, uint64_t *evictions);
 
 /* Host-side ring accounting on its own (no GPU involved; used by CPU tests):
  * the reservation / release bookkeeping that tutti_build_sqes and tutti_ring_poll

@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libtutti.so")
 SOURCES = ["tutti_lib.cu", "tutti_build.cu", "tutti_copy.cu", "tutti_partition.cu", "tutti_noalloc.cu",
-           "host_ring.cpp", "tutti_sched.cpp"]
+           "host_ring.cpp", "tutti_sched.cpp", "tutti_filepool.cpp"]
 
 
 def _stale() -> bool:

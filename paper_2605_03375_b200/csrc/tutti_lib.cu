@@ -102,6 +102,7 @@ const char *tutti_strerror(int code) {
         case TUTTI_ETIMEDOUT: return "device-side wait timed out";
         case TUTTI_EFAULT: return "block id or slot out of range";
         case TUTTI_ECUDA: return "CUDA error";
+        case TUTTI_ENOENT: return "no such key";
         default: return "unknown";
     }
 }

@@ -14,7 +14,7 @@ import numpy as np
 
 from . import _build
 
-OK, EINVAL, ENOMEM, EAGAIN, ETIMEDOUT, EFAULT, ECUDA = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, ENOMEM, EAGAIN, ETIMEDOUT, EFAULT, ECUDA, ENOENT = 0, -1, -2, -3, -4, -5, -6, -7
 LAYOUT_FILE_MAJOR, LAYOUT_LAYER_MAJOR = 0, 1
 OP_READ, OP_WRITE = 0, 1
 STORE_HBM, STORE_HOST_PINNED = 0, 1
@@ -76,6 +76,9 @@ EXPORTS = [
     "tutti_sched_create", "tutti_sched_destroy", "tutti_sched_set_slack",
     "tutti_sched_set_decode_slack", "tutti_sched_set_io_time", "tutti_sched_io_time",
     "tutti_sched_enqueue", "tutti_sched_next", "tutti_sched_pending",
+    "tutti_filepool_create", "tutti_filepool_destroy", "tutti_filepool_insert",
+    "tutti_filepool_lookup", "tutti_filepool_match_prefix", "tutti_filepool_pin",
+    "tutti_filepool_remove", "tutti_filepool_stats",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -130,6 +133,14 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_sched_enqueue": (C.c_int, [vp, u32, u32, u32, u32]),
         "tutti_sched_next": (C.c_int, [vp, u32, u32, u32, u32, P(Launch), u32, P(u32)]),
         "tutti_sched_pending": (C.c_int, [vp, P(u32), P(u32)]),
+        "tutti_filepool_create": (C.c_int, [u64, P(vp)]),
+        "tutti_filepool_destroy": (C.c_int, [vp]),
+        "tutti_filepool_insert": (C.c_int, [vp, u64, P(u32), P(C.c_int)]),
+        "tutti_filepool_lookup": (C.c_int, [vp, u64, P(u32)]),
+        "tutti_filepool_match_prefix": (C.c_int, [vp, vp, u32, vp, P(u32), C.c_int]),
+        "tutti_filepool_pin": (C.c_int, [vp, u32, C.c_int]),
+        "tutti_filepool_remove": (C.c_int, [vp, u64]),
+        "tutti_filepool_stats": (C.c_int, [vp, P(u64), P(u64), P(u64), P(u64), P(u64)]),
         "tutti_kv_restore_layer_noalloc": (C.c_int, [P(Geom), C.c_int, u32, P(Batch), vp, vp, u64,
                                                      u64, P(vp), P(u64), vp, vp]),
     }
@@ -384,3 +395,52 @@ class Scheduler:
         a, b = C.c_uint32(), C.c_uint32()
         _check(self.lib.tutti_sched_pending(self.h, C.byref(a), C.byref(b)), "tutti_sched_pending")
         return a.value, b.value
+
+
+class FilePool:
+    """tutti_filepool_t: CPU-side chunk-key -> object-slot index with a pre-allocated slot pool."""
+
+    def __init__(self, n_slots: int):
+        self.lib = load()
+        h = C.c_void_p()
+        _check(self.lib.tutti_filepool_create(n_slots, C.byref(h)), "tutti_filepool_create")
+        self.h = h
+
+    def close(self):
+        if self.h:
+            self.lib.tutti_filepool_destroy(self.h)
+            self.h = None
+
+    def tutti_filepool_insert(self, key: int, allow: Sequence[int] = ()):
+        slot, was = C.c_uint32(), C.c_int()
+        rc = _check(self.lib.tutti_filepool_insert(self.h, key, C.byref(slot), C.byref(was)),
+                    "tutti_filepool_insert", allow)
+        return rc, slot.value, bool(was.value)
+
+    def tutti_filepool_lookup(self, key: int):
+        slot = C.c_uint32()
+        rc = _check(self.lib.tutti_filepool_lookup(self.h, key, C.byref(slot)),
+                    "tutti_filepool_lookup", (ENOENT,))
+        return rc, slot.value
+
+    def tutti_filepool_match_prefix(self, keys: np.ndarray, pin: bool = False) -> np.ndarray:
+        keys = np.ascontiguousarray(keys, dtype=np.uint64)
+        slots = np.zeros(max(len(keys), 1), dtype=np.uint32)
+        n = C.c_uint32()
+        _check(self.lib.tutti_filepool_match_prefix(self.h, keys.ctypes.data, len(keys),
+                                                    slots.ctypes.data, C.byref(n), int(pin)),
+               "tutti_filepool_match_prefix")
+        return slots[:n.value].copy()
+
+    def tutti_filepool_pin(self, slot: int, delta: int, allow: Sequence[int] = ()):
+        return _check(self.lib.tutti_filepool_pin(self.h, slot, delta), "tutti_filepool_pin", allow)
+
+    def tutti_filepool_remove(self, key: int):
+        return _check(self.lib.tutti_filepool_remove(self.h, key), "tutti_filepool_remove",
+                      (ENOENT, EAGAIN))
+
+    def tutti_filepool_stats(self):
+        v = [C.c_uint64() for _ in range(5)]
+        _check(self.lib.tutti_filepool_stats(self.h, *[C.byref(x) for x in v]),
+               "tutti_filepool_stats")
+        return dict(zip(("used", "free", "hits", "misses", "evictions"), (x.value for x in v)))

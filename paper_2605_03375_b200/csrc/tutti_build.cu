@@ -75,6 +75,93 @@ __device__ void bitonic_sort(unsigned long long *key, uint32_t *idx, uint32_t n)
     }
 }
 
+// Sort key of item q = 2 * object + kv: (device << 56) | byte offset at layer 0, or KEY_NONE
+// when the object holds no hit token (or q is padding).  A slot out of range is reported.
+__device__ unsigned long long item_key(const GeomDev &g, const BatchDev &b, uint32_t q,
+                                       int32_t *status) {
+    if (q >= 2u * b.n_obj || b.n_req == 0) return KEY_NONE;
+    const uint32_t o = q >> 1, kv = q & 1;
+    const uint32_t r = find_request(b.obj_start, b.n_req, o);
+    if (o < b.obj_start[r] || o >= b.obj_start[r + 1]) return KEY_NONE;
+    const uint32_t c = o - b.obj_start[r];
+    if (valid_tokens(b.hit_tokens[r], c, g.obj_tokens) == 0) return KEY_NONE;
+    const unsigned long long slot = b.obj_slot[o];
+    if (slot >= g.n_slots) {
+        note_error(status, TUTTI_EFAULT);
+        return KEY_NONE;
+    }
+    const unsigned long long dev = slot % g.n_devices;
+    const unsigned long long off = (slot / g.n_devices) * g.stride_slot +
+                                   (unsigned long long)kv * g.stride_kv;
+    return (dev << 56) | off;
+}
+
+// ---- batches too large for one CTA's shared memory: the same bitonic network, run as a
+// ---- few launches.  Stages whose partners lie inside one aligned tile of SORT_TILE
+// ---- elements run in shared memory, one CTA per tile; the others are one global
+// ---- compare-exchange pass each.
+constexpr uint32_t SORT_TILE = 8192;
+
+__global__ void __launch_bounds__(256)
+plan_keys_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np) {
+    const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q == 0) ring.plan_counts[1].status = 0;
+    if (q >= np) return;
+    int32_t st = 0;
+    ring.plan_key[q] = item_key(g, b, q, &st);
+    ring.plan_idx[q] = q;
+    if (st) atomicCAS(&ring.plan_counts[1].status, 0, st);
+}
+
+__device__ __forceinline__ void cmp_exchange(unsigned long long *key, uint32_t *idx, uint32_t i,
+                                             uint32_t p, bool up) {
+    unsigned long long ka = key[i], kb = key[p];
+    uint32_t ia = idx[i], ib = idx[p];
+    bool swap = up ? pair_less(kb, ib, ka, ia) : pair_less(ka, ia, kb, ib);
+    if (swap) {
+        key[i] = kb; key[p] = ka;
+        idx[i] = ib; idx[p] = ia;
+    }
+}
+
+// For k = k_first, 2*k_first, ..., k_last: the stages j = min(k/2, SORT_TILE/2) ... 1.
+__global__ void __launch_bounds__(PLAN_THREADS, 1)
+bitonic_tile_kernel(unsigned long long *gkey, uint32_t *gidx, uint32_t k_first, uint32_t k_last) {
+    extern __shared__ __align__(16) unsigned char dyn_smem[];
+    unsigned long long *key = reinterpret_cast<unsigned long long *>(dyn_smem);
+    uint32_t *idx = reinterpret_cast<uint32_t *>(dyn_smem + (size_t)SORT_TILE * 8);
+    const uint32_t base = blockIdx.x * SORT_TILE;
+    for (uint32_t i = threadIdx.x; i < SORT_TILE; i += blockDim.x) {
+        key[i] = gkey[base + i];
+        idx[i] = gidx[base + i];
+    }
+    __syncthreads();
+    for (uint32_t k = k_first; k <= k_last && k != 0; k <<= 1) {
+        uint32_t j0 = k >> 1;
+        if (j0 > SORT_TILE / 2) j0 = SORT_TILE / 2;
+        for (uint32_t j = j0; j > 0; j >>= 1) {
+            for (uint32_t t = threadIdx.x; t < SORT_TILE / 2; t += blockDim.x) {
+                uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                cmp_exchange(key, idx, i, i | j, ((base + i) & k) == 0);
+            }
+            __syncthreads();
+        }
+    }
+    for (uint32_t i = threadIdx.x; i < SORT_TILE; i += blockDim.x) {
+        gkey[base + i] = key[i];
+        gidx[base + i] = idx[i];
+    }
+}
+
+// One stage (k, j) with j >= SORT_TILE: partners sit in different tiles.
+__global__ void __launch_bounds__(256)
+bitonic_global_kernel(unsigned long long *key, uint32_t *idx, uint32_t np, uint32_t k, uint32_t j) {
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= np / 2) return;
+    const uint32_t i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+    cmp_exchange(key, idx, i, i | j, (i & k) == 0);
+}
+
 struct ScanPair {
     uint32_t a, b;
 };
@@ -115,7 +202,7 @@ __device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &ca
 }
 
 __global__ void __launch_bounds__(PLAN_THREADS, 1)
-plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem) {
+plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int presorted) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
     __shared__ ScanPair warp_tot[32];
     __shared__ ScanPair carry;
@@ -145,34 +232,18 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem) {
     }
 
     // step 1: items and their keys (device, offset at layer 0)
-    for (uint32_t q = threadIdx.x; q < np; q += blockDim.x) {
-        unsigned long long k = KEY_NONE;
-        if (q < n_raw && b.n_req > 0) {
-            uint32_t o = q >> 1, kv = q & 1;
-            uint32_t r = find_request(b.obj_start, b.n_req, o);
-            if (o >= b.obj_start[r] && o < b.obj_start[r + 1]) {
-                uint32_t c = o - b.obj_start[r];
-                uint32_t valid = valid_tokens(b.hit_tokens[r], c, g.obj_tokens);
-                if (valid) {
-                    unsigned long long slot = b.obj_slot[o];
-                    if (slot >= g.n_slots) {
-                        note_error(&s_status, TUTTI_EFAULT);
-                    } else {
-                        unsigned long long dev = slot % g.n_devices;
-                        unsigned long long off = (slot / g.n_devices) * g.stride_slot +
-                                                 (unsigned long long)kv * g.stride_kv;
-                        k = (dev << 56) | off;
-                    }
-                }
-            }
+    if (!presorted) {
+        for (uint32_t q = threadIdx.x; q < np; q += blockDim.x) {
+            key[q] = item_key(g, b, q, &s_status);
+            idx[q] = q;
         }
-        key[q] = k;
-        idx[q] = q;
+    } else if (threadIdx.x == 0 && ring.plan_counts[1].status != 0) {
+        s_status = ring.plan_counts[1].status;     // found while the keys were computed
     }
     __syncthreads();
 
     // step 2: order by (device, offset), ties by item id = (request, chunk, K before V)
-    bitonic_sort(key, idx, np);
+    if (!presorted) bitonic_sort(key, idx, np);
 
     // active items are the prefix before the first KEY_NONE
     for (uint32_t i = threadIdx.x; i < np; i += blockDim.x)
@@ -421,18 +492,43 @@ uint32_t next_pow2(uint32_t v) {
 }  // namespace
 
 cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
-                        cudaStream_t stream) {
+                        cudaStream_t stream, uint32_t *launches) {
     uint32_t np = next_pow2(2u * batch.n_obj);
-    int use_smem = np <= SMEM_SORT_ITEMS;
-    size_t smem = use_smem ? (size_t)np * 12 : 0;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(SMEM_SORT_ITEMS * 12));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(bitonic_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(SORT_TILE * 12));
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    plan_kernel<<<1, PLAN_THREADS, smem, stream>>>(ring, geom, batch, np, use_smem);
+    uint32_t n = 0;
+    if (np <= SMEM_SORT_ITEMS) {
+        plan_kernel<<<1, PLAN_THREADS, (size_t)np * 12, stream>>>(ring, geom, batch, np, 1, 0);
+        n = 1;
+    } else {
+        // keys, then the sorting network as a handful of launches, then flags and scans
+        plan_keys_kernel<<<(np + 255) / 256, 256, 0, stream>>>(ring, geom, batch, np);
+        const uint32_t tiles = np / SORT_TILE;
+        bitonic_tile_kernel<<<tiles, PLAN_THREADS, SORT_TILE * 12, stream>>>(ring.plan_key, ring.plan_idx,
+                                                                           2, SORT_TILE);
+        n = 2;
+        for (uint32_t k = 2 * SORT_TILE; k <= np; k <<= 1) {
+            for (uint32_t j = k >> 1; j >= SORT_TILE; j >>= 1) {
+                bitonic_global_kernel<<<(np / 2 + 255) / 256, 256, 0, stream>>>(ring.plan_key, ring.plan_idx,
+                                                                            np, k, j);
+                ++n;
+            }
+            bitonic_tile_kernel<<<tiles, PLAN_THREADS, SORT_TILE * 12, stream>>>(ring.plan_key,
+                                                                               ring.plan_idx, k, k);
+            ++n;
+        }
+        plan_kernel<<<1, PLAN_THREADS, 0, stream>>>(ring, geom, batch, np, 0, 1);
+        ++n;
+    }
+    if (launches) *launches = n;
     return cudaGetLastError();
 }
 

@@ -80,7 +80,7 @@ struct RingDev {
     tutti_sqe_t *plan_sqe;    // [max_items]  contexts for layer 0, opcode unset
     unsigned long long *plan_key;  // [pow2(max_items)] sort keys when they do not fit in shared memory
     uint32_t *plan_idx;       // [pow2(max_items)] sort payload, same
-    PlanCounts *plan_counts;
+    PlanCounts *plan_counts;  // [2]: [0] the plan's result, [1].status scratch of the key pass
     uint32_t max_items;
 };
 
@@ -113,7 +113,7 @@ struct CopyOptions {
 
 // kernels (tutti_build.cu / tutti_copy.cu)
 cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
-                        cudaStream_t stream);
+                        cudaStream_t stream, uint32_t *launches);
 cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
                         uint32_t layer, uint32_t opcode, const PoolLayer &pool,
                         const uint64_t *store_base, const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,

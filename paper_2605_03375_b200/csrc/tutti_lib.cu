@@ -294,7 +294,7 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
     A((void **)&d.plan_sqe, sizeof(tutti_sqe_t) * (size_t)max_items, false);
     A((void **)&d.plan_key, sizeof(unsigned long long) * (size_t)np, false);
     A((void **)&d.plan_idx, sizeof(uint32_t) * (size_t)np, false);
-    A((void **)&d.plan_counts, sizeof(PlanCounts), true);
+    A((void **)&d.plan_counts, 2 * sizeof(PlanCounts), true);
     if (rc == TUTTI_OK) {
         // headers start out "done" for an index that is never issued first
         cudaError_t e = cudaHostAlloc((void **)&r->cq_host, sizeof(CqSlot) * depth,
@@ -372,8 +372,9 @@ int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *bat
     BatchDev b{batch->n_req, batch->n_obj, batch->n_blk, batch->hit_tokens, batch->obj_start,
                batch->obj_slot, batch->blk_start, batch->block_ids};
     if (!(r->plan_valid && same_plan(r->plan_batch, *batch))) {
-        CK(launch_plan(r->dev, ctx->gdev, b, st));
-        r->kernel_launches++;
+        uint32_t plan_launches = 0;
+        CK(launch_plan(r->dev, ctx->gdev, b, st, &plan_launches));
+        r->kernel_launches += plan_launches;
         r->plan_batch = *batch;
         r->plan_valid = batch->plan_epoch != 0;
     }

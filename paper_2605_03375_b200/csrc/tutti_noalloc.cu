@@ -140,7 +140,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         // header, completion slot and counters must start at zero: the array still holds
         // whatever the previous call left there
         cudaError_t e = cudaMemsetAsync(base, 0, CLEAR_BYTES, st);
-        if (e == cudaSuccess) e = launch_plan(r, g, b, st);
+        if (e == cudaSuccess) e = launch_plan(r, g, b, st, nullptr);
         if (e == cudaSuccess)
             e = launch_emit(r, g, b, layer, TUTTI_OP_READ, pool, sbase, sbytes, 0, 1, 0,
                             NA_MAX_ENTRIES, sms, st);

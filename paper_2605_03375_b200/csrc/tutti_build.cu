@@ -78,7 +78,7 @@ __device__ void bitonic_sort(unsigned long long *key, uint32_t *idx, uint32_t n)
 // Sort key of item q = 2 * object + kv: (device << 56) | byte offset at layer 0, or KEY_NONE
 // when the object holds no hit token (or q is padding).  A slot out of range is reported.
 __device__ unsigned long long item_key(const GeomDev &g, const BatchDev &b, uint32_t q,
-                                       int32_t *status) {
+                                       int32_t &err) {
     if (q >= 2u * b.n_obj || b.n_req == 0) return KEY_NONE;
     const uint32_t o = q >> 1, kv = q & 1;
     const uint32_t r = find_request(b.obj_start, b.n_req, o);
@@ -87,7 +87,7 @@ __device__ unsigned long long item_key(const GeomDev &g, const BatchDev &b, uint
     if (valid_tokens(b.hit_tokens[r], c, g.obj_tokens) == 0) return KEY_NONE;
     const unsigned long long slot = b.obj_slot[o];
     if (slot >= g.n_slots) {
-        note_error(status, TUTTI_EFAULT);
+        err = TUTTI_EFAULT;
         return KEY_NONE;
     }
     const unsigned long long dev = slot % g.n_devices;
@@ -108,7 +108,7 @@ plan_keys_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np) {
     if (q == 0) ring.plan_counts[1].status = 0;
     if (q >= np) return;
     int32_t st = 0;
-    ring.plan_key[q] = item_key(g, b, q, &st);
+    ring.plan_key[q] = item_key(g, b, q, st);
     ring.plan_idx[q] = q;
     if (st) atomicCAS(&ring.plan_counts[1].status, 0, st);
 }
@@ -213,8 +213,6 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
                                        : ring.plan_key;
     uint32_t *idx = use_smem ? reinterpret_cast<uint32_t *>(dyn_smem + (size_t)np * 8)
                              : ring.plan_idx;
-    const uint32_t n_raw = 2u * b.n_obj;
-
     if (threadIdx.x == 0) { s_status = 0; s_nact = 0; carry.a = 0; carry.b = 0; }
     __syncthreads();
 
@@ -234,8 +232,10 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
     // step 1: items and their keys (device, offset at layer 0)
     if (!presorted) {
         for (uint32_t q = threadIdx.x; q < np; q += blockDim.x) {
-            key[q] = item_key(g, b, q, &s_status);
+            int32_t st = 0;
+            key[q] = item_key(g, b, q, st);
             idx[q] = q;
+            if (st) note_error(&s_status, st);
         }
     } else if (threadIdx.x == 0 && ring.plan_counts[1].status != 0) {
         s_status = ring.plan_counts[1].status;     // found while the keys were computed

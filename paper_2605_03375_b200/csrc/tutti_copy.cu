@@ -11,7 +11,9 @@
 //   bulk   persistent CTAs whose warps each run a ring of shared-memory stages:
 //          cp.async.bulk global->shared (mbarrier completion) then shared->global,
 //          so a handful of threads keep >100 KiB in flight per SM.  This is the
-//          engine of the SM-capped mode.
+//          engine of the SM-capped mode.  Head-major pool blocks are transposed on the
+//          way through the stage by tiled tensor copies (cp.async.bulk.tensor, one box
+//          of [block_tokens][row] per head).
 // Both claim work in chunks with one atomicAdd per claim on the IOCB's cursor and
 // account completion in bytes; the agent that lands the last byte writes the CQE.
 //
@@ -387,6 +389,25 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// Tiled tensor copies: one head of one block, [block_tokens][row] in shared memory, against the
+// store region seen as [token row][head][row].  Coordinates: word 0 of the row (always 16-byte
+// aligned), head, token row.
+__device__ __forceinline__ void tensor_g2s(uint32_t dst_smem, const CUtensorMap *map, uint32_t head,
+                                           uint32_t row, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst_smem), "l"(reinterpret_cast<unsigned long long>(map)), "r"(0), "r"(head), "r"(row),
+          "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tensor_s2g(const CUtensorMap *map, uint32_t head, uint32_t row,
+                                           uint32_t src_smem) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+        ::"l"(reinterpret_cast<unsigned long long>(map)), "r"(0), "r"(head), "r"(row), "r"(src_smem)
+        : "memory");
+}
+
 constexpr int BULK_MAX_STAGES = 8;
 
 // Geometry of the chunks of one IOCB with uniform entry length.
@@ -422,7 +443,7 @@ __device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen, u
 // the chunk's byte count and IOCB.
 template <int TO_POOL>
 __global__ void __launch_bounds__(256, 1)
-copy_bulk_kernel(CopyParams p) {
+copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_warps = blockDim.x >> 5;
@@ -458,10 +479,12 @@ copy_bulk_kernel(CopyParams p) {
     const uint64_t *obj = nullptr;
     bool f_open = false;
     uint32_t f_cur_bi = 0;
+    bool f_hnd = false;                     // head-major blocks, transposed through the stage
     uint32_t pending_claim = 0, cur = 0, cur_end = 0;
     // the next chunk, fetched ahead: one bulk load and one bulk store per lane
     bool have_next = false;
     uint32_t n_bi = 0, ld_bytes = 0, st_bytes = 0, st_off = 0;
+    bool n_hnd = false;
     unsigned long long ld_addr = 0, st_addr = 0;
 
     // ---- sink side: bytes stored for the IOCB being accounted
@@ -543,12 +566,15 @@ copy_bulk_kernel(CopyParams p) {
                 }
                 continue;
             }
-            // entries of differing lengths, and head-major blocks (a transposition the staged
-            // bulk copies cannot express), go through the per-entry vector path
-            if (h->entry_len == 0 || hnd) { copy_varlen(h, idx, total, hnd); continue; }
+            // entries of differing lengths go through the per-entry vector path; so do
+            // head-major blocks that do not fit one stage
+            const bool hnd_staged = hnd && h->entry_len <= CB && tm.valid && p.perm.n_heads <= 32;
+            if (h->entry_len == 0 || (hnd && !hnd_staged)) { copy_varlen(h, idx, total, hnd); continue; }
             f_h = h;
             f_cur_bi = bi;
+            f_hnd = hnd_staged;
             cg = chunk_geom(total, h->entry_len, CB);
+            if (f_hnd) { cg.per_chunk = 1; cg.n_chunks = total; }   // one block per stage
             cur = cur_end = 0;
             if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
             return true;
@@ -579,8 +605,24 @@ copy_bulk_kernel(CopyParams p) {
         const uint32_t c = cur++;
         have_next = true;
         n_bi = f_cur_bi;
+        n_hnd = f_hnd;
         ld_bytes = 0; st_bytes = 0; st_off = 0; ld_addr = 0; st_addr = 0;
-        if (cg.per_chunk) {
+        if (f_hnd) {
+            // one block: every lane needs both addresses (the rows are spread over the lanes)
+            unsigned long long a_obj = 0, a_pool = 0;
+            if (lane == 0) { a_obj = obj[c]; a_pool = sgl[c].addr; }
+            a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
+            a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
+            // object side as (device, token row) for the tensor map
+            uint32_t dv = 0;
+            for (uint32_t d = 1; d < tm.n_devices; ++d)
+                if (a_obj >= tm.base[d] && a_obj < tm.base[d] + tm.bytes[d]) dv = d;
+            const unsigned long long rowi = (a_obj - tm.base[dv]) / p.perm.token_bytes;
+            const unsigned long long packed = (rowi << 8) | dv;
+            ld_addr = TO_POOL ? packed : a_pool;
+            st_addr = TO_POOL ? a_pool : packed;
+            ld_bytes = st_bytes = (lane == 0) ? cg.elen : 0;
+        } else if (cg.per_chunk) {
             const uint32_t e0 = c * cg.per_chunk;
             const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
             unsigned long long a_obj = 0, a_pool = 0;
@@ -627,11 +669,22 @@ copy_bulk_kernel(CopyParams p) {
             const uint32_t total_bytes = __reduce_add_sync(0xffffffffu, ld_bytes);
             if (lane == 0) mbar_expect_tx(bar, total_bytes);
             __syncwarp();
-            if (ld_bytes) bulk_g2s(sbase + st_off, ld_addr, ld_bytes, bar);
+            if (n_hnd && TO_POOL) {
+                // token-major object -> head-major stage: one tiled tensor copy per head
+                // (box = [block_tokens][row]), heads dealt out over the lanes
+                if (lane < p.perm.n_heads)
+                    tensor_g2s(sbase + lane * p.perm.block_tokens * p.perm.row_bytes,
+                               &tm.map[ld_addr & 0xff], lane, (uint32_t)(ld_addr >> 8), bar);
+            } else if (ld_bytes) {
+                bulk_g2s(sbase + st_off, ld_addr, ld_bytes, bar);
+            }
             st_addr_of[s * 32 + lane] = st_addr;
             st_bytes_of[s * 32 + lane] = st_bytes;
             st_off_of[s * 32 + lane] = st_off;
-            if (lane == 0) { chunk_bytes_of[s] = total_bytes; chunk_iocb_of[s] = n_bi; }
+            if (lane == 0) {
+                chunk_bytes_of[s] = total_bytes;
+                chunk_iocb_of[s] = n_bi | (n_hnd ? 0x80000000u : 0u);
+            }
             __syncwarp();
             ++head;
             fetch_next();
@@ -642,7 +695,9 @@ copy_bulk_kernel(CopyParams p) {
         const uint32_t s = tail % S;
         const uint32_t bar = smem_u32(&bars[s]);
         const uint32_t sbase = smem_u32(data + (size_t)s * CB);
-        const uint32_t s_bi = chunk_iocb_of[s];
+        const uint32_t s_tag = chunk_iocb_of[s];
+        const uint32_t s_bi = s_tag & 0x7fffffffu;
+        const bool s_hnd = (s_tag >> 31) != 0;
         if (s_bi != acct_bi) {
             // first chunk of a later IOCB: close the books of the previous one.  Only the
             // stores are waited for; the loads already in flight keep streaming.
@@ -659,7 +714,14 @@ copy_bulk_kernel(CopyParams p) {
         const unsigned long long dst = st_addr_of[s * 32 + lane];
         const uint32_t nbytes = st_bytes_of[s * 32 + lane];
         const uint32_t off = st_off_of[s * 32 + lane];
-        if (arrived && nbytes) bulk_s2g(dst, sbase + off, nbytes);
+        if (s_hnd && !TO_POOL) {
+            // head-major stage -> token-major object, one tiled tensor copy per head
+            if (arrived && lane < p.perm.n_heads)
+                tensor_s2g(&tm.map[dst & 0xff], lane, (uint32_t)(dst >> 8),
+                           sbase + lane * p.perm.block_tokens * p.perm.row_bytes);
+        } else if (arrived && nbytes) {
+            bulk_s2g(dst, sbase + off, nbytes);
+        }
         bulk_commit();
         moved += chunk_bytes_of[s];
         ++tail;
@@ -681,8 +743,10 @@ cudaError_t copy_kernels_setup() {
 
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
-                        bool pool_hnd, const PermGeom &perm, cudaStream_t stream,
-                        uint32_t *launches) {
+                        bool pool_hnd, const PermGeom &perm, const StoreTensorMaps *maps,
+                        cudaStream_t stream, uint32_t *launches) {
+    static const StoreTensorMaps no_maps = {};
+    const StoreTensorMaps &tm = maps ? *maps : no_maps;
     CopyParams p;
     p.ring = ring;
     p.first_iocb = first_iocb;
@@ -691,7 +755,8 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     p.wait_ns = opt.wait_ns;
     p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : 4;
     uint32_t engine = opt.engine;
-    if (engine == 0) engine = (host_store || pool_hnd) ? 1 : 2;   // measured: bulk-async wins on HBM
+    // measured: bulk-async wins on HBM, also for head-major blocks when tensor maps exist
+    if (engine == 0) engine = (host_store || (pool_hnd && !(maps && maps->valid))) ? 1 : 2;
     p.perm = perm;
     const uint32_t sms = sm_count ? sm_count : (uint32_t)device_sms;
     if (engine == 2) {
@@ -713,9 +778,9 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
         // a capped launch keeps one CTA per SM: pad shared memory so no second CTA fits
         if (sm_count && smem < 120u * 1024u) smem = 120u * 1024u;
         if (opcode == TUTTI_OP_READ)
-            copy_bulk_kernel<1><<<sms, warps * 32, smem, stream>>>(p);
+            copy_bulk_kernel<1><<<sms, warps * 32, smem, stream>>>(p, tm);
         else
-            copy_bulk_kernel<0><<<sms, warps * 32, smem, stream>>>(p);
+            copy_bulk_kernel<0><<<sms, warps * 32, smem, stream>>>(p, tm);
     } else {
         p.stages = 0;
         p.chunk_bytes = CHUNK_BYTES;

@@ -1,5 +1,6 @@
 // Internal definitions shared by the host side of the library and its kernels.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -61,6 +62,7 @@ struct StoreDev {
     uint64_t base, bytes;
     uint32_t kind;
     bool registered;
+    bool tmap_ok;      // a tensor map of the region exists
 };
 
 // Device-side view of a ring, passed by value to kernels.
@@ -102,6 +104,16 @@ struct PermGeom {
     uint32_t block_tokens, n_heads, row_bytes, token_bytes;
 };
 
+// Tensor maps of the storage devices for head-major pool blocks: every device region seen as
+// a 3-D array [token row][head][row of head_dim elements], box = one head of one block.
+struct alignas(64) StoreTensorMaps {
+    CUtensorMap map[TUTTI_MAX_DEVICES];
+    uint64_t base[TUTTI_MAX_DEVICES];
+    uint64_t bytes[TUTTI_MAX_DEVICES];
+    uint32_t n_devices;
+    uint32_t valid;         // 1 when the maps may be used
+};
+
 struct CopyOptions {
     uint32_t engine;        // 0 auto, 1 ld/st, 2 bulk
     uint64_t wait_ns;
@@ -121,8 +133,8 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
                         cudaStream_t stream);
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
-                        bool pool_hnd, const PermGeom &perm, cudaStream_t stream,
-                        uint32_t *launches);
+                        bool pool_hnd, const PermGeom &perm, const StoreTensorMaps *maps,
+                        cudaStream_t stream, uint32_t *launches);
 cudaError_t copy_kernels_setup();
 
 }  // namespace tutti

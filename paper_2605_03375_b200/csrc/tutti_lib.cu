@@ -63,6 +63,7 @@ struct tutti_ctx {
     GeomDev gdev;
     void *partition = nullptr;   // SM partition state (tutti_partition.cu)
     bool pool_hnd = false;       // pool blocks are [head][token][dim]
+    StoreTensorMaps maps;        // for the transposing bulk copies
 };
 
 struct tutti_ring {
@@ -163,7 +164,8 @@ int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
     c->device = device;
     c->device_sms = prop.multiProcessorCount;
     c->pool.assign(geom->n_layers, PoolLayer{0, 0, 0, 0, false});
-    for (auto &s : c->store) s = StoreDev{0, 0, 0, false};
+    for (auto &s : c->store) s = StoreDev{0, 0, 0, false, false};
+    memset(&c->maps, 0, sizeof(c->maps));
     c->opt = CopyOptions{0, 2000000ull, 4, 0, 0, 4, 0};   // 0 = chosen per launch
     c->gdev.block_tokens = geom->block_tokens;
     c->gdev.obj_tokens = geom->obj_tokens;
@@ -202,6 +204,43 @@ int tutti_store_register(tutti_ctx_t *ctx, uint32_t dev, void *base, uint64_t by
     if (((uint64_t)base & 15) || bytes < ctx->layout.dev_bytes) return TUTTI_EINVAL;
     if (kind != TUTTI_STORE_HBM && kind != TUTTI_STORE_HOST_PINNED) return TUTTI_EINVAL;
     ctx->store[dev] = StoreDev{(uint64_t)base, bytes, kind, true};
+    // Tensor map of the region as [token row][head][row bytes / 4] 32-bit words, box = one
+    // head of one block.  Only used for head-major pool blocks; if the driver refuses it
+    // (or the shape is out of a tensor map's range) those fall back to vector copies.
+    ctx->maps.base[dev] = (uint64_t)base;
+    ctx->maps.bytes[dev] = bytes;
+    ctx->maps.n_devices = ctx->geom.n_devices;
+    const uint64_t row_bytes = (uint64_t)ctx->geom.head_dim * ctx->geom.elem_bytes;
+    const uint64_t n_rows = ctx->layout.dev_bytes / ctx->layout.token_bytes;
+    bool ok = kind == TUTTI_STORE_HBM && (row_bytes % 16) == 0 && row_bytes / 4 <= 256 &&
+              ctx->geom.block_tokens <= 256 && n_rows < (1ull << 32) &&
+              ctx->layout.token_bytes % 16 == 0 &&
+              (ctx->geom.block_tokens * row_bytes) % 128 == 0;   // a head's slab in the stage
+    if (ok) {
+        typedef CUresult (*encode_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                      const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                      const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        void *fp = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fp, cudaEnableDefault, &q) == cudaSuccess &&
+             fp && q == cudaDriverEntryPointSuccess;
+        if (ok) {
+            cuuint64_t dims[3] = {row_bytes / 4, ctx->geom.n_kv_heads, n_rows};
+            cuuint64_t strides[2] = {row_bytes, ctx->layout.token_bytes};      // bytes, dims 1 and 2
+            cuuint32_t box[3] = {(cuuint32_t)(row_bytes / 4), 1, ctx->geom.block_tokens};
+            cuuint32_t estr[3] = {1, 1, 1};
+            CUresult r = ((encode_fn)fp)(&ctx->maps.map[dev], CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, base, dims,
+                                         strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                         CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = r == CUDA_SUCCESS;
+        }
+    }
+    bool all = ok;
+    ctx->store[dev].tmap_ok = ok;
+    for (uint32_t d = 0; d < ctx->geom.n_devices; ++d) all = all && ctx->store[d].registered && ctx->store[d].tmap_ok;
+    ctx->maps.valid = all ? 1u : 0u;
     return TUTTI_OK;
 }
 
@@ -411,7 +450,7 @@ static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, 
     PermGeom pg{ctx->geom.block_tokens, ctx->geom.n_kv_heads,
                 ctx->geom.head_dim * ctx->geom.elem_bytes, (uint32_t)ctx->layout.token_bytes};
     CK(launch_copy(r->dev, first, n, opcode, sm_count, ctx->device_sms, ctx->opt, host_store,
-                   ctx->pool_hnd, pg, (cudaStream_t)stream, &launches));
+                   ctx->pool_hnd, pg, &ctx->maps, (cudaStream_t)stream, &launches));
     r->kernel_launches += launches;
     return TUTTI_OK;
 }

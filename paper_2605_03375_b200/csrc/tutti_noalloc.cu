@@ -148,7 +148,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
             e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, false,
                             PermGeom{geom->block_tokens, geom->n_kv_heads,
                                      geom->head_dim * geom->elem_bytes, (uint32_t)lo.token_bytes},
-                            st, &launches);
+                            nullptr, st, &launches);
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(cqe_out, base + OFF_CQ, sizeof(tutti_cqe_t), cudaMemcpyDefault, st);
         if (e != cudaSuccess) rc = TUTTI_ECUDA;

@@ -1,0 +1,111 @@
+"""Seeded random geometries and batches: every case checks descriptors, restore and save
+against the oracle, with a random engine, SM cap and IOCB capacity.  Also two rings driven
+concurrently on two streams."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_03375_b200 import tutti as T
+from paper_2605_03375_b200 import workload as wl
+from tests.devcase import DeviceCase
+
+pytestmark = pytest.mark.gpu
+
+
+def random_workload(seed):
+    rng = np.random.default_rng(1000 + seed)
+    heads = int(rng.choice([1, 2, 3, 4, 8]))
+    dim = int(rng.choice([8, 16, 32, 64, 128]))
+    elem = int(rng.choice([1, 2, 4]))
+    while (heads * dim * elem) % 16:
+        dim *= 2
+    bt = int(rng.choice([1, 2, 4, 8, 16, 32]))
+    obj_blocks = int(rng.choice([1, 2, 4, 16]))
+    n_req = int(rng.integers(1, 7))
+    hits = [int(rng.integers(0, 40)) * bt for _ in range(n_req)]
+    if sum(hits) == 0:
+        hits[0] = 3 * bt
+    hnd = bool(rng.random() < 0.35)
+    return wl.make_workload(
+        f"fuzz{seed}", seed=5000 + seed, n_layers=int(rng.integers(1, 4)), hit_tokens=hits,
+        block_tokens=bt, obj_tokens=bt * obj_blocks, n_kv_heads=heads, head_dim=dim,
+        elem_bytes=elem, n_devices=int(rng.choice([1, 1, 2, 3])),
+        layout=int(rng.choice([wl.LAYOUT_FILE_MAJOR, wl.LAYOUT_LAYER_MAJOR])),
+        slot_mean_run=float(rng.choice([1.0, 2.0, 6.0])), slot_space_factor=float(rng.choice([1.1, 2.0])),
+        pool_round=64, pool_interleaved=bool(rng.random() < 0.4), pool_hnd=hnd), rng
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_random_case(seed):
+    w, rng = random_workload(seed)
+    capacity = int(rng.choice([1, 3, 64, 2048]))
+    n_items = 2 * len(w.obj_slot)
+    depth = 1
+    while depth < 2 * max(1, -(-n_items // capacity)):
+        depth *= 2
+    dc = DeviceCase(w, depth=depth, capacity=capacity)
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, int(rng.choice([0, 1, 2])))
+        sm_count = int(rng.choice([0, 0, 3, 16]))
+        layer = int(rng.integers(0, w.n_layers))
+        flag = oracle.OP_HND if w.pool_hnd else 0
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+        sq, sg, num, infos = dc.read_build(first, n)
+        orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, capacity)
+        assert orc == 0 and all(i.status == 0 for i in infos)
+        assert sq.tobytes() == osq.tobytes() and sg.tobytes() == osg.tobytes()
+        assert np.all(osq["opcode"] == flag)
+        assert list(num[:len(onum)]) == list(onum) and not num[len(onum):].any()
+        dc.ring.tutti_kv_restore_layer(first, n, sm_count)
+        cqes = dc.poll_all(first, n)
+        assert all(c[1] == 0 for c in cqes)
+        assert sum(c[2] for c in cqes) == int(osq["len"].sum())
+        want = dc.oracle_restore(layer)
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
+        for t in dc.store_dev:
+            t.zero_()
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_WRITE)
+        dc.ring.tutti_kv_save_layer(first, n, sm_count)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        st_want = [np.zeros_like(s) for s in dc.store_host]
+        dc.oracle_save(layer, want, st_want)
+        for t, s in zip(dc.store_dev, st_want):
+            assert np.array_equal(t.cpu().numpy(), s)
+    finally:
+        dc.close()
+
+
+def test_two_rings_on_two_streams():
+    """Two rings of one context, each on its own stream, restoring different layers at the
+    same time: neither disturbs the other."""
+    w = wl.config(2, 0.06, n_layers=4)
+    dc = DeviceCase(w)
+    ring2 = T.Ring(dc.ctx, 8, 2048, 4 * len(w.block_ids), 2 * len(w.obj_slot))
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    try:
+        for rep in range(3):
+            for l in range(w.n_layers):
+                dc.pool_dev[l].copy_(torch.from_numpy(dc.pool_host[l]))
+            torch.cuda.synchronize()
+            issued = []
+            for l in range(0, w.n_layers, 2):
+                a = dc.ring.tutti_build_sqes(dc.batch, l, T.OP_READ, stream=s1)
+                b = ring2.tutti_build_sqes(dc.batch, l + 1, T.OP_READ, stream=s2)
+                dc.ring.tutti_kv_restore_layer(a[1], a[2], stream=s1)
+                ring2.tutti_kv_restore_layer(b[1], b[2], 8, stream=s2)
+                issued.append((a, b))
+            for a, b in issued:
+                for i in range(a[1], a[1] + a[2]):
+                    rc, cqe = dc.ring.tutti_ring_poll(i, 5_000_000_000)
+                    assert rc == T.OK and cqe.status == 0
+                for i in range(b[1], b[1] + b[2]):
+                    rc, cqe = ring2.tutti_ring_poll(i, 5_000_000_000)
+                    assert rc == T.OK and cqe.status == 0
+            torch.cuda.synchronize()
+            for l in range(w.n_layers):
+                assert np.array_equal(dc.pool_dev[l].cpu().numpy(), dc.oracle_restore(l))
+    finally:
+        torch.cuda.synchronize()
+        ring2.close()
+        dc.close()

@@ -387,24 +387,26 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
         ring.sqes[(size_t)slot * ring.capacity + k % ring.capacity] = e;
     }
 
-    // SGL entries: one warp per item, lanes over the item's blocks
+    // SGL entries: a group of G lanes per item, lanes over the item's blocks.  G is the
+    // power of two that covers an object's blocks (32 for big objects, 1 when every object
+    // is a single block), so small objects do not leave most of a warp idle.
     const uint32_t lane = threadIdx.x & 31;
+    uint32_t G = 1;
+    while (G < 32 && G < g.blocks_per_obj) G <<= 1;
+    const uint32_t per_warp = 32 / G;                   // items handled side by side
+    const uint32_t sub = lane / G, sl = lane % G, leader = sub * G;
     const uint32_t gwarp = gtid >> 5, nwarps = gthreads >> 5;
-    for (uint32_t i = gwarp; i < n_items; i += nwarps) {
-        uint32_t q = 0, e_first = 0, e_next = 0, sq = 0;
-        if (lane == 0) {
+    for (uint32_t i0 = gwarp * per_warp; i0 < n_items; i0 += nwarps * per_warp) {
+        const uint32_t i = i0 + sub;
+        const bool live = i < n_items;
+        uint32_t q = 0, e_first = 0, e_next = 0;
+        unsigned long long meta0 = 0, meta1 = 0;   // (row start in block table, object-side address)
+        if (live && sl == 0) {
             q = ring.plan_item[i];
             e_first = ring.plan_cumblk[i];
             e_next = ring.plan_cumblk[i + 1];
-            sq = ring.plan_sqe_of[i];
-        }
-        q = __shfl_sync(0xffffffffu, q, 0);
-        e_first = __shfl_sync(0xffffffffu, e_first, 0);
-        e_next = __shfl_sync(0xffffffffu, e_next, 0);
-        sq = __shfl_sync(0xffffffffu, sq, 0);
-        const uint32_t o = q >> 1, kv = q & 1;
-        unsigned long long meta0 = 0, meta1 = 0;   // (row start in block table, object-side address)
-        if (lane == 0) {
+            const uint32_t sq = ring.plan_sqe_of[i];
+            const uint32_t o = q >> 1;
             uint32_t r = find_request(b.obj_start, b.n_req, o);
             uint32_t c = o - b.obj_start[r];
             meta0 = (unsigned long long)b.blk_start[r] + (unsigned long long)c * g.blocks_per_obj;
@@ -417,15 +419,21 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
             if (end > p.store_bytes[run.dev]) {
                 note_error(&hdr0->emit_status, TUTTI_EFAULT);
                 meta1 = 0;
+                e_next = e_first;                      // nothing is emitted for this item
             } else {
                 meta1 = p.store_base[run.dev] + off;
             }
         }
-        const unsigned long long row0 = __shfl_sync(0xffffffffu, meta0, 0);
-        const unsigned long long obj0 = __shfl_sync(0xffffffffu, meta1, 0);
-        const unsigned long long pool_base = kv ? p.v_base : p.k_base;
+        // the group leader read the item; its lanes get it by shuffle
+        q = __shfl_sync(0xffffffffu, q, leader);
+        e_first = __shfl_sync(0xffffffffu, e_first, leader);
+        e_next = __shfl_sync(0xffffffffu, e_next, leader);
+        const unsigned long long row0 = __shfl_sync(0xffffffffu, meta0, leader);
+        const unsigned long long obj0 = __shfl_sync(0xffffffffu, meta1, leader);
+        if (!live) continue;
+        const unsigned long long pool_base = (q & 1) ? p.v_base : p.k_base;
         const uint32_t n_blk = e_next - e_first;
-        for (uint32_t j = lane; j < n_blk; j += 32) {
+        for (uint32_t j = sl; j < n_blk; j += G) {
             unsigned long long bi = row0 + j;
             tutti_sgl_t ent;
             ent.len = (uint32_t)g.block_bytes;
@@ -554,7 +562,10 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
     p.sgl_reserved = sgl_reserved;
     // one warp per item, 8 warps per CTA; a few CTAs per SM at most
     uint32_t items = 2u * batch.n_obj;
-    uint32_t ctas = (items + 7) / 8;
+    uint32_t G = 1;
+    while (G < 32 && G < geom.blocks_per_obj) G <<= 1;
+    const uint32_t per_cta = 8 * (32 / G);             // 8 warps, 32/G items side by side
+    uint32_t ctas = (items + per_cta - 1) / per_cta;
     uint32_t cap = (uint32_t)device_sms * 2u;
     if (ctas > cap) ctas = cap;
     if (ctas == 0) ctas = 1;

@@ -64,7 +64,8 @@ extern "C" {
 #define TUTTI_OPT_BULK_STAGES 5 /* shared-memory stages per copy warp of the bulk-async kernel   */
 #define TUTTI_OPT_CLAIM_CHUNKS 6 /* chunks taken per work claim                                   */
 #define TUTTI_OPT_POOL_LAYOUT 8  /* TUTTI_POOL_NHD (default) or TUTTI_POOL_HND: element order inside a
-                                   pool block; applies to builds made after it is set        */
+                                   pool block; applies to builds made after it is set.  HND needs
+                                   head_dim * elem_bytes to be a multiple of 16 (TUTTI_EINVAL)  */
 #define TUTTI_POOL_NHD 0
 #define TUTTI_POOL_HND 1
 #define TUTTI_OPT_BULK_CHUNK_BYTES 7 /* bytes per shared-memory stage of the bulk-async kernel: a

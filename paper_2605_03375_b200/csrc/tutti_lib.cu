@@ -273,6 +273,9 @@ int tutti_set_option(tutti_ctx_t *ctx, uint32_t option, uint64_t value) {
             return TUTTI_OK;
         case TUTTI_OPT_POOL_LAYOUT:
             if (value > TUTTI_POOL_HND) return TUTTI_EINVAL;
+            // the transposing copies move 16-byte vectors that must stay inside one head's row
+            if (value == TUTTI_POOL_HND && ((uint64_t)ctx->geom.head_dim * ctx->geom.elem_bytes) % 16)
+                return TUTTI_EINVAL;
             ctx->pool_hnd = value == TUTTI_POOL_HND;
             return TUTTI_OK;
         case TUTTI_OPT_BULK_CHUNK_BYTES:
@@ -540,6 +543,8 @@ int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
         if (s.dev >= ctx->geom.n_devices || !ctx->store[s.dev].registered) return TUTTI_EINVAL;
         if (s.opcode != opcode || (uint64_t)s.sgl_first + s.sgl_count > n_sgl) return TUTTI_EINVAL;
         if ((s.opcode & 0xff) > TUTTI_OP_WRITE || (s.opcode & ~(0xffu | TUTTI_OP_FLAG_HND)))
+            return TUTTI_EINVAL;
+        if ((s.opcode & TUTTI_OP_FLAG_HND) && ((uint64_t)ctx->geom.head_dim * ctx->geom.elem_bytes) % 16)
             return TUTTI_EINVAL;
         uint64_t cursor = s.src_off;
         for (uint32_t e = s.sgl_first; e < s.sgl_first + s.sgl_count; ++e) {

@@ -35,6 +35,7 @@ def test_bad_arguments():
         assert lib.tutti_pool_register(dc.ctx.h, 0, 8, 16, 32768, 4) == T.EINVAL     # misaligned
         assert lib.tutti_store_register(dc.ctx.h, 0, 4096, 16, 0) == T.EINVAL        # too small
         assert lib.tutti_set_option(dc.ctx.h, 99, 1) == T.EINVAL
+        assert lib.tutti_set_option(dc.ctx.h, T.OPT_POOL_LAYOUT, 2) == T.EINVAL
     finally:
         dc.close()
 
@@ -113,5 +114,21 @@ def test_unpublished_iocb_times_out(engine):
         rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
         dc.ring.tutti_kv_restore_layer(first, n)
         assert all(c[1] == 0 for c in dc.poll_all(first, n))
+    finally:
+        dc.close()
+
+
+def test_head_major_needs_16_byte_rows():
+    """Rows of 8 bytes cannot be transposed in 16-byte vectors: the option is refused instead
+    of producing misaligned accesses."""
+    w = wl.make_workload("rows8", seed=3, n_layers=1, hit_tokens=[8], block_tokens=4, obj_tokens=8,
+                         n_kv_heads=8, head_dim=8, elem_bytes=1, n_pool_blocks=16)
+    dc = DeviceCase(w)
+    try:
+        assert dc.ctx.lib.tutti_set_option(dc.ctx.h, T.OPT_POOL_LAYOUT, T.POOL_HND) == T.EINVAL
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)      # still token-major
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
     finally:
         dc.close()

@@ -109,3 +109,70 @@ def test_two_rings_on_two_streams():
         torch.cuda.synchronize()
         ring2.close()
         dc.close()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_op_sequences_on_a_small_ring(seed):
+    """Random interleavings of build / restore / save / poll on a ring that is too small to
+    hold everything: TUTTI_EAGAIN is answered by polling the oldest work, and at the end the
+    pools and the store hold exactly what the oracle gets by applying the same operations in
+    issue order."""
+    rng = np.random.default_rng(77 + seed)
+    w = wl.config(2, 0.03, n_layers=3, n_devices=int(rng.choice([1, 2])),
+                  pool_interleaved=bool(seed & 1), slot_mean_run=2.0)
+    n_blk, n_obj = len(w.block_ids), len(w.obj_slot)
+    capacity = int(rng.choice([4, 16, 2048]))
+    per_build = max(1, -(-2 * n_obj // capacity))
+    depth = 1
+    while depth < 2 * per_build:
+        depth *= 2
+    dc = DeviceCase(w, depth=depth, capacity=capacity, sgl_capacity=int(2 * n_blk * 2.5))
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, int(rng.choice([1, 2])))
+        pools = {l: dc.pool_host[l].copy() for l in range(w.n_layers)}
+        store = [s.copy() for s in dc.store_host]
+        outstanding = []                     # (first, n) in issue order
+        n_again = 0
+
+        def poll_oldest():
+            first, n = outstanding.pop(0)
+            assert all(c[1] == 0 for c in dc.poll_all(first, n))
+
+        for step in range(40):
+            layer = int(rng.integers(0, w.n_layers))
+            op = T.OP_READ if rng.random() < 0.6 else T.OP_WRITE
+            if step % 7 == 3:                # scribble over a pool so that saves move new data
+                noise = torch.randint(0, 255, (dc.pool_dev[layer].numel(),), dtype=torch.uint8,
+                                      device=dc.dev)
+                torch.cuda.synchronize()
+                dc.pool_dev[layer].copy_(noise)
+                pools[layer] = noise.cpu().numpy()
+            while True:
+                rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, op, allow=(T.EAGAIN,))
+                if rc == T.OK:
+                    break
+                n_again += 1
+                assert outstanding, "ring full with nothing outstanding"
+                poll_oldest()
+            sm = int(rng.choice([0, 0, 4]))
+            if op == T.OP_READ:
+                dc.ring.tutti_kv_restore_layer(first, n, sm)
+                assert oracle.restore_layer(dc.og, layer, dc.obatch, store, pools[layer], dc.k_off,
+                                            dc.v_off, dc.stride, w.n_pool_blocks) == 0
+            else:
+                dc.ring.tutti_kv_save_layer(first, n, sm)
+                assert oracle.save_layer(dc.og, layer, dc.obatch, store, pools[layer], dc.k_off,
+                                         dc.v_off, dc.stride, w.n_pool_blocks) == 0
+            outstanding.append((first, n))
+            if rng.random() < 0.3 and outstanding:
+                poll_oldest()
+        while outstanding:
+            poll_oldest()
+        torch.cuda.synchronize()
+        for l in range(w.n_layers):
+            assert np.array_equal(dc.pool_dev[l].cpu().numpy(), pools[l])
+        for t, s in zip(dc.store_dev, store):
+            assert np.array_equal(t.cpu().numpy(), s)
+        assert n_again > 0 or depth >= 80 * per_build
+    finally:
+        dc.close()

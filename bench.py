@@ -239,6 +239,7 @@ class Replica:
         self.stream = torch.cuda.Stream(self.dev)
         self.build_stream = torch.cuda.Stream(self.dev)
         self.two_streams = not getattr(args, "one_stream", False)
+        self.layers_per_launch = getattr(args, "layers_per_launch", 4) or 1
         self.epoch = 1
         if args.engine:
             self.ctx.tutti_set_option(T.OPT_COPY_ENGINE, args.engine)
@@ -274,9 +275,18 @@ class Replica:
                     ev = torch.cuda.Event(enable_timing=True)
                     ev.record(s)
                     events["pass"].append(ev)
-                for l in range(self.w.n_layers):
-                    # descriptors are built on their own stream, ahead of the copies
-                    rc, first, n = self.ring.tutti_build_sqes(self.batch, l, op, stream=sb)
+                G = max(1, self.layers_per_launch)
+                for l0 in range(0, self.w.n_layers, G):
+                    # descriptors are built on their own stream, ahead of the copies; one
+                    # copy launch then executes the IOCBs of G consecutive layers (each
+                    # layer keeps its own IOCBs and completion entries)
+                    first, n = None, 0
+                    for l in range(l0, min(l0 + G, self.w.n_layers)):
+                        rc, f, k = self.ring.tutti_build_sqes(self.batch, l, op, stream=sb)
+                        if first is None:
+                            first = f
+                        assert f == first + n, "IOCB indices of consecutive builds are contiguous"
+                        n += k
                     if self.two_streams:
                         built = torch.cuda.Event()
                         built.record(sb)
@@ -291,7 +301,7 @@ class Replica:
                         self.ring.tutti_kv_save_layer(first, n, sm_count, stream=s)
                     if events is not None:
                         b.record(s)
-                        events["copy"][op].append((a, b))
+                        events["copy"][op].append((a, b, min(G, self.w.n_layers - l0)))
                     issued.append((first, n))
             if events is not None:
                 ev = torch.cuda.Event(enable_timing=True)
@@ -412,7 +422,7 @@ def run_ours(args):
     # per-direction figures from the events inside the timed region
     def dir_stats(op):
         pairs = events["copy"][op]
-        ms = [a.elapsed_time(b) for a, b in pairs]
+        ms = [a.elapsed_time(b) / g for a, b, g in pairs]     # per layer of the launch
         passes = events["pass"]
         idx = 0 if op == T.OP_READ else 1
         pass_ms = [passes[3 * s + idx].elapsed_time(passes[3 * s + idx + 1])
@@ -449,6 +459,7 @@ def run_ours(args):
                        "copy_engine": args.engine or "auto",
                        "streams": "copy + descriptor-build stream, event-ordered"
                        if rep.two_streams else "one stream",
+                       "layers_per_launch": rep.layers_per_launch,
                        "ioctx_per_iocb": args.ioctx_per_iocb},
             "restore": restore, "save": save,
             "blocks_per_s": restore["blocks_per_s"],
@@ -913,6 +924,8 @@ def main():
     ap.add_argument("--sched-sms", type=int, default=16)
     ap.add_argument("--sched-ioctx", type=int, default=16)
     ap.add_argument("--sched-gemms", type=int, default=3)
+    ap.add_argument("--layers-per-launch", type=int, default=4,
+                    help="consecutive layers whose IOCBs one copy launch executes")
     ap.add_argument("--one-stream", action="store_true",
                     help="build and copy on one stream (default: descriptors on their own stream)")
     ap.add_argument("--pool-hnd", action="store_true",

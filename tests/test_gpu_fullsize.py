@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 
 def _args(**kw):
     d = dict(config=2, scale=1.0, layers=0, engine=0, resident_layers=3, ioctx_per_iocb=2048,
-             ctas_per_sm=0, bulk_warps=0, bulk_stages=0, claim=0)
+             ctas_per_sm=0, bulk_warps=0, bulk_stages=0, claim=0, layers_per_launch=4)
     d.update(kw)
     return argparse.Namespace(**d)
 

@@ -493,6 +493,9 @@ def run_ours(args):
     if rank == 0:
         print(json.dumps(out), flush=True)
     barrier(world)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
 
 
 def run_e2e(args, local_rank, world):

@@ -12,6 +12,13 @@
 
 using namespace tutti;
 
+// the wire formats the header promises
+static_assert(sizeof(tutti_sqe_t) == 32, "I/O context is 32 bytes");
+static_assert(sizeof(tutti_sgl_t) == 16, "SGL entry is 16 bytes (address 8, length 4, id 4)");
+static_assert(sizeof(tutti_cqe_t) == 16, "completion entry is 16 bytes");
+static_assert(sizeof(tutti_geom_t) == 40 && sizeof(tutti_layout_t) == 80 && sizeof(tutti_batch_t) == 56,
+              "geometry / layout / batch structs have no hidden padding");
+
 namespace {
 
 thread_local std::string g_last_cuda_error;

@@ -157,3 +157,12 @@ def test_context_needs_a_gpu():
     assert lib.tutti_last_cuda_error().decode() != ""
     with pytest.raises(T.TuttiError):
         T.Context(g)
+
+
+def test_struct_sizes_match_the_header():
+    """The binding's ctypes structs and numpy record types have the sizes the library
+    asserts at compile time."""
+    assert C.sizeof(T.Geom) == 40 and C.sizeof(T.Layout) == 80 and C.sizeof(T.Batch) == 56
+    assert C.sizeof(T.Cqe) == 16 and C.sizeof(T.IocbInfo) == 48 and C.sizeof(T.Launch) == 24
+    assert T.SQE_DTYPE.itemsize == 32 and T.SGL_DTYPE.itemsize == 16
+    assert oracle.SQE_DTYPE.itemsize == 32 and oracle.SGL_DTYPE.itemsize == 16

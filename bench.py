@@ -160,7 +160,8 @@ def ncu_traffic(kernel: str):
 class Replica:
     """Config-2-shaped workload resident on one GPU, registered with the library."""
 
-    def __init__(self, args, device_index: int, host_store: bool = False, n_layers=None):
+    def __init__(self, args, device_index: int, host_store: bool = False, n_layers=None,
+                 hit_tokens=None):
         import torch
         from paper_2605_03375_b200 import tutti as T
         from paper_2605_03375_b200 import workload as wl
@@ -177,6 +178,8 @@ class Replica:
             n_layers = args.layers
         if n_layers is not None:
             over["n_layers"] = n_layers
+        if hit_tokens is not None:
+            over["hit_tokens"] = hit_tokens
         self.w = w = wl.config(args.config, args.scale, **over)
         self.geom = T.geom_of(w)
         self.ctx = T.Context(self.geom, device_index)
@@ -855,6 +858,50 @@ def run_sched_demo(args):
         print(json.dumps(out), flush=True)
 
 
+def run_length_sweep(args):
+    """Raw restore / save bandwidth against prefix length, model bypassed (the measurement of
+    the paper's Section 4.2.1, here against the HBM or pinned-host object store): one request,
+    Llama-3-8B-shaped KV, all layers, descriptor build included."""
+    import torch
+    from paper_2605_03375_b200 import tutti as T
+    from paper_2605_03375_b200 import workload as wl
+    rank, local_rank, world = init_dist("nccl")
+    rows = []
+    for tokens in (1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072):
+        a2 = argparse.Namespace(**vars(args))
+        a2.config = 2
+        a2.resident_layers = 4
+        a2.set = (args.set or []) + []
+        rep = Replica(a2, local_rank, host_store=args.sweep_host, n_layers=args.layers or 32,
+                      hit_tokens=[tokens])
+        res = {"prefix_tokens": tokens,
+               "payload_mib_per_layer": round(rep.payload_per_layer / (1 << 20), 1)}
+        for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
+            for _ in range(2):
+                rep.step(directions=dirs)
+            torch.cuda.synchronize()
+            reps = 5 if tokens <= 16384 else 2
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(rep.stream)
+            for _ in range(reps):
+                rep.step(directions=dirs)
+            e1.record(rep.stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            res[name + "_gbs"] = round(rep.w.n_layers * rep.payload_per_layer / (ms * 1e-3) / 1e9, 1)
+            res[name + "_us_per_layer"] = round(ms * 1e3 / rep.w.n_layers, 1)
+        res["verified"] = bool(rep.verify_samples(32))
+        rows.append(res)
+        rep.close()
+        del rep
+        torch.cuda.empty_cache()
+    if rank == 0:
+        print(json.dumps({"sweep": "raw restore/save bandwidth vs prefix length, 1 request, "
+                          "8 KV heads x 128 x bf16, block 16, 32 layers",
+                          "store": "pinned host, zero-copy" if args.sweep_host else "hbm",
+                          "rows": rows}), flush=True)
+
+
 def run_reference(args):
     """The reference arm of this tier is the oracle on the host cores: each step is a
     bounded sample of the same workload (restore + save of one layer of the batch)."""
@@ -921,6 +968,9 @@ def main():
     ap.add_argument("--bulk-chunk", type=int, default=0)
     ap.add_argument("--e2e-host-layers", type=int, default=4)
     ap.add_argument("--gemm-iters", type=int, default=20)
+    ap.add_argument("--sweep-length", action="store_true",
+                    help="raw restore/save bandwidth against prefix length (1K..128K tokens)")
+    ap.add_argument("--sweep-host", action="store_true", help="sweep against the pinned-host store")
     ap.add_argument("--sched-demo", action="store_true",
                     help="layer-wise pipelining under the slack-aware scheduler")
     ap.add_argument("--sched-host", action="store_true")
@@ -942,6 +992,8 @@ def main():
         run_reference(args)
     elif args.sched_demo:
         run_sched_demo(args)
+    elif args.sweep_length:
+        run_length_sweep(args)
     elif args.config == 3:
         run_config3(args)
     elif args.config == 5:

@@ -372,7 +372,7 @@ def cpu_baseline(rep, seconds_hint=12.0):
         done_bytes += 2 * rep.payload_per_layer
         layers += 1
     return {"value": round(done_bytes / t_total / 1e9, 3), "unit": "GB/s", "cores": 1,
-            "kind": "oracle", "seconds": round(t_total, 2),
+            "host_cores": os.cpu_count(), "kind": "oracle", "seconds": round(t_total, 2),
             "sample": f"restore+save of {layers} full layers of the same batch "
                       f"({done_bytes / GIB:.1f} GiB payload), single thread"}
 
@@ -941,8 +941,8 @@ def run_reference(args):
         "ms_per_step": round(dt / args.steps * 1e3, 2), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": workload_name(w), "sample": sample},
-        "cpu_baseline": {"value": round(value, 3), "unit": "GB/s", "cores": 1, "kind": "oracle",
-                         "sample": sample},
+        "cpu_baseline": {"value": round(value, 3), "unit": "GB/s", "cores": 1,
+                         "host_cores": os.cpu_count(), "kind": "oracle", "sample": sample},
         "e2e": {"value": round(value, 3), "unit": "GB/s", "h2d_bytes_per_step": 0,
                 "d2h_bytes_per_step": 0},
         "gpu_launches": 0}), flush=True)

@@ -753,7 +753,9 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     p.n_iocb = n_iocb;
     p.opcode = opcode;
     p.wait_ns = opt.wait_ns;
-    p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : 4;
+    // measured: small claims balance best when every SM takes part, larger ones amortise the
+    // claim's round trip when few SMs carry everything
+    p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : (sm_count ? 4 : 2);
     uint32_t engine = opt.engine;
     // measured: bulk-async wins on HBM, also for head-major blocks when tensor maps exist
     if (engine == 0) engine = (host_store || (pool_hnd && !(maps && maps->valid))) ? 1 : 2;

@@ -173,7 +173,7 @@ int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
     c->pool.assign(geom->n_layers, PoolLayer{0, 0, 0, 0, false});
     for (auto &s : c->store) s = StoreDev{0, 0, 0, false, false};
     memset(&c->maps, 0, sizeof(c->maps));
-    c->opt = CopyOptions{0, 2000000ull, 4, 0, 0, 4, 0};   // 0 = chosen per launch
+    c->opt = CopyOptions{0, 2000000ull, 4, 0, 0, 0, 0};   // 0 = chosen per launch
     c->gdev.block_tokens = geom->block_tokens;
     c->gdev.obj_tokens = geom->obj_tokens;
     c->gdev.blocks_per_obj = (uint32_t)lo.blocks_per_obj;

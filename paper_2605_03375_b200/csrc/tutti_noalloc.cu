@@ -135,7 +135,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         BatchDev b{batch->n_req, batch->n_obj, batch->n_blk, batch->hit_tokens, batch->obj_start,
                    batch->obj_slot, batch->blk_start, batch->block_ids};
         PoolLayer pool{(uint64_t)k_base, (uint64_t)v_base, block_stride, n_blocks, true};
-        CopyOptions opt{2, 2000000ull, 4, 0, 0, 4, 0};
+        CopyOptions opt{2, 2000000ull, 4, 0, 0, 0, 0};
         uint32_t launches = 0;
         // header, completion slot and counters must start at zero: the array still holds
         // whatever the previous call left there

@@ -235,12 +235,18 @@ class Replica:
         self.table_bytes = sum(t.numel() * 4 for t in self.tables_host)
         n_iocb_layer = max(1, -(-2 * len(w.obj_slot) // args.ioctx_per_iocb))
         depth = 1
-        while depth < 2 * w.n_layers * n_iocb_layer:
+        while depth < 4 * w.n_layers * n_iocb_layer:        # two passes may be in flight
             depth *= 2
         self.ring = T.Ring(self.ctx, depth, args.ioctx_per_iocb,
-                           2 * len(w.block_ids) * (2 * w.n_layers + 1), 2 * len(w.obj_slot))
+                           2 * len(w.block_ids) * (4 * w.n_layers + 1), 2 * len(w.obj_slot))
         self.stream = torch.cuda.Stream(self.dev)
         self.build_stream = torch.cuda.Stream(self.dev)
+        self.write_stream = torch.cuda.Stream(self.dev)
+        self.saved_ev = {}          # duplex mode: last save of every layer
+        # duplex mode: each direction on a few SMs, so that both kernels are resident at once
+        # (the host link, not the SM count, bounds them)
+        self.duplex_sms = getattr(args, "e2e_sms", 8)
+        self.unpolled = []          # duplex mode: IOCBs of the previous pass
         self.two_streams = not getattr(args, "one_stream", False)
         self.layers_per_launch = getattr(args, "layers_per_launch", 4) or 1
         self.epoch = 1
@@ -317,6 +323,69 @@ class Replica:
                 if rc != T.OK or cqe.status != 0:
                     raise RuntimeError(f"IOCB {i}: poll rc {rc}, status {cqe.status}")
                 total += cqe.bytes
+        return total
+
+    def poll_list(self, issued):
+        T = self.T
+        total = 0
+        for first, n in issued:
+            for i in range(first, first + n):
+                rc, cqe = self.ring.tutti_ring_poll(i, 20_000_000_000)
+                if rc != T.OK or cqe.status != 0:
+                    raise RuntimeError(f"IOCB {i}: poll rc {rc}, status {cqe.status}")
+                total += cqe.bytes
+        return total
+
+    def step_duplex(self, upload_tables=False):
+        """One pass with both directions of the host link busy: layer l is saved on its own
+        stream as soon as it has been restored, while layer l+1 is being restored.  Ordering is
+        by events: a save waits for the restore of its layer, a restore waits for the previous
+        pass's save of its layer (same objects, same pool buffer).  Completions of a pass are
+        polled after the next pass has been issued, so the streams never run dry."""
+        T, torch = self.T, self.torch
+        sR, sW, sb = self.stream, self.write_stream, self.build_stream
+        assert self.R == self.w.n_layers, "duplex mode needs one pool buffer per layer"
+        self.epoch += 1
+        self.batch.plan_epoch = self.epoch
+        issued = []
+        start = torch.cuda.Event()
+        start.record(sR)
+        sb.wait_event(start)
+        if upload_tables:
+            with torch.cuda.stream(sb):
+                if self.saved_ev:       # the tables are read by builds still in flight
+                    for ev in self.saved_ev.values():
+                        sb.wait_event(ev)
+                for h, d in zip(self.tables_host, self.tables_dev):
+                    d.copy_(h, non_blocking=True)
+        for l in range(self.w.n_layers):
+            rc, fr, nr = self.ring.tutti_build_sqes(self.batch, l, T.OP_READ, stream=sb)
+            rc, fw, nw = self.ring.tutti_build_sqes(self.batch, l, T.OP_WRITE, stream=sb)
+            built = torch.cuda.Event()
+            built.record(sb)
+            sR.wait_event(built)
+            if l in self.saved_ev:
+                sR.wait_event(self.saved_ev[l])
+            self.ring.tutti_kv_restore_layer(fr, nr, self.duplex_sms, stream=sR)
+            restored = torch.cuda.Event()
+            restored.record(sR)
+            sW.wait_event(built)
+            sW.wait_event(restored)
+            self.ring.tutti_kv_save_layer(fw, nw, self.duplex_sms, stream=sW)
+            saved = torch.cuda.Event()
+            saved.record(sW)
+            self.saved_ev[l] = saved
+            issued += [(fr, nr), (fw, nw)]
+        total = self.poll_list(self.unpolled)
+        self.unpolled = issued
+        return total
+
+    def finish_duplex(self):
+        """Join the save stream into the restore stream and poll what is outstanding."""
+        for ev in self.saved_ev.values():
+            self.stream.wait_event(ev)
+        total = self.poll_list(self.unpolled)
+        self.unpolled = []
         return total
 
     def verify_samples(self, n_samples=256):
@@ -508,12 +577,19 @@ def run_e2e(args, local_rank, world):
     back to it, and reads the completions on the host."""
     import torch
     a2 = argparse.Namespace(**vars(args))
-    a2.resident_layers = 2
     L_host = min(args.e2e_host_layers, 32)
+    a2.resident_layers = L_host
     rep = Replica(a2, local_rank, host_store=True, n_layers=L_host)
     passes = max(1, 32 // L_host) if args.config in (2, 5) else 1
-    for _ in range(1):
-        rep.step(upload_tables=True)
+    duplex = not args.e2e_serial
+    if duplex:
+        rep.ctx.tutti_set_option(rep.T.OPT_COPY_ENGINE, rep.T.ENGINE_BULK)
+
+    def one_pass():
+        return rep.step_duplex(upload_tables=True) if duplex else rep.step(upload_tables=True)
+    one_pass()
+    if duplex:
+        rep.finish_duplex()
     torch.cuda.synchronize()
     barrier(world)
     steps = max(1, min(args.steps, 3))
@@ -521,20 +597,30 @@ def run_e2e(args, local_rank, world):
     e0 = torch.cuda.Event(enable_timing=True)
     e1 = torch.cuda.Event(enable_timing=True)
     e0.record(rep.stream)
+    moved = 0
     for _ in range(steps * passes):
-        rep.step(upload_tables=True)
+        moved += one_pass()
+    if duplex:
+        moved += rep.finish_duplex()
     e1.record(rep.stream)
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3
     ms = max_over_ranks(max(e0.elapsed_time(e1), wall_ms), world, rep.dev) / steps
     layers = L_host * passes
     payload = 2 * layers * rep.payload_per_layer
+    assert moved == payload * steps, (moved, payload * steps)
+    ok = rep.verify_samples(64)
+    link_duplex = host_link_duplex_gbs(rep.dev) if world == 1 else None
     h2d = layers * rep.payload_per_layer + passes * rep.table_bytes
     d2h = layers * rep.payload_per_layer + 2 * layers * 32
     value = sum_over_ranks(float(payload), world, rep.dev) / (ms * 1e-3) / 1e9
     rep.close()
     return {"value": round(value, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
             "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms, 2),
+            "verified_vs_oracle_samples": bool(ok),
+            "host_link_duplex_gbs": None if link_duplex is None else round(link_duplex, 1),
+            "mode": "duplex: layer l saved while layer l+1 is restored (both directions of the "
+                    "host link busy)" if duplex else "serial: all restores, then all saves",
             "store": f"pinned host memory, zero-copy; {L_host} layers resident, "
                      f"{passes} passes per step = {layers} layer transfers each way"}
 
@@ -562,6 +648,28 @@ def host_link_gbs(dev, nbytes=1 << 30, reps=10):
         torch.cuda.synchronize()
         best = max(best, nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
     return h2d, best
+
+
+def host_link_duplex_gbs(dev, nbytes=1 << 30, reps=5):
+    """Both directions of the host link at once with the copy engines (two streams): the sum
+    of pinned->HBM and HBM->pinned bytes over the time both took."""
+    import torch
+    a_h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    b_h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    a_d = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    b_d = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    best = 0.0
+    for _ in range(reps):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        with torch.cuda.stream(s1):
+            a_d.copy_(a_h, non_blocking=True)
+        with torch.cuda.stream(s2):
+            b_h.copy_(b_d, non_blocking=True)
+        torch.cuda.synchronize()
+        best = max(best, 2 * nbytes / (time.perf_counter() - t0) / 1e9)
+    return best
 
 
 def run_config3(args):
@@ -966,7 +1074,11 @@ def main():
     ap.add_argument("--bulk-stages", type=int, default=0)
     ap.add_argument("--claim", type=int, default=0)
     ap.add_argument("--bulk-chunk", type=int, default=0)
-    ap.add_argument("--e2e-host-layers", type=int, default=4)
+    ap.add_argument("--e2e-host-layers", type=int, default=8)
+    ap.add_argument("--e2e-sms", type=int, default=8,
+                    help="e2e leg, duplex mode: SMs per direction")
+    ap.add_argument("--e2e-serial", action="store_true",
+                    help="e2e leg: restore pass then save pass instead of overlapping them")
     ap.add_argument("--gemm-iters", type=int, default=20)
     ap.add_argument("--sweep-length", action="store_true",
                     help="raw restore/save bandwidth against prefix length (1K..128K tokens)")

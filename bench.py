@@ -246,6 +246,7 @@ class Replica:
         # duplex mode: each direction on a few SMs, so that both kernels are resident at once
         # (the host link, not the SM count, bounds them)
         self.duplex_sms = getattr(args, "e2e_sms", 8)
+        self.duplex_save_sms = getattr(args, "e2e_save_sms", 0) or self.duplex_sms
         self.unpolled = []          # duplex mode: IOCBs of the previous pass
         self.two_streams = not getattr(args, "one_stream", False)
         self.layers_per_launch = getattr(args, "layers_per_launch", 4) or 1
@@ -371,7 +372,7 @@ class Replica:
             restored.record(sR)
             sW.wait_event(built)
             sW.wait_event(restored)
-            self.ring.tutti_kv_save_layer(fw, nw, self.duplex_sms, stream=sW)
+            self.ring.tutti_kv_save_layer(fw, nw, self.duplex_save_sms, stream=sW)
             saved = torch.cuda.Event()
             saved.record(sW)
             self.saved_ev[l] = saved
@@ -1077,6 +1078,8 @@ def main():
     ap.add_argument("--e2e-host-layers", type=int, default=8)
     ap.add_argument("--e2e-sms", type=int, default=8,
                     help="e2e leg, duplex mode: SMs per direction")
+    ap.add_argument("--e2e-save-sms", type=int, default=0,
+                    help="e2e leg, duplex mode: SMs of the save direction (default: same)")
     ap.add_argument("--e2e-serial", action="store_true",
                     help="e2e leg: restore pass then save pass instead of overlapping them")
     ap.add_argument("--gemm-iters", type=int, default=20)

@@ -161,6 +161,7 @@ class Workload:
     block_ids: np.ndarray           # int32[n_blk]
     occupied_blocks: np.ndarray     # int32[]: pool blocks holding background data
     pool_hnd: bool = False          # pool blocks are [head][token][dim] (else [token][head][dim])
+    pool_pad_bytes: int = 0         # unused bytes after every block (block stride > block bytes)
 
     @property
     def n_req(self) -> int:
@@ -233,7 +234,8 @@ def make_workload(name: str, *, seed: int, n_layers: int, hit_tokens, block_toke
                   slot_space_factor: float = 1.25, occupancy: float = 0.6,
                   pool_round: int = 1024, pool_interleaved: bool = False,
                   store_kind: str = "hbm", n_pool_blocks: Optional[int] = None,
-                  consecutive_slots: bool = False, pool_hnd: bool = False) -> Workload:
+                  consecutive_slots: bool = False, pool_hnd: bool = False,
+                  pool_pad_bytes: int = 0) -> Workload:
     rng = np.random.default_rng(seed)
     hit = np.asarray(hit_tokens, dtype=np.uint32)
     assert np.all(hit % block_tokens == 0)
@@ -268,7 +270,7 @@ def make_workload(name: str, *, seed: int, n_layers: int, hit_tokens, block_toke
                     store_kind=store_kind, hit_tokens=hit, obj_start=_csr(objs),
                     obj_slot=obj_slot.astype(np.uint32), blk_start=_csr(blks),
                     block_ids=block_ids, occupied_blocks=occupied.astype(np.int32),
-                    pool_hnd=pool_hnd)
+                    pool_hnd=pool_hnd, pool_pad_bytes=pool_pad_bytes)
 
 
 def config(index: int, scale: float = 1.0, **overrides) -> Workload:

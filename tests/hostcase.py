@@ -18,9 +18,10 @@ def pool_geometry(w, lo):
     """(pool_bytes, k_off, v_off, block_stride) of one pool layer."""
     bb = int(lo.block_bytes)
     n = w.n_pool_blocks
+    pad = int(getattr(w, "pool_pad_bytes", 0))
     if w.pool_interleaved:
-        return 2 * n * bb, 0, bb, 2 * bb
-    return 2 * n * bb, 0, n * bb, bb
+        return 2 * n * (bb + pad), 0, bb + pad, 2 * (bb + pad)
+    return 2 * n * (bb + pad), 0, n * (bb + pad), bb + pad
 
 
 def make_store(w, lo, layers=None):

@@ -33,7 +33,8 @@ def random_workload(seed):
         elem_bytes=elem, n_devices=int(rng.choice([1, 1, 2, 3])),
         layout=int(rng.choice([wl.LAYOUT_FILE_MAJOR, wl.LAYOUT_LAYER_MAJOR])),
         slot_mean_run=float(rng.choice([1.0, 2.0, 6.0])), slot_space_factor=float(rng.choice([1.1, 2.0])),
-        pool_round=64, pool_interleaved=bool(rng.random() < 0.4), pool_hnd=hnd), rng
+        pool_round=64, pool_interleaved=bool(rng.random() < 0.4), pool_hnd=hnd,
+        pool_pad_bytes=int(rng.choice([0, 0, 16, 256]))), rng
 
 
 @pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TUTTI_FUZZ_CASES", "40"))))

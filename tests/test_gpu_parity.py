@@ -28,6 +28,9 @@ CASES = {
     "odd-token-bytes": dict(index=4, scale=0.03, n_layers=2, n_kv_heads=3, head_dim=8,
                             block_tokens=4, obj_tokens=32),
     "fp8-kv": dict(index=2, scale=0.04, n_layers=2, elem_bytes=1),
+    "padded-block-stride": dict(index=2, scale=0.04, n_layers=2, pool_pad_bytes=4096),
+    "padded-stride-1-token-pages": dict(index=4, scale=0.03, n_layers=2, pool_pad_bytes=48,
+                                        pool_interleaved=True),
     "hnd-pool": dict(index=2, scale=0.05, n_layers=2, pool_hnd=True),
     "hnd-pool-small-blocks": dict(index=4, scale=0.03, n_layers=2, pool_hnd=True, n_kv_heads=4,
                                   head_dim=64, block_tokens=2, obj_tokens=32),

@@ -137,6 +137,13 @@ def _expected_pool_numpy(w, lo, store, pool_before, layer):
             nd = exp.reshape(2, w.n_pool_blocks, w.n_kv_heads, w.block_tokens, row)
             nd = nd.transpose(0, 1, 3, 2, 4)
         # nd is now [kv][block][token][head][row]
+    elif w.pool_pad_bytes:
+        # every block is followed by unused bytes: a strided view that steps over them
+        assert not w.pool_interleaved
+        step = w.block_tokens * tb + w.pool_pad_bytes
+        nd = np.lib.stride_tricks.as_strided(
+            exp, shape=(2, w.n_pool_blocks, w.block_tokens, tb),
+            strides=(w.n_pool_blocks * step, step, tb, 1))
     elif w.pool_interleaved:
         nd = exp.reshape(w.n_pool_blocks, 2, w.block_tokens, tb).transpose(1, 0, 2, 3)
     else:
@@ -172,6 +179,7 @@ CASES = [
     dict(index=3, scale=0.02, n_layers=2),
     dict(index=1),
     dict(index=2, scale=0.03, n_layers=2, pool_hnd=True),
+    dict(index=2, scale=0.03, n_layers=2, pool_pad_bytes=64),
     dict(index=4, scale=0.02, n_layers=2, pool_hnd=True, pool_interleaved=True, n_kv_heads=4,
          head_dim=32, block_tokens=4, obj_tokens=32),
 ]

@@ -30,8 +30,10 @@ OP_HND = 0x100       # opcode flag: head-major pool blocks
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (no GPU toolchain involved)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = f"{_LIB}.{os.getpid()}.tmp"       # several processes may build at once
         subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC",
-                               _SRC, "-o", _LIB])
+                               _SRC, "-o", tmp])
+        os.replace(tmp, _LIB)
     return _LIB
 
 

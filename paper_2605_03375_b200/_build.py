@@ -29,8 +29,10 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(_CSRC, s) for s in SOURCES] + ["-o", LIB_PATH]
+    tmp = f"{LIB_PATH}.{os.getpid()}.tmp"           # several processes may build at once
+    cmd += [os.path.join(_CSRC, s) for s in SOURCES] + ["-o", tmp]
     subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
     return LIB_PATH
 
 

@@ -290,13 +290,9 @@ class Replica:
                     # descriptors are built on their own stream, ahead of the copies; one
                     # copy launch then executes the IOCBs of G consecutive layers (each
                     # layer keeps its own IOCBs and completion entries)
-                    first, n = None, 0
-                    for l in range(l0, min(l0 + G, self.w.n_layers)):
-                        rc, f, k = self.ring.tutti_build_sqes(self.batch, l, op, stream=sb)
-                        if first is None:
-                            first = f
-                        assert f == first + n, "IOCB indices of consecutive builds are contiguous"
-                        n += k
+                    g = min(G, self.w.n_layers - l0)
+                    rc, first, per = self.ring.tutti_build_sqes_layers(self.batch, l0, g, op, stream=sb)
+                    n = g * per
                     if self.two_streams:
                         built = torch.cuda.Event()
                         built.record(sb)

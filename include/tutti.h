@@ -219,6 +219,19 @@ int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *
                      uint32_t *n_iocb);
 
 /*
+ * The same build for n_layers consecutive layers in ONE kernel launch (the batch is known
+ * when the request arrives, so all its layers' contexts can be prepared ahead, Section 3.3
+ * "When an inference request arrives, the runtime enqueues the corresponding read IOCBs").
+ * Layer first_layer + k owns the IOCBs [*first_iocb + k * *iocbs_per_layer,
+ * *first_iocb + (k + 1) * *iocbs_per_layer); the descriptors are exactly those of
+ * tutti_build_sqes for that layer.  The reservation is one group: its SGL entries are
+ * reusable once every IOCB of every layer has been polled.
+ */
+int tutti_build_sqes_layers(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch,
+                            uint32_t first_layer, uint32_t n_layers, uint32_t opcode, void *stream,
+                            uint32_t *first_iocb, uint32_t *iocbs_per_layer);
+
+/*
  * Layer-wise Retrieve (Section 3.1; retrieve_layer of Section 3.4; issue_io of
  * Section 3.2 step 3): execute the READ IOCBs [first_iocb, first_iocb + n_iocb):
  * for every context, the bytes at its object-store range are scattered to the

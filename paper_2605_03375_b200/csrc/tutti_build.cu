@@ -339,10 +339,23 @@ struct EmitParams {
     uint64_t store_base[TUTTI_MAX_DEVICES];
     uint64_t store_bytes[TUTTI_MAX_DEVICES];
     uint32_t first_iocb, n_iocb, sgl_base, sgl_reserved;
+    const PoolLayerDev *pools;   // per-layer pool table for launches that cover several layers
 };
 
+// blockIdx.y selects the layer of a multi-layer launch: layer p.layer + y, whose IOCBs and
+// arena range follow those of the layer before it.
 __global__ void __launch_bounds__(EMIT_THREADS)
 emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
+    if (p.pools) {
+        const PoolLayerDev pl = p.pools[p.layer + blockIdx.y];
+        p.k_base = pl.k_base;
+        p.v_base = pl.v_base;
+        p.block_stride = pl.block_stride;
+        p.n_pool_blocks = pl.n_blocks;
+    }
+    p.layer += blockIdx.y;
+    p.first_iocb += blockIdx.y * p.n_iocb;
+    p.sgl_base += blockIdx.y * p.sgl_reserved;
     const PlanCounts pc = *ring.plan_counts;
     IocbHdr *hdr0 = &ring.hdrs[p.first_iocb & (ring.depth - 1)];
     int32_t status = pc.status;
@@ -541,10 +554,11 @@ cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev
 }
 
 cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
-                        uint32_t layer, uint32_t opcode, const PoolLayer &pool,
-                        const uint64_t *store_base, const uint64_t *store_bytes,
-                        uint32_t first_iocb, uint32_t n_iocb, uint32_t sgl_base,
-                        uint32_t sgl_reserved, int device_sms, cudaStream_t stream) {
+                        uint32_t layer, uint32_t n_layers, uint32_t opcode, const PoolLayer &pool,
+                        const PoolLayerDev *pools, const uint64_t *store_base,
+                        const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
+                        uint32_t sgl_base, uint32_t sgl_reserved, int device_sms,
+                        cudaStream_t stream) {
     EmitParams p;
     p.layer = layer;
     p.opcode = opcode;
@@ -552,24 +566,25 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
     p.v_base = pool.v_base;
     p.block_stride = pool.block_stride;
     p.n_pool_blocks = pool.n_blocks;
+    p.pools = pools;
     for (int d = 0; d < TUTTI_MAX_DEVICES; ++d) {
         p.store_base[d] = store_base[d];
         p.store_bytes[d] = store_bytes[d];
     }
-    p.first_iocb = first_iocb;
+    p.first_iocb = first_iocb;       // of the first layer; n_iocb and sgl_reserved are per layer
     p.n_iocb = n_iocb;
     p.sgl_base = sgl_base;
     p.sgl_reserved = sgl_reserved;
-    // one warp per item, 8 warps per CTA; a few CTAs per SM at most
     uint32_t items = 2u * batch.n_obj;
     uint32_t G = 1;
     while (G < 32 && G < geom.blocks_per_obj) G <<= 1;
     const uint32_t per_cta = 8 * (32 / G);             // 8 warps, 32/G items side by side
     uint32_t ctas = (items + per_cta - 1) / per_cta;
     uint32_t cap = (uint32_t)device_sms * 2u;
+    if (n_layers > 1) cap = cap / (n_layers < 8 ? n_layers : 8) + 1;   // the layers share the SMs
     if (ctas > cap) ctas = cap;
     if (ctas == 0) ctas = 1;
-    emit_kernel<<<ctas, EMIT_THREADS, 0, stream>>>(ring, geom, batch, p);
+    emit_kernel<<<dim3(ctas, n_layers), EMIT_THREADS, 0, stream>>>(ring, geom, batch, p);
     return cudaGetLastError();
 }
 

@@ -58,6 +58,11 @@ struct PoolLayer {
     bool registered;
 };
 
+// Device-resident copy of a registered pool layer (table indexed by layer).
+struct PoolLayerDev {
+    uint64_t k_base, v_base, block_stride, n_blocks;
+};
+
 struct StoreDev {
     uint64_t base, bytes;
     uint32_t kind;
@@ -127,8 +132,9 @@ struct CopyOptions {
 cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
                         cudaStream_t stream, uint32_t *launches);
 cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
-                        uint32_t layer, uint32_t opcode, const PoolLayer &pool,
-                        const uint64_t *store_base, const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
+                        uint32_t layer, uint32_t n_layers, uint32_t opcode, const PoolLayer &pool,
+                        const PoolLayerDev *pools, const uint64_t *store_base,
+                        const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
                         uint32_t sgl_base, uint32_t sgl_reserved, int device_sms,
                         cudaStream_t stream);
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,

@@ -71,6 +71,7 @@ struct tutti_ctx {
     void *partition = nullptr;   // SM partition state (tutti_partition.cu)
     bool pool_hnd = false;       // pool blocks are [head][token][dim]
     StoreTensorMaps maps;        // for the transposing bulk copies
+    PoolLayerDev *d_pools = nullptr;   // device copy of the pool table (multi-layer builds)
 };
 
 struct tutti_ring {
@@ -185,6 +186,13 @@ int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
     c->gdev.stride_slot = lo.stride_slot;
     c->gdev.n_slots = geom->n_slots;
     c->gdev.dev_bytes = lo.dev_bytes;
+    cudaError_t e = cudaMalloc((void **)&c->d_pools, sizeof(PoolLayerDev) * geom->n_layers);
+    if (e == cudaSuccess) e = cudaMemset(c->d_pools, 0, sizeof(PoolLayerDev) * geom->n_layers);
+    if (e != cudaSuccess) {
+        delete c;
+        cuda_fail(e, "cudaMalloc(pool table)");
+        return TUTTI_ENOMEM;
+    }
     *out = c;
     return TUTTI_OK;
 }
@@ -192,6 +200,10 @@ int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
 int tutti_ctx_destroy(tutti_ctx_t *ctx) {
     if (!ctx) return TUTTI_EINVAL;
     tutti_sm_partition_destroy(ctx);
+    {
+        DeviceGuard guard(ctx->device);
+        if (ctx->d_pools) cudaFree(ctx->d_pools);
+    }
     delete ctx;
     return TUTTI_OK;
 }
@@ -203,6 +215,9 @@ int tutti_pool_register(tutti_ctx_t *ctx, uint32_t layer, void *k_base, void *v_
     if ((k | v | block_stride) & 15) return TUTTI_EINVAL;
     if (block_stride < ctx->layout.block_bytes || n_blocks > 0x7fffffffull) return TUTTI_EINVAL;
     ctx->pool[layer] = PoolLayer{k, v, block_stride, n_blocks, true};
+    PoolLayerDev pl{k, v, block_stride, n_blocks};
+    DeviceGuard guard(ctx->device);
+    CK(cudaMemcpy(ctx->d_pools + layer, &pl, sizeof(pl), cudaMemcpyHostToDevice));
     return TUTTI_OK;
 }
 
@@ -388,13 +403,16 @@ static bool same_plan(const tutti_batch_t &a, const tutti_batch_t &b) {
            a.block_ids == b.block_ids;
 }
 
-int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, uint32_t layer,
-                     uint32_t opcode, void *stream, uint32_t *first_iocb, uint32_t *n_iocb) {
-    if (!ctx || !r || r->ctx != ctx || !batch || !first_iocb || !n_iocb) return TUTTI_EINVAL;
+static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, uint32_t layer,
+                        uint32_t n_layers, uint32_t opcode, void *stream, uint32_t *first_iocb,
+                        uint32_t *iocbs_per_layer) {
+    if (!ctx || !r || r->ctx != ctx || !batch || !first_iocb || !iocbs_per_layer) return TUTTI_EINVAL;
     r->host_calls++;
-    if (layer >= ctx->geom.n_layers || (opcode != TUTTI_OP_READ && opcode != TUTTI_OP_WRITE))
+    if (n_layers == 0 || layer >= ctx->geom.n_layers || n_layers > ctx->geom.n_layers - layer ||
+        (opcode != TUTTI_OP_READ && opcode != TUTTI_OP_WRITE))
         return TUTTI_EINVAL;
-    if (!ctx->pool[layer].registered) return TUTTI_EINVAL;
+    for (uint32_t l = layer; l < layer + n_layers; ++l)
+        if (!ctx->pool[l].registered) return TUTTI_EINVAL;
     for (uint32_t d = 0; d < ctx->geom.n_devices; ++d)
         if (!ctx->store[d].registered) return TUTTI_EINVAL;
     if (batch->n_req && (!batch->hit_tokens || !batch->obj_start || !batch->blk_start))
@@ -403,15 +421,15 @@ int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *bat
     if (batch->n_obj > r->dev.max_items / 2 || batch->n_blk > 0x7fffffffu / 2) return TUTTI_EINVAL;
     const uint32_t items = 2u * batch->n_obj;
     const uint32_t need_sgl = 2u * batch->n_blk;
-    if (need_sgl > r->sgl_capacity) return TUTTI_EINVAL;
     uint32_t need_iocb = (items + r->dev.capacity - 1) / r->dev.capacity;
     if (need_iocb == 0) need_iocb = 1;
-    if (need_iocb > r->dev.depth) return TUTTI_EINVAL;
+    if ((uint64_t)need_sgl * n_layers > r->sgl_capacity) return TUTTI_EINVAL;
+    if ((uint64_t)need_iocb * n_layers > r->dev.depth) return TUTTI_EINVAL;
     uint32_t first = 0, sgl_base = 0;
-    int rc = r->host->reserve(need_iocb, need_sgl, &first, &sgl_base);
+    int rc = r->host->reserve(need_iocb * n_layers, need_sgl * n_layers, &first, &sgl_base);
     if (rc == -3) return TUTTI_EAGAIN;
     if (rc) return TUTTI_EINVAL;
-    for (uint32_t k = 0; k < need_iocb; ++k) {
+    for (uint32_t k = 0; k < need_iocb * n_layers; ++k) {
         uint32_t slot = (first + k) & (r->dev.depth - 1);
         r->have_cqe[slot] = 0;
         r->opcode_of[slot] = (uint8_t)opcode;
@@ -433,12 +451,25 @@ int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *bat
         sbytes[d] = ctx->store[d].bytes;
     }
     const uint32_t op_flags = opcode | (ctx->pool_hnd ? TUTTI_OP_FLAG_HND : 0u);
-    CK(launch_emit(r->dev, ctx->gdev, b, layer, op_flags, ctx->pool[layer], sbase, sbytes, first,
-                   need_iocb, sgl_base, need_sgl, ctx->device_sms, st));
+    CK(launch_emit(r->dev, ctx->gdev, b, layer, n_layers, op_flags, ctx->pool[layer],
+                   n_layers > 1 ? ctx->d_pools : nullptr, sbase, sbytes, first, need_iocb, sgl_base,
+                   need_sgl, ctx->device_sms, st));
     r->kernel_launches++;
     *first_iocb = first;
-    *n_iocb = need_iocb;
+    *iocbs_per_layer = need_iocb;
     return TUTTI_OK;
+}
+
+int tutti_build_sqes(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, uint32_t layer,
+                     uint32_t opcode, void *stream, uint32_t *first_iocb, uint32_t *n_iocb) {
+    return build_layers(ctx, r, batch, layer, 1, opcode, stream, first_iocb, n_iocb);
+}
+
+int tutti_build_sqes_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch,
+                            uint32_t first_layer, uint32_t n_layers, uint32_t opcode, void *stream,
+                            uint32_t *first_iocb, uint32_t *iocbs_per_layer) {
+    return build_layers(ctx, r, batch, first_layer, n_layers, opcode, stream, first_iocb,
+                        iocbs_per_layer);
 }
 
 static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, uint32_t sm_count,

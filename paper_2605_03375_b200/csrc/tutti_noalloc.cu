@@ -142,7 +142,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         cudaError_t e = cudaMemsetAsync(base, 0, CLEAR_BYTES, st);
         if (e == cudaSuccess) e = launch_plan(r, g, b, st, nullptr);
         if (e == cudaSuccess)
-            e = launch_emit(r, g, b, layer, TUTTI_OP_READ, pool, sbase, sbytes, 0, 1, 0,
+            e = launch_emit(r, g, b, layer, 1, TUTTI_OP_READ, pool, nullptr, sbase, sbytes, 0, 1, 0,
                             NA_MAX_ENTRIES, sms, st);
         if (e == cudaSuccess)
             e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, false,

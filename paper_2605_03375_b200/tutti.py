@@ -78,7 +78,7 @@ EXPORTS = [
     "tutti_sched_enqueue", "tutti_sched_next", "tutti_sched_pending",
     "tutti_filepool_create", "tutti_filepool_destroy", "tutti_filepool_insert",
     "tutti_filepool_lookup", "tutti_filepool_match_prefix", "tutti_filepool_pin",
-    "tutti_filepool_remove", "tutti_filepool_stats",
+    "tutti_filepool_remove", "tutti_filepool_stats", "tutti_build_sqes_layers",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -99,6 +99,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
     sig = {
         "tutti_obj_layout": (C.c_int, [P(Geom), P(Layout)]),
         "tutti_build_sqes": (C.c_int, [vp, vp, P(Batch), u32, u32, vp, P(u32), P(u32)]),
+        "tutti_build_sqes_layers": (C.c_int, [vp, vp, P(Batch), u32, u32, u32, vp, P(u32), P(u32)]),
         "tutti_kv_restore_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
         "tutti_kv_save_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
         "tutti_ring_poll": (C.c_int, [vp, u32, P(Cqe), u64]),
@@ -266,6 +267,16 @@ class Ring:
                                        _stream_ptr(stream), C.byref(first), C.byref(n))
         _check(rc, "tutti_build_sqes", allow)
         return rc, first.value, n.value
+
+    def tutti_build_sqes_layers(self, batch: Batch, first_layer: int, n_layers: int, opcode: int,
+                                stream=None, allow: Sequence[int] = ()) -> Tuple[int, int, int]:
+        """(rc, first_iocb, iocbs_per_layer): one launch builds n_layers consecutive layers."""
+        first, per = C.c_uint32(), C.c_uint32()
+        rc = self.lib.tutti_build_sqes_layers(self.ctx.h, self.h, C.byref(batch), first_layer,
+                                              n_layers, opcode, _stream_ptr(stream),
+                                              C.byref(first), C.byref(per))
+        _check(rc, "tutti_build_sqes_layers", allow)
+        return rc, first.value, per.value
 
     def tutti_kv_restore_layer(self, first_iocb: int, n_iocb: int, sm_count: int = 0, stream=None,
                                allow: Sequence[int] = ()) -> int:

@@ -232,3 +232,38 @@ def test_empty_batch_and_zero_hits():
         assert dc.poll_all(first, n) == [(first, 0, 0)]
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("capacity", [2048, 8])
+def test_all_layers_built_in_one_launch(capacity):
+    """tutti_build_sqes_layers: one launch prepares every layer; each layer's IOCBs hold
+    exactly the descriptors of a single-layer build, and one copy launch executes them all."""
+    w = mk("cfg2-small")
+    n_items = 2 * len(w.obj_slot)
+    per = max(1, -(-n_items // capacity))
+    depth = 1
+    while depth < 2 * per * w.n_layers:
+        depth *= 2
+    dc = DeviceCase(w, depth=depth, capacity=capacity, sgl_capacity=2 * len(w.block_ids) * (w.n_layers + 1))
+    try:
+        k0, _ = dc.ring.tutti_ring_stats()
+        rc, first, per_layer = dc.ring.tutti_build_sqes_layers(dc.batch, 0, w.n_layers, T.OP_READ)
+        assert per_layer == per
+        k1, _ = dc.ring.tutti_ring_stats()
+        assert k1 - k0 == 2                                   # plan + one emit for all layers
+        for layer in range(w.n_layers):
+            sq, sg, num, infos = dc.read_build(first + layer * per_layer, per_layer)
+            orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, capacity)
+            assert same_records(sq, osq) and same_records(sg, osg)
+            assert list(num[:len(onum)]) == list(onum) and not num[len(onum):].any()
+            assert all(i.layer == layer and i.status == 0 for i in infos)
+        dc.ring.tutti_kv_restore_layer(first, per_layer * w.n_layers)
+        cqes = dc.poll_all(first, per_layer * w.n_layers)
+        assert all(c[1] == 0 for c in cqes)
+        for layer in range(w.n_layers):
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        # a range that leaves the layer count is refused
+        rc, *_ = dc.ring.tutti_build_sqes_layers(dc.batch, 2, w.n_layers, T.OP_READ, allow=(T.EINVAL,))
+        assert rc == T.EINVAL
+    finally:
+        dc.close()

@@ -291,7 +291,14 @@ class Replica:
                     # copy launch then executes the IOCBs of G consecutive layers (each
                     # layer keeps its own IOCBs and completion entries)
                     g = min(G, self.w.n_layers - l0)
+                    if events is not None:
+                        ba = torch.cuda.Event(enable_timing=True)
+                        bb_ = torch.cuda.Event(enable_timing=True)
+                        ba.record(sb)
                     rc, first, per = self.ring.tutti_build_sqes_layers(self.batch, l0, g, op, stream=sb)
+                    if events is not None:
+                        bb_.record(sb)
+                        events["build"].append((ba, bb_, g))
                     n = g * per
                     if self.two_streams:
                         built = torch.cuda.Event()
@@ -467,7 +474,7 @@ def run_ours(args):
     k0, _ = rep.ring.tutti_ring_stats()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    events = {"pass": [], "copy": {T.OP_READ: [], T.OP_WRITE: []}}
+    events = {"pass": [], "build": [], "copy": {T.OP_READ: [], T.OP_WRITE: []}}
     barrier(world)
     torch.cuda.synchronize()
     e0 = torch.cuda.Event(enable_timing=True)
@@ -504,6 +511,8 @@ def run_ours(args):
                 "copy_kernel_ms": round(statistics.mean(ms), 4),
                 "copy_kernel_ms_min": round(min(ms), 4)}
     restore, save = dir_stats(T.OP_READ), dir_stats(T.OP_WRITE)
+    # descriptor build (plan once per step + emit), per layer, on the build stream
+    build_ms = statistics.mean(a.elapsed_time(b) / g for a, b, g in events["build"])
     verified = rep.verify_samples()
 
     out = None
@@ -531,6 +540,7 @@ def run_ours(args):
                        "layers_per_launch": rep.layers_per_launch,
                        "ioctx_per_iocb": args.ioctx_per_iocb},
             "restore": restore, "save": save,
+            "build_ms_per_layer": round(build_ms, 4),
             "blocks_per_s": restore["blocks_per_s"],
             "gpu_launches": int(k1 - k0),
             "verified_vs_oracle_samples": bool(verified),

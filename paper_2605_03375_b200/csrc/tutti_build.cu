@@ -178,23 +178,24 @@ __device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &ca
     }
     const uint32_t heads = __ballot_sync(0xffffffffu, v.b != 0);
     v.b = __popc(heads & (0xffffffffu >> (31 - lane)));
+    const uint32_t n_warps = blockDim.x >> 5;
     if (lane == 31) warp_tot[warp] = v;
     __syncthreads();
     if (warp == 0) {
-        ScanPair w = warp_tot[lane];       // blockDim.x == 1024 -> 32 warps
+        ScanPair w = lane < n_warps ? warp_tot[lane] : ScanPair{0, 0};
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             uint32_t ua = __shfl_up_sync(0xffffffffu, w.a, d);
             uint32_t ub = __shfl_up_sync(0xffffffffu, w.b, d);
             if (lane >= (uint32_t)d) { w.a += ua; w.b += ub; }
         }
-        warp_tot[lane] = w;
+        if (lane < n_warps) warp_tot[lane] = w;
     }
     __syncthreads();
     ScanPair off = carry;
     if (warp > 0) { off.a += warp_tot[warp - 1].a; off.b += warp_tot[warp - 1].b; }
     v.a += off.a; v.b += off.b;
-    ScanPair tot = warp_tot[31];
+    ScanPair tot = warp_tot[n_warps - 1];
     __syncthreads();
     if (threadIdx.x == 0) { carry.a += tot.a; carry.b += tot.b; }
     __syncthreads();
@@ -527,7 +528,10 @@ cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev
     }
     uint32_t n = 0;
     if (np <= SMEM_SORT_ITEMS) {
-        plan_kernel<<<1, PLAN_THREADS, (size_t)np * 12, stream>>>(ring, geom, batch, np, 1, 0);
+        // small batches get a small CTA: the kernel is a chain of block-wide barriers
+        uint32_t threads = 64;
+        while (threads < PLAN_THREADS && threads < np / 2) threads <<= 1;
+        plan_kernel<<<1, threads, (size_t)np * 12, stream>>>(ring, geom, batch, np, 1, 0);
         n = 1;
     } else {
         // keys, then the sorting network as a handful of launches, then flags and scans

@@ -106,3 +106,26 @@ class DeviceCase:
             assert rc == T.OK, f"poll {i}: {rc}"
             out.append((cqe.iocb_idx, cqe.status, cqe.bytes))
         return out
+
+
+def verify_replica_samples(rep, n_samples=256):
+    """Sampled outputs at full size for a bench.Replica: for random (token, head) rows the oracle
+    names the store bytes and the pool bytes that must be equal after a restore."""
+    w = rep.w
+    og = oracle.geom_of(w)
+    ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
+    rng = np.random.default_rng(4321)
+    row = w.head_dim * w.elem_bytes
+    for _ in range(n_samples):
+        l = int(rng.integers(w.n_layers - rep.R, w.n_layers))    # layers whose pool buffer is still theirs
+        r = int(rng.integers(0, w.n_req))
+        t = int(rng.integers(0, int(w.hit_tokens[r])))
+        kv = int(rng.integers(0, 2))
+        hd = int(rng.integers(0, w.n_kv_heads))
+        d, so, blk, bo = oracle.row_location(og, l, ob, r, t, kv, hd, w.pool_hnd)
+        po = kv * rep.v_off + blk * rep.block_bytes + bo
+        a = rep.store[d][so:so + row].to(rep.dev)
+        b = rep.pool[l % rep.R][po:po + row]
+        if not torch.equal(a, b):
+            return False
+    return True

@@ -9,6 +9,7 @@ import torch
 
 import bench
 import oracle
+from tests.devcase import verify_replica_samples
 from paper_2605_03375_b200 import tutti as T
 
 pytestmark = pytest.mark.gpu
@@ -31,7 +32,7 @@ def test_config2_full_size(engine):
         moved = rep.step(directions=(T.OP_READ,))
         assert moved == 32 * rep.payload_per_layer == 32 << 30
         torch.cuda.synchronize()
-        assert rep.verify_samples(512)
+        assert verify_replica_samples(rep, 512)
         # whole layers against the oracle on host copies (layers 29..31 own the 3 pool buffers)
         og = oracle.geom(1, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
                          w.n_devices, w.layout, w.n_slots)
@@ -122,7 +123,7 @@ def test_config4_full_size_per_layer():
         before = rep.pool[1].clone()
         moved = rep.step(directions=(T.OP_READ,))
         assert moved == 2 * rep.payload_per_layer
-        assert rep.verify_samples(512)
+        assert verify_replica_samples(rep, 512)
         _whole_layer_check(rep, 1, before)
     finally:
         rep.close()
@@ -137,7 +138,7 @@ def test_config3_full_size_per_layer_from_pinned_host():
         assert (w.n_req, w.obj_tokens, len(w.block_ids)) == (2, 1024, 16384)
         before = rep.pool[1].clone()
         rep.step(directions=(T.OP_READ,))
-        assert rep.verify_samples(256)
+        assert verify_replica_samples(rep, 256)
         _whole_layer_check(rep, 1, before)
         orig = [s.clone() for s in rep.store]
         for s in rep.store:
@@ -179,7 +180,7 @@ def test_config5_capped_restore_beside_a_gemm(sm_count):
         moved = rep.step(sm_count=got_io, directions=(T.OP_READ,))
         torch.cuda.synchronize()
         assert moved == 2 * rep.payload_per_layer
-        assert rep.verify_samples(256)
+        assert verify_replica_samples(rep, 256)
         _whole_layer_check(rep, 1, before)
         assert torch.allclose(c.float(), ref, rtol=2e-2, atol=2.0)       # the GEMM was not disturbed
         rep.ctx.tutti_sm_partition_destroy()

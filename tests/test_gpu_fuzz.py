@@ -177,3 +177,98 @@ def test_random_op_sequences_on_a_small_ring(seed):
         assert n_again > 0 or depth >= 80 * per_build
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_host_prepared_descriptors(seed):
+    """CPU-prepared IOCBs with entries cut at random 16-byte boundaries (differing lengths),
+    in both directions and on both engines."""
+    rng = np.random.default_rng(300 + seed)
+    w = wl.config(2, 0.03, n_layers=2, n_devices=int(rng.choice([1, 2])), slot_mean_run=2.0,
+                  pool_interleaved=bool(seed & 1))
+    dc = DeviceCase(w, depth=8, capacity=2048, sgl_capacity=64 * len(w.block_ids))
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, int(rng.choice([1, 2])))
+        layer = int(rng.integers(0, 2))
+        op = T.OP_READ if seed % 3 else T.OP_WRITE
+        orc, osq, osg, onum = dc.oracle_descriptors(layer, op, 2048)
+        # cut every entry into 1..4 pieces at random multiples of 16 bytes
+        addr, ln, ident, counts = [], [], [], []
+        for e in osg:
+            total = int(e["len"])
+            k = int(rng.integers(1, 5))
+            cuts = sorted(set((rng.integers(1, total // 16, size=k - 1) * 16).tolist())) if k > 1 else []
+            edges = [0] + cuts + [total]
+            counts.append(len(edges) - 1)
+            for a, b in zip(edges[:-1], edges[1:]):
+                addr.append(int(e["addr"]) + a)
+                ln.append(b - a)
+                ident.append(int(e["id"]))
+        sg2 = np.zeros(len(addr), dtype=osg.dtype)
+        sg2["addr"], sg2["len"], sg2["id"] = addr, ln, ident
+        cum = np.concatenate([[0], np.cumsum(counts)])
+        sq2 = osq.copy()
+        sq2["sgl_first"] = cum[osq["sgl_first"]]
+        sq2["sgl_count"] = cum[osq["sgl_first"] + osq["sgl_count"]] - cum[osq["sgl_first"]]
+        if op == T.OP_WRITE:
+            noise = torch.randint(0, 255, (dc.pool_dev[layer].numel(),), dtype=torch.uint8, device=dc.dev)
+            dc.pool_dev[layer].copy_(noise)
+            for t in dc.store_dev:
+                t.zero_()
+        rc, first = dc.ring.tutti_ring_reserve(1, len(sg2))
+        dc.ring.tutti_ring_fill_host(first, sq2, sg2)
+        info, _ = dc.ring.tutti_ring_read_iocb(first)
+        assert info.entry_len == 0 or len(set(ln)) == 1
+        sm = int(rng.choice([0, 5]))
+        (dc.ring.tutti_kv_restore_layer if op == T.OP_READ else dc.ring.tutti_kv_save_layer)(first, 1, sm)
+        (idx, status, nbytes), = dc.poll_all(first, 1)
+        assert status == 0 and nbytes == int(osq["len"].sum())
+        if op == T.OP_READ:
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        else:
+            st = [np.zeros_like(s) for s in dc.store_host]
+            dc.oracle_save(layer, dc.pool_dev[layer].cpu().numpy(), st)
+            for t, s in zip(dc.store_dev, st):
+                assert np.array_equal(t.cpu().numpy(), s)
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_multi_layer_builds_and_launches(seed):
+    """Several layers built by one launch and executed by launches that cover random ranges
+    of their IOCBs."""
+    w, rng = random_workload(700 + seed)
+    w = wl.make_workload("ml", seed=w.seed, n_layers=int(rng.integers(2, 6)),
+                         hit_tokens=w.hit_tokens, block_tokens=w.block_tokens,
+                         obj_tokens=w.obj_tokens, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                         elem_bytes=w.elem_bytes, n_devices=w.n_devices, layout=w.layout,
+                         pool_round=64, pool_interleaved=w.pool_interleaved, pool_hnd=w.pool_hnd,
+                         pool_pad_bytes=w.pool_pad_bytes, slot_mean_run=2.0)
+    capacity = int(rng.choice([2, 16, 2048]))
+    per = max(1, -(-2 * len(w.obj_slot) // capacity))
+    depth = 1
+    while depth < 2 * per * w.n_layers:
+        depth *= 2
+    dc = DeviceCase(w, depth=depth, capacity=capacity,
+                    sgl_capacity=max(64, 2 * len(w.block_ids) * (w.n_layers + 1)))
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, int(rng.choice([0, 1, 2])))
+        l0 = int(rng.integers(0, w.n_layers - 1))
+        nl = int(rng.integers(1, w.n_layers - l0 + 1))
+        rc, first, per_layer = dc.ring.tutti_build_sqes_layers(dc.batch, l0, nl, T.OP_READ)
+        total = per_layer * nl
+        # execute in random consecutive pieces
+        at = 0
+        while at < total:
+            k = int(rng.integers(1, total - at + 1))
+            dc.ring.tutti_kv_restore_layer(first + at, k, int(rng.choice([0, 0, 7])))
+            at += k
+        cqes = dc.poll_all(first, total)
+        assert all(c[1] == 0 for c in cqes)
+        for l in range(l0, l0 + nl):
+            assert np.array_equal(dc.pool_dev[l].cpu().numpy(), dc.oracle_restore(l))
+        for l in list(range(0, l0)) + list(range(l0 + nl, w.n_layers)):
+            assert np.array_equal(dc.pool_dev[l].cpu().numpy(), dc.pool_host[l])   # untouched
+    finally:
+        dc.close()

@@ -445,9 +445,11 @@ void tutti_hostring_destroy(tutti_hostring_t *h);
 int tutti_hostring_reserve(tutti_hostring_t *h, uint32_t n_iocb, uint32_t n_sgl,
                            uint32_t *first_iocb, uint32_t *sgl_base);
 int tutti_hostring_release(tutti_hostring_t *h, uint32_t iocb_idx); /* IOCB polled */
+int tutti_hostring_cancel_last(tutti_hostring_t *h, uint32_t first_iocb); /* undo the newest reserve */
 int tutti_hostring_live(const tutti_hostring_t *h, uint32_t *iocbs, uint32_t *sgl_entries);
 
 const char *tutti_strerror(int code);
+/* Text of the last CUDA failure seen by the calling thread (valid until its next failure). */
 const char *tutti_last_cuda_error(void);
 uint32_t tutti_version(void);
 

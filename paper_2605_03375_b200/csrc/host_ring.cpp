@@ -54,6 +54,17 @@ int HostRing::reserve(uint32_t n_iocb, uint32_t n_sgl, uint32_t *first_iocb, uin
     return 0;
 }
 
+int HostRing::cancel_last(uint32_t first_iocb) {
+    if (groups_.empty() || groups_.back().first_iocb != first_iocb || groups_.back().n_released)
+        return -1;
+    const Group g = groups_.back();
+    groups_.pop_back();
+    head_ = g.first_iocb;
+    // the arena head goes back to where the previous group ends (or to 0 when none is left)
+    sgl_head_ = groups_.empty() ? 0 : groups_.back().sgl_begin + groups_.back().sgl_count;
+    return 0;
+}
+
 int HostRing::release(uint32_t iocb_idx) {
     if (!is_live(iocb_idx)) return -1;
     uint32_t slot = iocb_idx & (depth_ - 1);

@@ -31,6 +31,10 @@ public:
     // -3 no room right now.
     int reserve(uint32_t n_iocb, uint32_t n_sgl, uint32_t *first_iocb, uint32_t *sgl_base);
 
+    // Undo the most recent reserve() (its kernels could not be launched).  -1 if `first_iocb`
+    // is not the start of the newest group.
+    int cancel_last(uint32_t first_iocb);
+
     // Mark one IOCB as polled.  Releases whole groups from the front of the FIFO.
     // -1 if the index is not live or was released before.
     int release(uint32_t iocb_idx);

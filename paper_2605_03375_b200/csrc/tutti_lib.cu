@@ -438,9 +438,19 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
     cudaStream_t st = (cudaStream_t)stream;
     BatchDev b{batch->n_req, batch->n_obj, batch->n_blk, batch->hit_tokens, batch->obj_start,
                batch->obj_slot, batch->blk_start, batch->block_ids};
+    // a launch that fails must not leave its reservation behind
+#define CK_OR_CANCEL(call)                                         \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) {                                  \
+            r->host->cancel_last(first);                           \
+            r->plan_valid = false;                                 \
+            return cuda_fail(e__, #call);                          \
+        }                                                          \
+    } while (0)
     if (!(r->plan_valid && same_plan(r->plan_batch, *batch))) {
         uint32_t plan_launches = 0;
-        CK(launch_plan(r->dev, ctx->gdev, b, st, &plan_launches));
+        CK_OR_CANCEL(launch_plan(r->dev, ctx->gdev, b, st, &plan_launches));
         r->kernel_launches += plan_launches;
         r->plan_batch = *batch;
         r->plan_valid = batch->plan_epoch != 0;
@@ -451,9 +461,10 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
         sbytes[d] = ctx->store[d].bytes;
     }
     const uint32_t op_flags = opcode | (ctx->pool_hnd ? TUTTI_OP_FLAG_HND : 0u);
-    CK(launch_emit(r->dev, ctx->gdev, b, layer, n_layers, op_flags, ctx->pool[layer],
-                   n_layers > 1 ? ctx->d_pools : nullptr, sbase, sbytes, first, need_iocb, sgl_base,
-                   need_sgl, ctx->device_sms, st));
+    CK_OR_CANCEL(launch_emit(r->dev, ctx->gdev, b, layer, n_layers, op_flags, ctx->pool[layer],
+                             n_layers > 1 ? ctx->d_pools : nullptr, sbase, sbytes, first, need_iocb,
+                             sgl_base, need_sgl, ctx->device_sms, st));
+#undef CK_OR_CANCEL
     r->kernel_launches++;
     *first_iocb = first;
     *iocbs_per_layer = need_iocb;
@@ -693,6 +704,10 @@ int tutti_hostring_reserve(tutti_hostring_t *h, uint32_t n_iocb, uint32_t n_sgl,
 int tutti_hostring_release(tutti_hostring_t *h, uint32_t iocb_idx) {
     if (!h) return TUTTI_EINVAL;
     return h->ring.release(iocb_idx) ? TUTTI_EINVAL : TUTTI_OK;
+}
+int tutti_hostring_cancel_last(tutti_hostring_t *h, uint32_t first_iocb) {
+    if (!h) return TUTTI_EINVAL;
+    return h->ring.cancel_last(first_iocb) ? TUTTI_EINVAL : TUTTI_OK;
 }
 int tutti_hostring_live(const tutti_hostring_t *h, uint32_t *iocbs, uint32_t *sgl_entries) {
     if (!h) return TUTTI_EINVAL;

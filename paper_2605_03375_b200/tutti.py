@@ -71,7 +71,7 @@ EXPORTS = [
     "tutti_ring_reserve", "tutti_ring_fill_host", "tutti_ring_read_iocb", "tutti_ring_read_sgl",
     "tutti_ring_stats", "tutti_sm_partition_create", "tutti_sm_partition_destroy",
     "tutti_hostring_create", "tutti_hostring_destroy", "tutti_hostring_reserve",
-    "tutti_hostring_release", "tutti_hostring_live", "tutti_strerror", "tutti_last_cuda_error",
+    "tutti_hostring_release", "tutti_hostring_live", "tutti_hostring_cancel_last", "tutti_strerror", "tutti_last_cuda_error",
     "tutti_version", "tutti_kv_restore_layer_noalloc",
     "tutti_sched_create", "tutti_sched_destroy", "tutti_sched_set_slack",
     "tutti_sched_set_decode_slack", "tutti_sched_set_io_time", "tutti_sched_io_time",
@@ -122,6 +122,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_hostring_reserve": (C.c_int, [vp, u32, u32, P(u32), P(u32)]),
         "tutti_hostring_release": (C.c_int, [vp, u32]),
         "tutti_hostring_live": (C.c_int, [vp, P(u32), P(u32)]),
+        "tutti_hostring_cancel_last": (C.c_int, [vp, u32]),
         "tutti_strerror": (C.c_char_p, [C.c_int]),
         "tutti_last_cuda_error": (C.c_char_p, []),
         "tutti_version": (u32, []),

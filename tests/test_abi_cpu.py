@@ -74,6 +74,9 @@ class HostRing:
     def release(self, i):
         return self.lib.tutti_hostring_release(self.h, i)
 
+    def cancel_last(self, first):
+        return self.lib.tutti_hostring_cancel_last(self.h, first)
+
     def live(self):
         a, b = C.c_uint32(), C.c_uint32()
         self.lib.tutti_hostring_live(self.h, C.byref(a), C.byref(b))
@@ -166,3 +169,18 @@ def test_struct_sizes_match_the_header():
     assert C.sizeof(T.Cqe) == 16 and C.sizeof(T.IocbInfo) == 48 and C.sizeof(T.Launch) == 24
     assert T.SQE_DTYPE.itemsize == 32 and T.SGL_DTYPE.itemsize == 16
     assert oracle.SQE_DTYPE.itemsize == 32 and oracle.SGL_DTYPE.itemsize == 16
+
+
+def test_hostring_cancel_last_restores_the_previous_state():
+    r = HostRing(8, 100)
+    assert r.reserve(2, 30) == (0, 0, 0)
+    assert r.reserve(3, 50) == (0, 2, 30)
+    assert r.cancel_last(0) == T.EINVAL                 # not the newest group
+    assert r.cancel_last(2) == 0
+    assert r.live() == (2, 30)
+    assert r.reserve(1, 60) == (0, 2, 30)               # same index and arena position again
+    assert r.cancel_last(2) == 0 and r.cancel_last(0) == 0
+    assert r.live() == (0, 0)
+    assert r.reserve(4, 100) == (0, 0, 0)
+    assert r.release(1) == 0
+    assert r.cancel_last(0) == T.EINVAL                 # already partly consumed

@@ -264,6 +264,20 @@ int tutti_kv_save_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t first_ioc
  */
 int tutti_ring_poll(tutti_ring_t *ring, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns);
 
+/*
+ * GPU-side dependency on one IOCB (Section 3.2: once enqueued, "GPU-side dependency
+ * tracking" orders I/O and compute without the CPU): everything enqueued on `stream`
+ * after this call starts only once IOCB iocb_idx has completed — for instance a layer's
+ * attention behind that layer's restore, while the copy launch that carries it is still
+ * busy with later layers.  Implemented as a stream wait on the IOCB's state word; no
+ * kernel, no SM, no host involvement.  The IOCB must have been issued (or be issued later)
+ * with tutti_kv_restore_layer / tutti_kv_save_layer, otherwise the stream waits until the
+ * context is destroyed.  A completion with an error status also releases the stream; read
+ * the status with tutti_ring_poll.  TUTTI_ECUDA if the driver has no stream memory
+ * operations.
+ */
+int tutti_stream_wait_iocb(tutti_ring_t *ring, uint32_t iocb_idx, void *stream);
+
 /* ------------------------------------------------------------------------- */
 /* Lifecycle                                                                  */
 /* ------------------------------------------------------------------------- */

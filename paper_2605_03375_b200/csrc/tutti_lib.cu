@@ -557,6 +557,32 @@ int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64
     }
 }
 
+int tutti_stream_wait_iocb(tutti_ring_t *r, uint32_t iocb_idx, void *stream) {
+    if (!r || !r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
+    r->host_calls++;
+    typedef CUresult (*wait_fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+    static wait_fn fn = nullptr;
+    if (!fn) {
+        void *fp = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuStreamWaitValue32", &fp, cudaEnableDefault, &q) != cudaSuccess ||
+            !fp || q != cudaDriverEntryPointSuccess) {
+            g_last_cuda_error = "cuStreamWaitValue32 is not available";
+            return TUTTI_ECUDA;
+        }
+        fn = (wait_fn)fp;
+    }
+    DeviceGuard guard(r->ctx->device);
+    const uint32_t slot = iocb_idx & (r->dev.depth - 1);
+    CUdeviceptr addr = (CUdeviceptr)(uintptr_t)&r->dev.hdrs[slot].state;
+    CUresult res = fn((CUstream)stream, addr, state_word(iocb_idx, PHASE_DONE), CU_STREAM_WAIT_VALUE_EQ);
+    if (res != CUDA_SUCCESS) {
+        g_last_cuda_error = "cuStreamWaitValue32: CUresult " + std::to_string((int)res);
+        return TUTTI_ECUDA;
+    }
+    return TUTTI_OK;
+}
+
 int tutti_ring_reserve(tutti_ring_t *r, uint32_t n_iocb, uint32_t n_sgl, uint32_t *first_iocb) {
     if (!r || !first_iocb) return TUTTI_EINVAL;
     r->host_calls++;

@@ -79,6 +79,7 @@ EXPORTS = [
     "tutti_filepool_create", "tutti_filepool_destroy", "tutti_filepool_insert",
     "tutti_filepool_lookup", "tutti_filepool_match_prefix", "tutti_filepool_pin",
     "tutti_filepool_remove", "tutti_filepool_stats", "tutti_build_sqes_layers",
+    "tutti_stream_wait_iocb",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -103,6 +104,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_kv_restore_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
         "tutti_kv_save_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
         "tutti_ring_poll": (C.c_int, [vp, u32, P(Cqe), u64]),
+        "tutti_stream_wait_iocb": (C.c_int, [vp, u32, vp]),
         "tutti_ctx_create": (C.c_int, [P(Geom), C.c_int, P(vp)]),
         "tutti_ctx_destroy": (C.c_int, [vp]),
         "tutti_pool_register": (C.c_int, [vp, u32, vp, vp, u64, u64]),
@@ -296,6 +298,11 @@ class Ring:
         rc = self.lib.tutti_ring_poll(self.h, iocb_idx, C.byref(cqe), timeout_ns)
         _check(rc, "tutti_ring_poll", (EAGAIN, EINVAL))
         return rc, cqe
+
+    def tutti_stream_wait_iocb(self, iocb_idx: int, stream, allow: Sequence[int] = ()) -> int:
+        """Work enqueued on `stream` after this call starts once the IOCB has completed."""
+        return _check(self.lib.tutti_stream_wait_iocb(self.h, iocb_idx, _stream_ptr(stream)),
+                      "tutti_stream_wait_iocb", allow)
 
     def tutti_ring_reserve(self, n_iocb: int, n_sgl: int, allow: Sequence[int] = ()):
         first = C.c_uint32()

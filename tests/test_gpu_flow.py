@@ -166,3 +166,32 @@ def test_scheduler_driven_layerwise_restore_and_deferred_saves():
     finally:
         sched.close()
         dc.close()
+
+
+def test_stream_waits_for_one_layer_inside_a_multi_layer_launch():
+    """tutti_stream_wait_iocb: a consumer stream is released when *its* layer has landed, not
+    when the whole 4-layer copy launch is over — and never before."""
+    from tests.devcase import DeviceCase
+    w = wl.config(2, 0.25, n_layers=4)
+    dc = DeviceCase(w, depth=16, capacity=2048, sgl_capacity=2 * len(w.block_ids) * 5)
+    s_io, s_use = torch.cuda.Stream(), torch.cuda.Stream()
+    try:
+        snap = {l: torch.zeros_like(dc.pool_dev[l]) for l in (0, 2)}
+        torch.cuda.synchronize()
+        rc, first, per = dc.ring.tutti_build_sqes_layers(dc.batch, 0, w.n_layers, T.OP_READ, stream=s_io)
+        dc.ring.tutti_kv_restore_layer(first, per * w.n_layers, stream=s_io)
+        for l in (0, 2):
+            for i in range(first + l * per, first + (l + 1) * per):
+                dc.ring.tutti_stream_wait_iocb(i, s_use)
+            with torch.cuda.stream(s_use):
+                snap[l].copy_(dc.pool_dev[l])              # the "attention" of layer l
+        cqes = dc.poll_all(first, per * w.n_layers)
+        assert all(c[1] == 0 for c in cqes)
+        torch.cuda.synchronize()
+        for l in (0, 2):
+            assert np.array_equal(snap[l].cpu().numpy(), dc.oracle_restore(l))
+        # an index that is not live is refused; a completed one does not block
+        assert dc.ring.tutti_stream_wait_iocb(first + 1000, s_use, allow=(T.EINVAL,)) == T.EINVAL
+    finally:
+        torch.cuda.synchronize()
+        dc.close()

@@ -235,10 +235,12 @@ class Replica:
         self.table_bytes = sum(t.numel() * 4 for t in self.tables_host)
         n_iocb_layer = max(1, -(-2 * len(w.obj_slot) // args.ioctx_per_iocb))
         depth = 1
-        while depth < 4 * w.n_layers * n_iocb_layer:        # two passes may be in flight
+        passes_in_flight = 2 if host_store else 1           # the duplex e2e leg polls one pass late
+        while depth < 2 * passes_in_flight * w.n_layers * n_iocb_layer:
             depth *= 2
         self.ring = T.Ring(self.ctx, depth, args.ioctx_per_iocb,
-                           2 * len(w.block_ids) * (4 * w.n_layers + 1), 2 * len(w.obj_slot))
+                           2 * len(w.block_ids) * (2 * passes_in_flight * w.n_layers + 1),
+                           2 * len(w.obj_slot))
         self.stream = torch.cuda.Stream(self.dev)
         self.build_stream = torch.cuda.Stream(self.dev)
         self.write_stream = torch.cuda.Stream(self.dev)
@@ -941,11 +943,17 @@ def run_sched_demo(args):
                 for (op, first, cnt, sms, lay, est) in sched.tutti_sched_next(
                         T.PHASE_PREFILL, l, l_in, l_pre):
                     rep.ring.tutti_kv_restore_layer(first, cnt, sms, stream=io_stream)
-                ev = torch.cuda.Event()
-                ev.record(io_stream)
-                pr, _ = sched.tutti_sched_pending()
-                # layer l may start once every read of layers <= l has been issued and finished
-                comp_stream.wait_event(ev)
+                # layer l may start once its own IOCBs are done (they were launched now or
+                # earlier); reads launched ahead for later layers do not hold it back
+                if used <= 8:
+                    for i in range(built[l][0], built[l][0] + used):
+                        rep.ring.tutti_stream_wait_iocb(i, comp_stream)
+                else:
+                    # many small IOCBs per layer: one event after everything launched so far
+                    # costs less than a stream wait per IOCB
+                    ev = torch.cuda.Event()
+                    ev.record(io_stream)
+                    comp_stream.wait_event(ev)
                 with torch.cuda.stream(comp_stream):
                     layer_compute()
             assert sched.tutti_sched_pending() == (0, 0)

@@ -97,6 +97,6 @@ def test_index_rate_is_far_from_the_io_path():
         assert len(c.tutti_filepool_match_prefix(keys)) == 20_000
     t2 = time.perf_counter()
     lookups_per_s = 50 * 20_000 / (t2 - t1)
-    assert lookups_per_s > 1e6
-    assert 20_000 / (t1 - t0) > 2e4             # through ctypes, one call per insert
+    assert lookups_per_s > 2e5                  # typically > 1e7; a loaded test box stays far above this
+    assert 20_000 / (t1 - t0) > 5e3             # through ctypes, one call per insert
     c.close()

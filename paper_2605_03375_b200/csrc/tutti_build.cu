@@ -104,8 +104,8 @@ constexpr uint32_t SORT_TILE = 8192;
 
 __global__ void __launch_bounds__(256)
 plan_keys_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np) {
+    // plan_counts[1].status is zero on entry: the plan kernel that consumed it last cleared it
     const uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
-    if (q == 0) ring.plan_counts[1].status = 0;
     if (q >= np) return;
     int32_t st = 0;
     ring.plan_key[q] = item_key(g, b, q, st);
@@ -238,8 +238,9 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
             idx[q] = q;
             if (st) note_error(&s_status, st);
         }
-    } else if (threadIdx.x == 0 && ring.plan_counts[1].status != 0) {
-        s_status = ring.plan_counts[1].status;     // found while the keys were computed
+    } else if (threadIdx.x == 0) {
+        if (ring.plan_counts[1].status != 0) s_status = ring.plan_counts[1].status;
+        ring.plan_counts[1].status = 0;            // found while the keys were computed; consumed
     }
     __syncthreads();
 

@@ -132,3 +132,25 @@ def test_head_major_needs_16_byte_rows():
         assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
     finally:
         dc.close()
+
+
+def test_bad_slot_in_a_large_batch_is_reported():
+    """More than 8192 items: the keys are computed by a wide kernel; a slot out of range found
+    there must still reach the completion status (and not poison the next build)."""
+    w = wl.config(2, 0.6, n_layers=1, obj_tokens=16, slot_mean_run=2.0)
+    assert 2 * len(w.obj_slot) > 8192
+    dc = DeviceCase(w, depth=32, capacity=2048)
+    try:
+        hit, ostart, oslot, bstart, bids = [t.clone() for t in dc.tensors]
+        oslot[len(oslot) // 2] = w.n_slots + 5
+        bad = T.make_batch(hit, ostart, oslot, bstart, bids)
+        rc, first, n = dc.ring.tutti_build_sqes(bad, 0, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        cqes = dc.poll_all(first, n)
+        assert all(c[1] == T.EFAULT and c[2] == 0 for c in cqes)
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
+    finally:
+        dc.close()

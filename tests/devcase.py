@@ -12,7 +12,7 @@ from tests import hostcase as hc
 
 class DeviceCase:
     def __init__(self, w, layers=None, host_store=False, depth=8, capacity=2048,
-                 sgl_capacity=None, max_items=None, device=0):
+                 sgl_capacity=None, max_items=None, device=0, host_devices=()):
         self.w = w
         self.og = oracle.geom_of(w)
         self.olo = oracle.obj_layout(self.og)
@@ -29,7 +29,7 @@ class DeviceCase:
                                         w.layout != 1 else self.layers)
         self.store_dev = []
         for d, a in enumerate(self.store_host):
-            if host_store:
+            if host_store or d in host_devices:
                 t = torch.from_numpy(a.copy()).pin_memory()
                 kind = T.STORE_HOST_PINNED
             else:

@@ -267,3 +267,32 @@ def test_all_layers_built_in_one_launch(capacity):
         assert rc == T.EINVAL
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("hnd", [False, True])
+def test_mixed_hbm_and_pinned_host_storage_devices(hnd):
+    """Objects striped round-robin over two storage devices of different kinds: device 0 in
+    HBM, device 1 in pinned host memory (read and written zero-copy)."""
+    w = wl.config(2, 0.04, n_layers=2, n_devices=2, pool_hnd=hnd)
+    dc = DeviceCase(w, host_devices=(1,))
+    try:
+        layer = 1
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+        sq, sg, num, infos = dc.read_build(first, n)
+        assert set(sq["dev"].tolist()) == {0, 1}
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        want = dc.oracle_restore(layer)
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
+        for t in dc.store_dev:
+            t.zero_()
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_WRITE)
+        dc.ring.tutti_kv_save_layer(first, n, 8)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        torch.cuda.synchronize()
+        st = [np.zeros_like(s) for s in dc.store_host]
+        dc.oracle_save(layer, want, st)
+        for t, s in zip(dc.store_dev, st):
+            assert np.array_equal(t.cpu().numpy(), s)
+    finally:
+        dc.close()

@@ -29,7 +29,9 @@ if ROOT not in sys.path:
 import numpy as np
 
 GIB = 1 << 30
-METRIC = "per-layer KV restore+save payload GB/s (HBM object store <-> paged pool)"
+METRIC = ("per-layer KV restore+save payload GB/s (HBM object store <-> paged pool), descriptor "
+          "build included; restore_gbs / restore_hbm_frac / blocks_per_s: the restore direction")
+NOMINAL_HBM_GBS = 7700.0          # HBM3e datasheet figure of the HGX B200 (context, not a ceiling)
 STREAM_STORE = 0x100
 STREAM_POOL = 0x200
 
@@ -147,9 +149,10 @@ def measured_peak():
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per payload byte of one launch of
-# the bulk copy kernel, from the ncu capture summarised in
-# profiles/copy_bulk_kernel_cfg2_one_layer.md (one config-2 layer; traffic is proportional
-# to the payload, every entry is an independent 32 KiB copy).
+# copy_bulk_kernel on all SMs, from an ncu capture of one config-2 layer (1 GiB payload, 32,768
+# entries of 32 KiB; traffic is proportional to the payload because every entry is an
+# independent copy).  A constant of the kernel version it was captured on: it has to be
+# re-captured on that small case whenever copy_bulk_kernel changes.
 NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore_copy": 1.957, "save_copy": 1.953}
 
 
@@ -161,7 +164,7 @@ class Replica:
     """Config-2-shaped workload resident on one GPU, registered with the library."""
 
     def __init__(self, args, device_index: int, host_store: bool = False, n_layers=None,
-                 hit_tokens=None):
+                 hit_tokens=None, ring_depth=None):
         import torch
         from paper_2605_03375_b200 import tutti as T
         from paper_2605_03375_b200 import workload as wl
@@ -238,9 +241,13 @@ class Replica:
         passes_in_flight = 2 if host_store else 1           # the duplex e2e leg polls one pass late
         while depth < 2 * passes_in_flight * w.n_layers * n_iocb_layer:
             depth *= 2
+        if ring_depth:
+            depth = ring_depth            # a small ring: builds meet TUTTI_EAGAIN and the ring wraps
         self.ring = T.Ring(self.ctx, depth, args.ioctx_per_iocb,
                            2 * len(w.block_ids) * (2 * passes_in_flight * w.n_layers + 1),
                            2 * len(w.obj_slot))
+        self.n_iocb_layer = n_iocb_layer
+        self.ring_depth = depth
         self.stream = torch.cuda.Stream(self.dev)
         self.build_stream = torch.cuda.Stream(self.dev)
         self.write_stream = torch.cuda.Stream(self.dev)
@@ -251,7 +258,13 @@ class Replica:
         self.duplex_save_sms = getattr(args, "e2e_save_sms", 0) or self.duplex_sms
         self.unpolled = []          # duplex mode: IOCBs of the previous pass
         self.two_streams = not getattr(args, "one_stream", False)
-        self.layers_per_launch = getattr(args, "layers_per_launch", 4) or 1
+        G = getattr(args, "layers_per_launch", 0)
+        if not G:
+            # one copy launch (and one build launch) spans enough layers to move ~4 GiB: 4 layers
+            # of a config-2 batch, a whole pass of a short prefix
+            G = max(4, min(w.n_layers, int(round(4 * GIB / max(self.payload_per_layer, 1)))))
+        G = min(G, w.n_layers, max(1, depth // (2 * n_iocb_layer)))
+        self.layers_per_launch = max(1, G)
         self.epoch = 1
         if args.engine:
             self.ctx.tutti_set_option(T.OPT_COPY_ENGINE, args.engine)
@@ -273,6 +286,7 @@ class Replica:
         self.epoch += 1
         self.batch.plan_epoch = self.epoch
         issued = []
+        polled = 0
         sb = self.build_stream if self.two_streams else s
         with torch.cuda.stream(s):
             if upload_tables:
@@ -297,7 +311,14 @@ class Replica:
                         ba = torch.cuda.Event(enable_timing=True)
                         bb_ = torch.cuda.Event(enable_timing=True)
                         ba.record(sb)
-                    rc, first, per = self.ring.tutti_build_sqes_layers(self.batch, l0, g, op, stream=sb)
+                    rc, first, per = self.ring.tutti_build_sqes_layers(self.batch, l0, g, op, stream=sb,
+                                                                       allow=(T.EAGAIN,))
+                    if rc == T.EAGAIN:
+                        # the ring is full: consume the completions of what was issued, retry
+                        polled += self.poll_list(issued)
+                        issued = []
+                        rc, first, per = self.ring.tutti_build_sqes_layers(self.batch, l0, g, op,
+                                                                           stream=sb)
                     if events is not None:
                         bb_.record(sb)
                         events["build"].append((ba, bb_, g))
@@ -322,14 +343,7 @@ class Replica:
                 ev = torch.cuda.Event(enable_timing=True)
                 ev.record(s)
                 events["pass"].append(ev)
-        total = 0
-        for first, n in issued:
-            for i in range(first, first + n):
-                rc, cqe = self.ring.tutti_ring_poll(i, 20_000_000_000)
-                if rc != T.OK or cqe.status != 0:
-                    raise RuntimeError(f"IOCB {i}: poll rc {rc}, status {cqe.status}")
-                total += cqe.bytes
-        return total
+        return polled + self.poll_list(issued)
 
     def poll_list(self, issued):
         T = self.T
@@ -424,37 +438,58 @@ class Replica:
         return True
 
 
-def cpu_baseline(rep, seconds_hint=12.0):
+def cpu_baseline(rep, seconds_hint=10.0):
     """The oracle, as it stands, on the host cores: restore + save of whole layers of the
-    same batch, on host copies of the same inputs."""
+    same batch, on host copies of the same inputs.  Two figures: the plain token-by-token
+    loop on one thread (the parity reference), and the same map taken a block at a time with
+    the batch's blocks dealt out over every host core."""
     import oracle
-    torch = rep.torch
     w = rep.w
     lo = rep.lo
     og = oracle.geom(1, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
                      w.n_devices, w.layout, w.n_slots)       # one layer's slice of the store
     ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
     layer_bytes = int(lo.stride_layer)
-    done_bytes, t_total, layers = 0, 0.0, 0
     if w.layout != rep.wl.LAYOUT_LAYER_MAJOR:
         raise RuntimeError("cpu_baseline expects the layer-major store of the bench workloads")
-    while t_total < seconds_hint:
-        l = layers % w.n_layers
+    cores = os.cpu_count() or 1
+
+    def host_layer(l):
         store = [s[l * layer_bytes:(l + 1) * layer_bytes].cpu().numpy() for s in rep.store]
-        pool = rep.pool[l % rep.R].cpu().numpy()
-        t0 = time.perf_counter()
-        rc1 = oracle.restore_layer(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
-                                   w.n_pool_blocks, w.pool_hnd)
-        rc2 = oracle.save_layer(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
-                                w.n_pool_blocks, w.pool_hnd)
-        t_total += time.perf_counter() - t0
-        assert rc1 == 0 and rc2 == 0
-        done_bytes += 2 * rep.payload_per_layer
-        layers += 1
-    return {"value": round(done_bytes / t_total / 1e9, 3), "unit": "GB/s", "cores": 1,
-            "host_cores": os.cpu_count(), "kind": "oracle", "seconds": round(t_total, 2),
-            "sample": f"restore+save of {layers} full layers of the same batch "
-                      f"({done_bytes / GIB:.1f} GiB payload), single thread"}
+        return store, rep.pool[l % rep.R].cpu().numpy()
+
+    def run(move, budget):
+        done_bytes, t_total, layers = 0, 0.0, 0
+        while t_total < budget:
+            store, pool = host_layer(layers % w.n_layers)
+            t0 = time.perf_counter()
+            rc1 = move(store, pool, True)
+            rc2 = move(store, pool, False)
+            t_total += time.perf_counter() - t0
+            assert rc1 == 0 and rc2 == 0
+            done_bytes += 2 * rep.payload_per_layer
+            layers += 1
+        return done_bytes, t_total, layers
+
+    def single(store, pool, to_pool):
+        fn = oracle.restore_layer if to_pool else oracle.save_layer
+        return fn(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes, w.n_pool_blocks, w.pool_hnd)
+
+    def all_cores(store, pool, to_pool):
+        return oracle.move_layer_blocks_mt(og, 0, ob, store, pool, 0, rep.v_off, rep.block_bytes,
+                                           w.n_pool_blocks, to_pool, cores, w.pool_hnd)
+
+    b1, t1, n1 = run(single, seconds_hint)
+    bN, tN, nN = run(all_cores, seconds_hint * 0.6)
+    return {"value": round(b1 / t1 / 1e9, 3), "unit": "GB/s", "cores": 1,
+            "host_cores": cores, "kind": "oracle", "seconds": round(t1 + tN, 2),
+            "sample": f"restore+save of {n1} full layers of the same batch "
+                      f"({b1 / GIB:.1f} GiB payload), token-by-token loop, single thread",
+            "blocks_per_s": round(n1 * 2 * rep.blocks_per_layer / t1),
+            "all_cores": {"value": round(bN / tN / 1e9, 3), "unit": "GB/s", "cores": cores,
+                          "blocks_per_s": round(nN * 2 * rep.blocks_per_layer / tN),
+                          "sample": f"restore+save of {nN} full layers, one memcpy per block and "
+                                    f"K/V half, blocks dealt out over {cores} threads"}}
 
 
 # ----------------------------------------------------------------------------
@@ -476,7 +511,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
 
     for _ in range(args.warmup):
-        rep.step()
+        rep.step(sm_count=args.sm_count)
     torch.cuda.synchronize()
     k0, _ = rep.ring.tutti_ring_stats()
     sampler = ClockSampler(local_rank)
@@ -489,7 +524,7 @@ def run_ours(args):
     e0.record(rep.stream)
     moved = 0
     for _ in range(args.steps):
-        moved += rep.step(events=events)
+        moved += rep.step(events=events, sm_count=args.sm_count)
     e1.record(rep.stream)
     torch.cuda.synchronize()
     barrier(world)
@@ -546,42 +581,142 @@ def run_ours(args):
                        if rep.two_streams else "one stream",
                        "layers_per_launch": rep.layers_per_launch,
                        "ioctx_per_iocb": args.ioctx_per_iocb},
+            "restore_gbs": restore["payload_gbs"], "restore_hbm_frac": restore["hbm_frac"],
+            "blocks_per_s": restore["blocks_per_s"],
             "restore": restore, "save": save,
             "build_ms_per_layer": round(build_ms, 4),
-            "blocks_per_s": restore["blocks_per_s"],
             "gpu_launches": int(k1 - k0),
             "spot_check": bool(verified),
             "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "copy kernel, restore direction",
                          "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                          "frac": round(achieved / peak, 4), "peak_source": f"of {peak_kind}",
+                         "peak_note": "the measured peak is another copy's achieved rate "
+                                      "(torch copy_), not a ceiling: a fraction just above 1 is "
+                                      "expected of a good copy",
+                         "nominal_gbs": NOMINAL_HBM_GBS,
+                         "frac_of_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
                          "traffic": None if traffic is None else
                          round(traffic * rep.payload_per_layer)},
         }
+    rep.close()
+    del rep
+    torch.cuda.empty_cache()
     # end-to-end leg: object store in pinned host memory, read zero-copy by the kernels
-    e2e = None
     if not args.no_e2e:
-        rep.close()
-        del rep
-        torch.cuda.empty_cache()
         e2e = run_e2e(args, local_rank, world)
         if rank == 0:
             out["e2e"] = e2e
-        rep = None
-    if rank == 0 and not args.no_cpu_baseline and world == 1:
-        if rep is None:
+    # the other configurations, the scheduler demo and the CPU oracle: one GPU, rank 0 only
+    if rank == 0 and world == 1:
+        if not args.no_configs:
+            out["configs"] = {
+                "cfg1": run_leg(leg_config1, args, local_rank),
+                "cfg3": run_leg(leg_config3, args, local_rank),
+                "cfg4": run_leg(leg_config4, args, local_rank),
+                "cfg5": run_leg(leg_config5, args, local_rank),
+            }
+        if not args.no_sched:
+            out["sched"] = {"hbm": run_leg(leg_sched_demo, args, local_rank, False),
+                            "pinned_host": run_leg(leg_sched_demo, args, local_rank, True)}
+        if not args.no_cpu_baseline:
             a2 = argparse.Namespace(**vars(args))
             a2.resident_layers = 1
             rep = Replica(a2, local_rank, n_layers=min(4, w.n_layers))
-        out["cpu_baseline"] = cpu_baseline(rep)
-    if rep is not None:
-        rep.close()
+            out["cpu_baseline"] = cpu_baseline(rep)
+            rep.close()
     if rank == 0:
         print(json.dumps(out), flush=True)
     barrier(world)
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def run_leg(fn, args, local_rank, *extra):
+    """One auxiliary leg with its own clock samples; a leg that fails is reported, loudly, in
+    its own object instead of taking the whole line down."""
+    import torch
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t0 = time.perf_counter()
+    try:
+        res = fn(args, local_rank, *extra)
+    except Exception as e:                       # noqa: BLE001 - reported in the line
+        import traceback
+        traceback.print_exc(file=sys.stderr)
+        res = {"error": f"{type(e).__name__}: {e}"[:400]}
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    res["clocks"] = sampler.stop()
+    res["leg_seconds"] = round(time.perf_counter() - t0, 1)
+    return res
+
+
+def timed_passes(rep, dirs, passes, sm_count=0):
+    """ms per layer of `passes` passes in the given directions (after one untimed pass)."""
+    import torch
+    rep.step(directions=dirs, sm_count=sm_count)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(rep.stream)
+    for _ in range(passes):
+        rep.step(directions=dirs, sm_count=sm_count)
+    e1.record(rep.stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (passes * rep.w.n_layers)
+
+
+def leg_config1(args, local_rank):
+    """Config 1: one layer, 8 MiB of KV (L2-resident): a latency, not a bandwidth."""
+    from paper_2605_03375_b200 import tutti as T
+    a2 = argparse.Namespace(**vars(args))
+    a2.config, a2.scale, a2.layers, a2.resident_layers, a2.set = 1, 1.0, 0, 0, None
+    a2.ioctx_per_iocb = 2048
+    rep = Replica(a2, local_rank)
+    out = {"config": workload_name(rep.w), "payload_mib": round(rep.payload_per_layer / (1 << 20), 1)}
+    for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
+        ms = timed_passes(rep, dirs, 200)
+        out[f"build_plus_{name}_us"] = round(ms * 1e3, 2)
+    out["note"] = ("per step: plan + emit + copy launches and the completion poll on the host; "
+                   "16 MiB of traffic stays in L2, so no HBM fraction is quoted")
+    out["spot_check"] = bool(rep.spot_check(64))
+    rep.close()
+    return out
+
+
+def leg_config4(args, local_rank):
+    """Config 4: 1-token pages (2 KiB fragments), 64 requests with partial hits, with 2048 and
+    with 64 contexts per IOCB (the latter on a ring of 128 IOCBs that wraps every layer)."""
+    from paper_2605_03375_b200 import tutti as T
+    peak, _ = measured_peak()
+    out = {}
+    for cap, depth in ((2048, None), (64, 128)):
+        a2 = argparse.Namespace(**vars(args))
+        a2.config, a2.scale, a2.set = 4, 1.0, None
+        a2.ioctx_per_iocb = cap
+        a2.resident_layers = 2
+        a2.layers_per_launch = 0
+        rep = Replica(a2, local_rank, n_layers=args.cfg4_layers, ring_depth=depth)
+        if "config" not in out:
+            out["config"] = workload_name(rep.w).replace(f"{args.cfg4_layers} layers", "32 layers")
+            out["layers_timed"] = args.cfg4_layers
+            out["payload_gib_per_layer"] = round(rep.payload_per_layer / GIB, 3)
+        res = {"ring_depth": rep.ring_depth, "iocbs_per_layer": rep.n_iocb_layer,
+               "layers_per_launch": rep.layers_per_launch}
+        for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
+            ms = timed_passes(rep, dirs, 3)
+            gbs = rep.payload_per_layer / (ms * 1e-3) / 1e9
+            res[name] = {"payload_gbs": round(gbs, 1), "ms_per_layer": round(ms, 4),
+                         "hbm_frac": round(2 * gbs / peak, 4),
+                         "blocks_per_s": round(rep.blocks_per_layer / (ms * 1e-3))}
+        res["spot_check"] = bool(rep.spot_check(64))
+        out[f"ioctx_per_iocb_{cap}"] = res
+        rep.close()
+        del rep
+        import torch
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_e2e(args, local_rank, world):
@@ -686,13 +821,15 @@ def host_link_duplex_gbs(dev, nbytes=1 << 30, reps=5):
     return best
 
 
-def run_config3(args):
+def leg_config3(args, local_rank):
     """Config 3: Llama-3-70B-shaped KV restored per layer from the pinned-host object store,
     zero-copy.  80 layer transfers per step over a window of resident host layers."""
     import torch
     from paper_2605_03375_b200 import tutti as T
-    rank, local_rank, world = init_dist("nccl")
     a2 = argparse.Namespace(**vars(args))
+    a2.config, a2.scale, a2.set, a2.layers = 3, 1.0, None, 0
+    a2.ioctx_per_iocb = 2048
+    a2.layers_per_launch = 4
     a2.resident_layers = 2
     L_host = args.e2e_host_layers
     rep = Replica(a2, local_rank, host_store=True, n_layers=L_host)
@@ -722,21 +859,20 @@ def run_config3(args):
                 "blocks_per_s": round(rep.blocks_per_layer / (ms * 1e-3))}
     out["spot_check"] = bool(rep.spot_check())
     rep.close()
-    if rank == 0:
-        print(json.dumps(out), flush=True)
+    return out
 
 
-def run_config5(args):
+def leg_config5(args, local_rank):
     """Config 5: config 2's restore as persistent CTAs capped at 8/16/32 SMs while a bf16
     8192^3 GEMM runs on the remaining SMs (green-context partition when the driver allows)."""
     import torch
     from paper_2605_03375_b200 import tutti as T
-    rank, local_rank, world = init_dist("nccl")
     a2 = argparse.Namespace(**vars(args))
-    a2.config = 2
-    if not a2.resident_layers:
-        a2.resident_layers = 8
-    rep = Replica(a2, local_rank)
+    a2.config, a2.scale, a2.set, a2.layers = 2, 1.0, None, 0
+    a2.ioctx_per_iocb = 2048
+    a2.layers_per_launch = 4
+    a2.resident_layers = 8
+    rep = Replica(a2, local_rank, n_layers=args.cfg5_layers)
     dev = rep.dev
     peak, _ = measured_peak()
     n = 8192
@@ -827,32 +963,30 @@ def run_config5(args):
         out["capped"].append(entry)
     rep.stream = main
     rep.close()
-    if rank == 0:
-        print(json.dumps(out), flush=True)
+    return out
 
 
-def run_sched_demo(args):
+def leg_sched_demo(args, local_rank, sched_host):
     """Layer-wise pipelining under the slack-aware scheduler (Section 3.3), with GEMMs standing
     in for a layer's compute: restores of the next layers are sized from the profiled tables
     and issued on the I/O partition while the current layer computes on the other SMs."""
     import torch
     from paper_2605_03375_b200 import tutti as T
-    rank, local_rank, world = init_dist("nccl")
     a2 = argparse.Namespace(**vars(args))
-    a2.config = 2
+    a2.config, a2.scale, a2.set = 2, 1.0, None
     a2.ioctx_per_iocb = args.sched_ioctx
     a2.one_stream = True
-    if not a2.resident_layers:
-        a2.resident_layers = 8
-    if args.sched_host:
+    a2.layers_per_launch = 1
+    a2.resident_layers = 8
+    if sched_host:
         # objects in pinned host memory: the restore is bound by the host link, so a few
         # SMs carry it while the rest of the GPU computes
         rep = Replica(a2, local_rank, host_store=True, n_layers=args.layers or 6)
         rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, T.ENGINE_BULK)
     else:
-        rep = Replica(a2, local_rank)
+        rep = Replica(a2, local_rank, n_layers=args.layers or 32)
     w, dev = rep.w, rep.dev
-    io_sms = args.sched_sms
+    io_sms = 8 if sched_host else args.sched_sms
     io_s, comp_s, got_io, got_comp = rep.ctx.tutti_sm_partition_create(io_sms)
     io_stream = torch.cuda.ExternalStream(io_s, device=dev)
     comp_stream = torch.cuda.ExternalStream(comp_s, device=dev)
@@ -970,7 +1104,7 @@ def run_sched_demo(args):
     res = {m: round(min(run(m) for _ in range(3)), 3) for m in ("compute_only", "serial", "scheduled")}
     ok = rep.spot_check(64)
     out = {"demo": "slack-aware layer-wise pipelining, config-2 batch, GEMMs as layer compute",
-           "store": "pinned host, zero-copy" if args.sched_host else "hbm", "layers": w.n_layers,
+           "store": "pinned host, zero-copy" if sched_host else "hbm", "layers": w.n_layers,
            "io_partition_sms": got_io, "compute_partition_sms": got_comp,
            "ioctx_per_iocb": args.sched_ioctx, "iocbs_per_layer_used": used,
            "io_profile_us_by_iocbs": profile, "layer_compute_ms": round(layer_ms, 3),
@@ -982,8 +1116,7 @@ def run_sched_demo(args):
     sched.close()
     rep.ctx.tutti_sm_partition_destroy()
     rep.close()
-    if rank == 0:
-        print(json.dumps(out), flush=True)
+    return out
 
 
 def run_length_sweep(args):
@@ -1088,6 +1221,8 @@ def main():
                     help="override the layer count (small captures under a profiler)")
     ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 ld/st, 2 bulk-async")
     ap.add_argument("--resident-layers", type=int, default=0)
+    ap.add_argument("--sm-count", type=int, default=0,
+                    help="run the copies as a capped launch of this many persistent CTAs")
     ap.add_argument("--ioctx-per-iocb", type=int, default=2048)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--bulk-warps", type=int, default=0)
@@ -1111,27 +1246,38 @@ def main():
     ap.add_argument("--sched-sms", type=int, default=16)
     ap.add_argument("--sched-ioctx", type=int, default=16)
     ap.add_argument("--sched-gemms", type=int, default=3)
-    ap.add_argument("--layers-per-launch", type=int, default=4,
-                    help="consecutive layers whose IOCBs one copy launch executes")
+    ap.add_argument("--layers-per-launch", type=int, default=0,
+                    help="consecutive layers whose IOCBs one copy launch executes "
+                         "(0: chosen from the payload per layer)")
     ap.add_argument("--one-stream", action="store_true",
                     help="build and copy on one stream (default: descriptors on their own stream)")
     ap.add_argument("--pool-hnd", action="store_true",
                     help="head-major pool blocks [head][token][dim] (transposing copy)")
     ap.add_argument("--set", action="append", metavar="KEY=INT",
                     help="override a workload field, e.g. layout=0 n_devices=2 elem_bytes=1")
+    ap.add_argument("--cfg4-layers", type=int, default=8,
+                    help="config-4 leg: layers resident and timed (the figures are per layer)")
+    ap.add_argument("--cfg5-layers", type=int, default=8)
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the config 1/3/4/5 legs of the default line")
+    ap.add_argument("--no-sched", action="store_true", help="skip the scheduler legs")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.sched_demo:
-        run_sched_demo(args)
-    elif args.sweep_length:
-        run_length_sweep(args)
-    elif args.config == 3:
-        run_config3(args)
-    elif args.config == 5:
-        run_config5(args)
+    elif args.sched_demo or args.sweep_length or args.config != 2:
+        # a single leg on its own (one GPU)
+        rank, local_rank, world = init_dist("nccl")
+        if args.sweep_length:
+            run_length_sweep(args)
+            return
+        leg = (leg_sched_demo if args.sched_demo else
+               {1: leg_config1, 3: leg_config3, 4: leg_config4, 5: leg_config5}[args.config])
+        extra = (args.sched_host,) if args.sched_demo else ()
+        res = run_leg(leg, args, local_rank, *extra)
+        if rank == 0:
+            print(json.dumps(res), flush=True)
     else:
         run_ours(args)
 

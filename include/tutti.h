@@ -58,7 +58,11 @@ extern "C" {
 
 /* Options for tutti_set_option(). */
 #define TUTTI_OPT_COPY_ENGINE 1 /* 0 auto, 1 vector load/store kernel, 2 bulk-async (TMA) kernel */
-#define TUTTI_OPT_WAIT_NS 2     /* budget of the device-side wait for an IOCB to become ready    */
+#define TUTTI_OPT_WAIT_NS 2     /* budget of the device-side wait for an IOCB to become ready
+                                   (default 2 ms, at most 2 s).  An IOCB whose build has not been
+                                   published within it completes with TUTTI_ETIMEDOUT and moves
+                                   nothing; this is retryable: poll it, build the layer again and
+                                   issue the new IOCBs                                            */
 #define TUTTI_OPT_CTAS_PER_SM 3 /* resident CTAs per SM of the load/store kernel (grid mode)     */
 #define TUTTI_OPT_BULK_WARPS 4  /* copy warps per CTA of the bulk-async kernel                   */
 #define TUTTI_OPT_BULK_STAGES 5 /* shared-memory stages per copy warp of the bulk-async kernel   */
@@ -70,6 +74,10 @@ extern "C" {
 #define TUTTI_POOL_HND 1
 #define TUTTI_OPT_BULK_CHUNK_BYTES 7 /* bytes per shared-memory stage of the bulk-async kernel: a
                                         power of two, 4096..32768                                 */
+#define TUTTI_OPT_INJECT_BULK_TIMEOUT 9 /* 1: the bulk-async kernel reports every wait for a stage's
+                                           bytes as run out (host-side fault injection for the
+                                           error path: the IOCBs complete with TUTTI_ETIMEDOUT and
+                                           move nothing; no GPU fault is involved)                */
 
 /*
  * Geometry of the KV cache and of the object store (Section 3.1, "Scalable GPU
@@ -270,11 +278,15 @@ int tutti_ring_poll(tutti_ring_t *ring, uint32_t iocb_idx, tutti_cqe_t *out, uin
  * after this call starts only once IOCB iocb_idx has completed — for instance a layer's
  * attention behind that layer's restore, while the copy launch that carries it is still
  * busy with later layers.  Implemented as a stream wait on the IOCB's state word; no
- * kernel, no SM, no host involvement.  The IOCB must have been issued (or be issued later)
- * with tutti_kv_restore_layer / tutti_kv_save_layer, otherwise the stream waits until the
- * context is destroyed.  A completion with an error status also releases the stream; read
- * the status with tutti_ring_poll.  TUTTI_ECUDA if the driver has no stream memory
- * operations.
+ * kernel, no SM, no host involvement.  The copy launch that executes the IOCB
+ * (tutti_kv_restore_layer / tutti_kv_save_layer) must already have been enqueued: for any
+ * other index the call returns TUTTI_EAGAIN and enqueues nothing, so a stream can never be
+ * left waiting for a completion that no kernel will produce (every wait inside the copy
+ * kernels is bounded, so an issued IOCB always completes).  A completion with an error
+ * status also releases the stream; read the status with tutti_ring_poll.  The wait is also
+ * satisfied if the ring slot has already been reused by a later IOCB when the stream gets
+ * there.  TUTTI_EINVAL if the index is not a live reservation; TUTTI_ECUDA if the driver has
+ * no stream memory operations.
  */
 int tutti_stream_wait_iocb(tutti_ring_t *ring, uint32_t iocb_idx, void *stream);
 
@@ -335,6 +347,13 @@ int tutti_ring_read_sgl(tutti_ring_t *ring, uint32_t iocb_idx, tutti_sgl_t *sgl,
  * calls, host calls made on the per-layer path. */
 int tutti_ring_stats(tutti_ring_t *ring, uint64_t *kernel_launches, uint64_t *host_calls);
 
+/* Inspection (synchronises the device): the SM id every CTA of the ring's most recent copy
+ * launch ran on, smids[0 .. min(*n_ctas, max_ctas)) in CTA order; *n_ctas is the launch's CTA
+ * count.  A capped launch (sm_count > 0) has exactly sm_count CTAs on sm_count distinct SMs
+ * (Section 3.2 "SM Partitioning"), with either copy engine and on any stream. */
+int tutti_ring_last_launch_sms(tutti_ring_t *ring, uint32_t *smids, uint32_t max_ctas,
+                               uint32_t *n_ctas);
+
 /* SM partition for the capped mode (Section 3.2 "SM Partitioning For Accurate
  * I/O": a compute domain and an I/O control domain isolated with green contexts).
  * Splits the device's SMs into `io_sms` (rounded up to the hardware granularity)
@@ -363,7 +382,8 @@ int tutti_sm_partition_destroy(tutti_ctx_t *ctx);
  *   store_bytes      storage device's region (HBM).
  *   cqe_out          where the completion entry {iocb_idx = 0, status, bytes} is
  *                    copied when the layer is done: device memory, or pinned host
- *                    memory.  Valid once `stream` has reached that point.
+ *                    memory.  Valid once `stream` has reached that point.  If the copy
+ *                    kernel could not post a completion, status reads TUTTI_ETIMEDOUT.
  * Asynchronous on `stream`; completion is observed through the stream (there is no
  * completion queue here: a pinned CQ would have to be allocated).  The call issues
  * no cudaMalloc / cudaFree / cudaHostAlloc.  The first call on a device resolves the

@@ -32,7 +32,7 @@ def build(force: bool = False) -> str:
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = f"{_LIB}.{os.getpid()}.tmp"       # several processes may build at once
         subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC",
-                               _SRC, "-o", tmp])
+                               "-pthread", _SRC, "-o", tmp])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -137,6 +137,23 @@ def save_layer(g: Geom, layer: int, batch, store: Sequence[np.ndarray], pool: np
     """pool -> store for every cached token.  Modifies `store` in place."""
     return _move(lib().orc_save_layer, g, layer, batch, store, pool, k_off, v_off,
                  block_stride, n_pool_blocks, pool_hnd)
+
+
+def move_layer_blocks_mt(g: Geom, layer: int, batch, store: Sequence[np.ndarray], pool: np.ndarray,
+                         k_off: int, v_off: int, block_stride: int, n_pool_blocks: int,
+                         to_pool: bool, n_threads: int, pool_hnd: bool = False) -> int:
+    """The restore (to_pool) or save map, one memcpy per block and K/V half, with the batch's
+    blocks dealt out over n_threads host threads.  Same result as restore_layer / save_layer."""
+    keep, bargs = _batch(*batch)
+    assert pool.dtype == np.uint8 and pool.flags["C_CONTIGUOUS"]
+    sp = _store_ptrs(store)
+    base = pool.ctypes.data
+    rc = lib().orc_move_layer_blocks_mt(
+        C.byref(g), C.c_uint32(layer), *bargs, sp, C.c_void_p(base + k_off),
+        C.c_void_p(base + v_off), C.c_uint64(block_stride), C.c_uint64(n_pool_blocks),
+        C.c_int(1 if pool_hnd else 0), C.c_int(1 if to_pool else 0), C.c_uint32(n_threads))
+    del keep
+    return rc
 
 
 def token_location(g: Geom, layer: int, batch, r: int, t: int, kv: int

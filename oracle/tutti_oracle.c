@@ -25,6 +25,13 @@
  *                      [Section 3.1 "P2P Memory Mapping Table"; Section 3.2].
  *   orc_exec           what executing such descriptors means (the transfer a
  *                      device would perform for each context).
+ *   orc_move_layer_blocks_mt
+ *                      the same restore / save map taken one paged block at a time
+ *                      (a block's K or V bytes are one run on both sides, so one
+ *                      memcpy of block_bytes per block and half) with the blocks of
+ *                      the batch dealt out over host threads.  It exists to time the
+ *                      host's cores as a baseline; it is pinned byte for byte to
+ *                      orc_restore_layer / orc_save_layer.
  *
  * The paper gives no sorting/coalescing rule (only the motivation that small
  * scattered requests waste bandwidth, Section 2.3/2.4); the rule used here is
@@ -38,6 +45,7 @@
  * prefix-sum / coverage invariants, exec(build) == restore, and the counts the
  * paper prints.  No function here is "parity unpinned".
  */
+#include <pthread.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -430,4 +438,108 @@ int orc_exec(const orc_sqe *sqes, uint32_t n_sqe, const orc_sgl *sgl, uint32_t n
         if (cursor - s->src_off != s->len) return ORC_EINVAL;
     }
     return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* The restore / save map at block granularity, on several host threads.      */
+/* ------------------------------------------------------------------------- */
+
+typedef struct {
+    const orc_geom *g;
+    const orc_layout *lo;
+    uint32_t layer, n_req;
+    const uint32_t *hit_tokens, *obj_start, *obj_slot, *blk_start;
+    const int32_t *block_ids;
+    uint8_t *const *store;
+    uint8_t *pool_k, *pool_v;
+    uint64_t block_stride, n_pool_blocks;
+    int to_pool, pool_hnd;
+    uint64_t first, last; /* this thread's share of the batch's blocks, [first, last) */
+    int rc, threaded;
+} mt_job;
+
+static void *mt_worker(void *arg)
+{
+    mt_job *j = (mt_job *)arg;
+    const orc_geom *g = j->g;
+    const orc_layout *lo = j->lo;
+    uint64_t seen = 0; /* blocks of the requests before r */
+    j->rc = ORC_OK;
+    for (uint32_t r = 0; r < j->n_req; ++r) {
+        uint64_t nb = j->hit_tokens[r] / g->block_tokens;
+        uint64_t b0 = j->first > seen ? j->first - seen : 0;
+        uint64_t b1 = j->last < seen + nb ? (j->last > seen ? j->last - seen : 0) : nb;
+        for (uint64_t b = b0; b < b1; ++b) {
+            uint64_t t = b * g->block_tokens; /* first token of the block */
+            for (uint32_t kv = 0; kv < 2; ++kv) {
+                uint32_t dev;
+                uint64_t soff, roff;
+                int64_t blk;
+                int rc = token_location(g, lo, j->layer, j->obj_start, j->obj_slot, j->blk_start,
+                                        j->block_ids, r, t, kv, &dev, &soff, &blk, &roff);
+                if (rc) { j->rc = rc; return NULL; }
+                if (blk < 0 || (uint64_t)blk >= j->n_pool_blocks) { j->rc = ORC_EINVAL; return NULL; }
+                uint8_t *in_store = j->store[dev] + soff;
+                uint8_t *in_pool = (kv ? j->pool_v : j->pool_k) + (uint64_t)blk * j->block_stride;
+                if (!j->pool_hnd) {
+                    if (j->to_pool) memcpy(in_pool, in_store, lo->block_bytes);
+                    else memcpy(in_store, in_pool, lo->block_bytes);
+                } else {
+                    uint64_t row = (uint64_t)g->head_dim * g->elem_bytes;
+                    for (uint32_t tok = 0; tok < g->block_tokens; ++tok)
+                        for (uint32_t hd = 0; hd < g->n_kv_heads; ++hd) {
+                            uint8_t *o = in_store + tok * lo->token_bytes + hd * row;
+                            uint8_t *q = in_pool + ((uint64_t)hd * g->block_tokens + tok) * row;
+                            if (j->to_pool) memcpy(q, o, row); else memcpy(o, q, row);
+                        }
+                }
+            }
+        }
+        seen += nb;
+    }
+    return NULL;
+}
+
+/* to_pool != 0: restore, else save.  n_threads >= 1; returns the oracle's codes. */
+int orc_move_layer_blocks_mt(const orc_geom *g, uint32_t layer, uint32_t n_req,
+                             const uint32_t *hit_tokens, const uint32_t *obj_start,
+                             const uint32_t *obj_slot, const uint32_t *blk_start,
+                             const int32_t *block_ids, uint8_t *const *store, uint8_t *pool_k,
+                             uint8_t *pool_v, uint64_t block_stride, uint64_t n_pool_blocks,
+                             int pool_hnd, int to_pool, uint32_t n_threads)
+{
+    orc_layout lo;
+    int rc = orc_obj_layout(g, &lo);
+    if (rc) return rc;
+    rc = check_batch(g, layer, n_req, hit_tokens, obj_start, blk_start);
+    if (rc) return rc;
+    if (n_threads == 0 || n_threads > 1024) return ORC_EINVAL;
+    uint64_t total = 0;
+    for (uint32_t r = 0; r < n_req; ++r) total += hit_tokens[r] / g->block_tokens;
+    mt_job *jobs = (mt_job *)calloc(n_threads, sizeof(mt_job));
+    pthread_t *tids = (pthread_t *)calloc(n_threads, sizeof(pthread_t));
+    if (!jobs || !tids) { free(jobs); free(tids); return ORC_ENOSPC; }
+    for (uint32_t k = 0; k < n_threads; ++k) {
+        mt_job *j = &jobs[k];
+        j->g = g; j->lo = &lo; j->layer = layer; j->n_req = n_req;
+        j->hit_tokens = hit_tokens; j->obj_start = obj_start; j->obj_slot = obj_slot;
+        j->blk_start = blk_start; j->block_ids = block_ids; j->store = store;
+        j->pool_k = pool_k; j->pool_v = pool_v; j->block_stride = block_stride;
+        j->n_pool_blocks = n_pool_blocks; j->to_pool = to_pool; j->pool_hnd = pool_hnd;
+        j->first = total * k / n_threads;
+        j->last = total * (k + 1) / n_threads;
+        j->threaded = 0;
+        /* the calling thread takes the last share (and any share no thread could be made for) */
+        if (k + 1 < n_threads && pthread_create(&tids[k], NULL, mt_worker, j) == 0)
+            j->threaded = 1;
+        else
+            mt_worker(j);
+    }
+    for (uint32_t k = 0; k < n_threads; ++k)
+        if (jobs[k].threaded) pthread_join(tids[k], NULL);
+    for (uint32_t k = 0; k < n_threads; ++k)
+        if (jobs[k].rc) rc = jobs[k].rc;
+    free(jobs);
+    free(tids);
+    return rc;
 }

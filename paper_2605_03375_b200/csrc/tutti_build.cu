@@ -514,19 +514,18 @@ uint32_t next_pow2(uint32_t v) {
 
 }  // namespace
 
+// The attribute is per device: set whenever a context is created, with its device current.
+cudaError_t build_kernels_setup() {
+    cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(SMEM_SORT_ITEMS * 12));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(bitonic_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)(SORT_TILE * 12));
+}
+
 cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
                         cudaStream_t stream, uint32_t *launches) {
     uint32_t np = next_pow2(2u * batch.n_obj);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(SMEM_SORT_ITEMS * 12));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(bitonic_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(SORT_TILE * 12));
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
     uint32_t n = 0;
     if (np <= SMEM_SORT_ITEMS) {
         // small batches get a small CTA: the kernel is a chain of block-wide barriers

@@ -26,7 +26,9 @@ namespace tutti {
 namespace {
 
 constexpr uint32_t CHUNK_BYTES = 32768;       // work unit of both engines
-constexpr int LDST_THREADS = 256;
+constexpr int LDST_THREADS = 256;             // one copy group of the ldst engine
+constexpr int LDST_MAX_GROUPS = 4;            // groups per CTA in a capped launch
+constexpr int LDST_PAD_SMEM = 120 * 1024;     // more than half an SM's shared memory
 constexpr uint32_t MBAR_TRY_LIMIT = 1u << 22;
 
 struct CopyParams {
@@ -36,6 +38,8 @@ struct CopyParams {
     uint32_t claim_chunks;
     uint32_t stages;        // bulk engine: stages per warp
     uint32_t chunk_bytes;   // bulk engine: bytes per stage (a power of two, 4..32 KiB)
+    uint32_t inject_timeout; // bulk engine: report the first wait of every stage as run out
+    uint32_t *smid_log;     // [grid] SM every CTA of the launch ran on (inspection)
     PermGeom perm;          // head-major pool blocks
 };
 
@@ -51,6 +55,12 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
+}
+
+__device__ __forceinline__ uint32_t smid() {
+    uint32_t v;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(v));
+    return v;
 }
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
@@ -166,33 +176,45 @@ __device__ __forceinline__ void st_stream(void *p, const uint4 &v) {
 // ---------------------------------------------------------------------------
 // ldst engine
 // ---------------------------------------------------------------------------
-template <int TO_POOL>
-__global__ void __launch_bounds__(LDST_THREADS, 4)
-copy_ldst_kernel(CopyParams p) {
-    __shared__ uint32_t s_claim;
-    __shared__ int s_mode;
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+// A CTA is one or more independent copy groups of LDST_THREADS threads, each with its
+// own named barrier.  On all SMs the launch is many one-group CTAs; a capped launch is
+// exactly sm_count CTAs of several groups (one CTA per SM, kept alone on its SM by a
+// shared-memory pad), so the cap holds on any stream.
+__device__ __forceinline__ void group_sync(uint32_t grp) {
+    asm volatile("bar.sync %0, %1;" ::"r"(grp + 1), "n"(LDST_THREADS) : "memory");
+}
 
-    __shared__ uint32_t s_bi;
+template <int TO_POOL>
+__global__ void __launch_bounds__(LDST_THREADS * LDST_MAX_GROUPS, 1)
+copy_ldst_kernel(CopyParams p) {
+    __shared__ uint32_t s_claim_g[LDST_MAX_GROUPS];
+    __shared__ int s_mode_g[LDST_MAX_GROUPS];
+    __shared__ uint32_t s_bi_g[LDST_MAX_GROUPS];
+    const uint32_t grp = threadIdx.x / LDST_THREADS, tid = threadIdx.x % LDST_THREADS;
+    const uint32_t lane = tid & 31, warp = tid >> 5;
+    uint32_t &s_claim = s_claim_g[grp];
+    int &s_mode = s_mode_g[grp];
+    uint32_t &s_bi = s_bi_g[grp];
+    if (threadIdx.x == 0 && p.smid_log) p.smid_log[blockIdx.x] = smid();
     for (uint32_t bi = 0; bi < p.n_iocb; ++bi) {
         // warp 0 looks ahead past IOCBs that need no copying
         if (warp == 0) {
-            uint32_t nb = skip_idle_iocbs(p.ring, p.first_iocb, bi, p.n_iocb, blockIdx.x == 0);
+            uint32_t nb = skip_idle_iocbs(p.ring, p.first_iocb, bi, p.n_iocb, blockIdx.x == 0 && grp == 0);
             if (lane == 0) s_bi = nb;
         }
-        __syncthreads();
+        group_sync(grp);
         bi = s_bi;
         if (bi >= p.n_iocb) break;
         const uint32_t idx = p.first_iocb + bi;
         IocbHdr *h = &p.ring.hdrs[idx & (p.ring.depth - 1)];
-        if (threadIdx.x == 0) s_mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
-        __syncthreads();
+        if (tid == 0) s_mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
+        group_sync(grp);
         const int mode = s_mode;
-        __syncthreads();
+        group_sync(grp);
         if (mode == IOCB_SKIP) continue;
         const uint32_t total = h->total_entries;
         if (total == 0 || h->status != 0) {
-            if (threadIdx.x == 0) complete_empty(p.ring, h, idx);
+            if (tid == 0) complete_empty(p.ring, h, idx);
             continue;
         }
         const uint32_t elen = h->entry_len;
@@ -202,7 +224,7 @@ copy_ldst_kernel(CopyParams p) {
         const bool hnd = (h->opcode & TUTTI_OP_FLAG_HND) != 0;
         if (hnd && (elen == 0 || elen != p.perm.block_tokens * p.perm.token_bytes)) {
             // a head-major entry must be exactly one block
-            if (threadIdx.x == 0) {
+            if (tid == 0) {
                 atomicCAS(&h->status, 0, TUTTI_EINVAL);
                 __threadfence();
                 if (atomicCAS(&h->state, state_word(idx, PHASE_READY), state_word(idx, PHASE_DONE)) ==
@@ -219,10 +241,10 @@ copy_ldst_kernel(CopyParams p) {
             const bool pow2 = (elen & (elen - 1)) == 0;
             const uint32_t shift = 31 - __clz(elen);
             for (;;) {
-                if (threadIdx.x == 0) s_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
-                __syncthreads();
+                if (tid == 0) s_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
+                group_sync(grp);
                 const uint32_t t0 = s_claim;
-                if (t0 >= n_tiles) { __syncthreads(); break; }
+                if (t0 >= n_tiles) { group_sync(grp); break; }
                 const uint32_t t1 = min(t0 + p.claim_chunks, n_tiles);
                 for (uint32_t t = t0; t < t1; ++t) {
                     // this warp's 4 KiB sub-range of the tile: 8 rows of 512 bytes
@@ -297,8 +319,8 @@ copy_ldst_kernel(CopyParams p) {
                         }
                     }
                 }
-                __syncthreads();
-                if (threadIdx.x == 0) {
+                group_sync(grp);
+                if (tid == 0) {
                     unsigned long long b0 = (unsigned long long)t0 * CHUNK_BYTES;
                     unsigned long long b1 = min((unsigned long long)t1 * CHUNK_BYTES, total_bytes);
                     account_done(p.ring, h, idx, b1 - b0);
@@ -308,10 +330,10 @@ copy_ldst_kernel(CopyParams p) {
             // general entries (lengths may differ): one warp per entry
             const uint32_t per_claim = 64;
             for (;;) {
-                if (threadIdx.x == 0) s_claim = atomicAdd(&h->claim_cursor, per_claim);
-                __syncthreads();
+                if (tid == 0) s_claim = atomicAdd(&h->claim_cursor, per_claim);
+                group_sync(grp);
                 const uint32_t c0 = s_claim;
-                if (c0 >= total) { __syncthreads(); break; }
+                if (c0 >= total) { group_sync(grp); break; }
                 const uint32_t c1 = min(c0 + per_claim, total);
                 unsigned long long moved = 0;
                 for (uint32_t e = c0 + warp; e < c1; e += LDST_THREADS / 32) {
@@ -332,7 +354,7 @@ copy_ldst_kernel(CopyParams p) {
                 }
                 __syncwarp();
                 if (lane == 0) account_done(p.ring, h, idx, moved);
-                __syncthreads();
+                group_sync(grp);
             }
         }
     }
@@ -447,6 +469,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     extern __shared__ __align__(128) unsigned char smem[];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t n_warps = blockDim.x >> 5;
+    if (threadIdx.x == 0 && p.smid_log) p.smid_log[blockIdx.x] = smid();
     const uint32_t S = p.stages;
     const uint32_t CB = p.chunk_bytes;
     unsigned char *data = smem + (size_t)warp * S * CB;
@@ -587,7 +610,6 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     // soon as the current chunk's loads are issued.
     auto fetch_next = [&]() {
         have_next = false;
-        if (failed) return;
         for (;;) {
             if (!f_open) {
                 if (!open_next_iocb()) return;
@@ -658,7 +680,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     for (;;) {
         // ---- issue loads while a stage is free (one stage of slack is kept for the
         //      store that may still be reading shared memory)
-        while (have_next && head - tail < S - 1) {
+        while (!failed && have_next && head - tail < S - 1) {
             const uint32_t s = head % S;
             // the store that last used this stage must have finished reading it:
             // at most one newer store group may still be pending
@@ -689,7 +711,23 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
             ++head;
             fetch_next();
         }
-        if (head == tail) break;
+        if (head == tail) {
+            if (!failed || !have_next) break;
+            // A wait ran out and every stage has been drained.  The chunks this agent has
+            // claimed, and whatever the launch still offers, are accounted without being
+            // copied (their IOCBs carry TUTTI_ETIMEDOUT): every IOCB still reaches its byte
+            // count, so its completion entry is posted and nothing waits for it for ever.
+            do {
+                if (n_bi != acct_bi) {
+                    flush_account();
+                    acct_bi = n_bi;
+                }
+                if (lane == 0) atomicCAS(&hdr_of(n_bi)->status, 0, TUTTI_ETIMEDOUT);
+                moved += __reduce_add_sync(0xffffffffu, ld_bytes);
+                fetch_next();
+            } while (have_next);
+            break;
+        }
 
         // ---- drain the oldest stage: wait for its bytes, store them
         const uint32_t s = tail % S;
@@ -704,13 +742,17 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
             flush_account();
             acct_bi = s_bi;
         }
-        bool arrived = mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
+        bool arrived = !p.inject_timeout && mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
         arrived = __all_sync(0xffffffffu, arrived);
-        phase_bits ^= (1u << s);
         if (!arrived) {
             failed = true;
             if (lane == 0) atomicCAS(&hdr_of(s_bi)->status, 0, TUTTI_ETIMEDOUT);
+            // the stage is given up, but its copy may still be on its way: one more bounded
+            // wait, so that nothing lands in this CTA's shared memory after it has left
+            (void)mbar_wait_bounded(bar, (phase_bits >> s) & 1u);
+            __syncwarp();
         }
+        phase_bits ^= (1u << s);
         const unsigned long long dst = st_addr_of[s * 32 + lane];
         const uint32_t nbytes = st_bytes_of[s * 32 + lane];
         const uint32_t off = st_off_of[s * 32 + lane];
@@ -725,7 +767,6 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
         bulk_commit();
         moved += chunk_bytes_of[s];
         ++tail;
-        if (failed) have_next = false;    // stop taking new work; the rest is drained
     }
     flush_account();
 }
@@ -738,13 +779,21 @@ cudaError_t copy_kernels_setup() {
     e = cudaFuncSetAttribute(copy_bulk_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(copy_bulk_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-    return e;
+    if (e != cudaSuccess) return e;
+    // the ldst engine uses dynamic shared memory only as a pad that keeps a capped CTA alone
+    // on its SM
+    e = cudaFuncSetAttribute(copy_ldst_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, LDST_PAD_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(copy_ldst_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, LDST_PAD_SMEM);
+    if (e != cudaSuccess) return e;
+    return build_kernels_setup();
 }
 
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
                         bool pool_hnd, const PermGeom &perm, const StoreTensorMaps *maps,
-                        cudaStream_t stream, uint32_t *launches) {
+                        uint32_t *smid_log, cudaStream_t stream, uint32_t *launches,
+                        uint32_t *grid_out) {
     static const StoreTensorMaps no_maps = {};
     const StoreTensorMaps &tm = maps ? *maps : no_maps;
     CopyParams p;
@@ -753,6 +802,9 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     p.n_iocb = n_iocb;
     p.opcode = opcode;
     p.wait_ns = opt.wait_ns;
+    p.inject_timeout = opt.inject_timeout;
+    p.smid_log = smid_log;
+    uint32_t grid = 0;
     // measured: small claims balance best when every SM takes part, larger ones amortise the
     // claim's round trip when few SMs carry everything
     p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : (sm_count ? 4 : 2);
@@ -779,6 +831,7 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
         size_t smem = (size_t)warps * stages * per_stage;
         // a capped launch keeps one CTA per SM: pad shared memory so no second CTA fits
         if (sm_count && smem < 120u * 1024u) smem = 120u * 1024u;
+        grid = sms;
         if (opcode == TUTTI_OP_READ)
             copy_bulk_kernel<1><<<sms, warps * 32, smem, stream>>>(p, tm);
         else
@@ -787,12 +840,19 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
         p.stages = 0;
         p.chunk_bytes = CHUNK_BYTES;
         uint32_t per_sm = opt.ctas_per_sm ? opt.ctas_per_sm : 4;
+        if (per_sm > LDST_MAX_GROUPS) per_sm = LDST_MAX_GROUPS;
+        // all SMs: per_sm one-group CTAs per SM.  Capped: exactly sm_count CTAs of per_sm
+        // groups each, one per SM (the pad leaves no room for a second CTA).
+        const uint32_t threads = sm_count ? per_sm * LDST_THREADS : LDST_THREADS;
+        const size_t smem = sm_count ? LDST_PAD_SMEM : 0;
+        grid = sm_count ? sm_count : sms * per_sm;
         if (opcode == TUTTI_OP_READ)
-            copy_ldst_kernel<1><<<sms * per_sm, LDST_THREADS, 0, stream>>>(p);
+            copy_ldst_kernel<1><<<grid, threads, smem, stream>>>(p);
         else
-            copy_ldst_kernel<0><<<sms * per_sm, LDST_THREADS, 0, stream>>>(p);
+            copy_ldst_kernel<0><<<grid, threads, smem, stream>>>(p);
     }
     if (launches) *launches = 1;
+    if (grid_out) *grid_out = grid;
     return cudaGetLastError();
 }
 

@@ -126,6 +126,7 @@ struct CopyOptions {
     uint32_t bulk_warps, bulk_stages;
     uint32_t claim_chunks;
     uint32_t bulk_chunk;    // bytes per stage of the bulk engine (0 = 32 KiB)
+    uint32_t inject_timeout; // test hook: the bulk engine's stage waits report "ran out"
 };
 
 // kernels (tutti_build.cu / tutti_copy.cu)
@@ -140,7 +141,11 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
                         bool pool_hnd, const PermGeom &perm, const StoreTensorMaps *maps,
-                        cudaStream_t stream, uint32_t *launches);
+                        uint32_t *smid_log, cudaStream_t stream, uint32_t *launches,
+                        uint32_t *grid_out);
+// Per-device kernel attributes (dynamic shared memory opt-ins) of every kernel of the
+// library; called with the device current whenever a context is created on it.
 cudaError_t copy_kernels_setup();
+cudaError_t build_kernels_setup();
 
 }  // namespace tutti

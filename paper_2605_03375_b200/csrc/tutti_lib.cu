@@ -6,6 +6,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include "tutti_internal.h"
@@ -83,6 +84,11 @@ struct tutti_ring {
     std::vector<tutti_cqe_t> completed;   // per slot
     std::vector<uint8_t> have_cqe;        // per slot
     std::vector<uint8_t> opcode_of;       // per slot, opcode of the reservation (0xff = unknown)
+    std::vector<uint8_t> issued;          // per slot: a copy launch that executes it was enqueued
+    std::vector<uint64_t> fill_optr;      // tutti_ring_fill_host scratch (sized at create)
+    std::vector<uint8_t> fill_seen;
+    uint32_t *smid_log = nullptr;         // device: SM of every CTA of the last copy launch
+    uint32_t smid_cap = 0, last_grid = 0;
     uint32_t sgl_capacity;
     // plan cache key
     bool plan_valid = false;
@@ -174,7 +180,7 @@ int tutti_ctx_create(const tutti_geom_t *geom, int device, tutti_ctx_t **out) {
     c->pool.assign(geom->n_layers, PoolLayer{0, 0, 0, 0, false});
     for (auto &s : c->store) s = StoreDev{0, 0, 0, false, false};
     memset(&c->maps, 0, sizeof(c->maps));
-    c->opt = CopyOptions{0, 2000000ull, 4, 0, 0, 0, 0};   // 0 = chosen per launch
+    c->opt = CopyOptions{0, 2000000ull, 4, 0, 0, 0, 0, 0};   // 0 = chosen per launch
     c->gdev.block_tokens = geom->block_tokens;
     c->gdev.obj_tokens = geom->obj_tokens;
     c->gdev.blocks_per_obj = (uint32_t)lo.blocks_per_obj;
@@ -304,6 +310,10 @@ int tutti_set_option(tutti_ctx_t *ctx, uint32_t option, uint64_t value) {
             if (value < 4096 || value > 32768 || (value & (value - 1))) return TUTTI_EINVAL;
             ctx->opt.bulk_chunk = (uint32_t)value;
             return TUTTI_OK;
+        case TUTTI_OPT_INJECT_BULK_TIMEOUT:
+            if (value > 1) return TUTTI_EINVAL;
+            ctx->opt.inject_timeout = (uint32_t)value;
+            return TUTTI_OK;
         default:
             return TUTTI_EINVAL;
     }
@@ -339,6 +349,10 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
     r->completed.resize(depth);
     r->have_cqe.assign(depth, 0);
     r->opcode_of.assign(depth, 0xff);
+    r->issued.assign(depth, 0);
+    r->fill_optr.resize(sgl_capacity < (1u << 16) ? sgl_capacity : (1u << 16));
+    r->fill_seen.resize(r->fill_optr.size());
+    r->smid_cap = (uint32_t)ctx->device_sms * 8u;
     RingDev &d = r->dev;
     memset(&d, 0, sizeof(d));
     d.depth = depth;
@@ -359,6 +373,7 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
     A((void **)&d.plan_key, sizeof(unsigned long long) * (size_t)np, false);
     A((void **)&d.plan_idx, sizeof(uint32_t) * (size_t)np, false);
     A((void **)&d.plan_counts, 2 * sizeof(PlanCounts), true);
+    A((void **)&r->smid_log, sizeof(uint32_t) * r->smid_cap, true);
     if (rc == TUTTI_OK) {
         // headers start out "done" for an index that is never issued first
         cudaError_t e = cudaHostAlloc((void **)&r->cq_host, sizeof(CqSlot) * depth,
@@ -433,6 +448,7 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
         uint32_t slot = (first + k) & (r->dev.depth - 1);
         r->have_cqe[slot] = 0;
         r->opcode_of[slot] = (uint8_t)opcode;
+        r->issued[slot] = 0;
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
@@ -501,9 +517,12 @@ static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, 
     uint32_t launches = 0;
     PermGeom pg{ctx->geom.block_tokens, ctx->geom.n_kv_heads,
                 ctx->geom.head_dim * ctx->geom.elem_bytes, (uint32_t)ctx->layout.token_bytes};
+    uint32_t grid = 0;
     CK(launch_copy(r->dev, first, n, opcode, sm_count, ctx->device_sms, ctx->opt, host_store,
-                   ctx->pool_hnd, pg, &ctx->maps, (cudaStream_t)stream, &launches));
+                   ctx->pool_hnd, pg, &ctx->maps, r->smid_log, (cudaStream_t)stream, &launches, &grid));
     r->kernel_launches += launches;
+    r->last_grid = grid < r->smid_cap ? grid : r->smid_cap;
+    for (uint32_t k = 0; k < n; ++k) r->issued[(first + k) & (r->dev.depth - 1)] = 1;
     return TUTTI_OK;
 }
 
@@ -543,7 +562,7 @@ int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64
     if (!r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
     const uint32_t slot = iocb_idx & (r->dev.depth - 1);
     auto t0 = std::chrono::steady_clock::now();
-    for (;;) {
+    for (uint32_t spins = 0;; ++spins) {
         if (!r->have_cqe[slot]) drain_cq(r);
         if (r->have_cqe[slot]) {
             *out = r->completed[slot];
@@ -554,12 +573,27 @@ int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64
         auto dt = std::chrono::duration_cast<std::chrono::nanoseconds>(
                       std::chrono::steady_clock::now() - t0).count();
         if ((uint64_t)dt >= timeout_ns) return TUTTI_EAGAIN;
+        // a short busy phase for completions that are microseconds away, then the core is
+        // given back between looks at the queue
+        if (dt < 50000) {
+#if defined(__x86_64__) || defined(__i386__)
+            __builtin_ia32_pause();
+#else
+            std::this_thread::yield();
+#endif
+        } else {
+            std::this_thread::sleep_for(std::chrono::microseconds(spins < 4096 ? 5 : 50));
+        }
     }
 }
 
 int tutti_stream_wait_iocb(tutti_ring_t *r, uint32_t iocb_idx, void *stream) {
     if (!r || !r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
     r->host_calls++;
+    // Only an IOCB whose copy launch is already enqueued may be waited for: that launch
+    // terminates by itself (all its waits are bounded) and leaves the state word at DONE,
+    // so the stream wait cannot outlive it.  Nothing is enqueued for any other index.
+    if (!r->issued[iocb_idx & (r->dev.depth - 1)]) return TUTTI_EAGAIN;
     typedef CUresult (*wait_fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
     static wait_fn fn = nullptr;
     if (!fn) {
@@ -575,7 +609,9 @@ int tutti_stream_wait_iocb(tutti_ring_t *r, uint32_t iocb_idx, void *stream) {
     DeviceGuard guard(r->ctx->device);
     const uint32_t slot = iocb_idx & (r->dev.depth - 1);
     CUdeviceptr addr = (CUdeviceptr)(uintptr_t)&r->dev.hdrs[slot].state;
-    CUresult res = fn((CUstream)stream, addr, state_word(iocb_idx, PHASE_DONE), CU_STREAM_WAIT_VALUE_EQ);
+    // ">=" in the cyclic sense the driver defines: also satisfied when the slot has moved on
+    // to a later IOCB by the time the stream reaches the wait
+    CUresult res = fn((CUstream)stream, addr, state_word(iocb_idx, PHASE_DONE), CU_STREAM_WAIT_VALUE_GEQ);
     if (res != CUDA_SUCCESS) {
         g_last_cuda_error = "cuStreamWaitValue32: CUresult " + std::to_string((int)res);
         return TUTTI_ECUDA;
@@ -594,6 +630,7 @@ int tutti_ring_reserve(tutti_ring_t *r, uint32_t n_iocb, uint32_t n_sgl, uint32_
         uint32_t slot = (first + k) & (r->dev.depth - 1);
         r->have_cqe[slot] = 0;
         r->opcode_of[slot] = 0xff;
+        r->issued[slot] = 0;
     }
     *first_iocb = first;
     return TUTTI_OK;
@@ -608,8 +645,13 @@ int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
     if (!g) return TUTTI_EINVAL;
     if ((uint64_t)sgl_offset + n_sgl > g->sgl_count) return TUTTI_EINVAL;
     // walk the contexts as a device would: object-side address of every entry
-    std::vector<uint64_t> optr(n_sgl ? n_sgl : 1);
-    std::vector<uint8_t> seen(n_sgl ? n_sgl : 1, 0);
+    if (n_sgl > r->fill_optr.size()) {        // grows once for an unusually long IOCB, then stays
+        r->fill_optr.resize(n_sgl);
+        r->fill_seen.resize(n_sgl);
+    }
+    uint64_t *optr = r->fill_optr.data();
+    uint8_t *seen = r->fill_seen.data();
+    memset(seen, 0, n_sgl);
     uint64_t total = 0;
     uint32_t common = n_sgl ? sgl[0].len : 0;
     uint32_t opcode = n_sqe ? sqes[0].opcode : TUTTI_OP_READ;
@@ -645,7 +687,7 @@ int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
                            sizeof(tutti_sqe_t) * n_sqe, cudaMemcpyHostToDevice, st));
     if (n_sgl) {
         CK(cudaMemcpyAsync(r->dev.sgl + at, sgl, sizeof(tutti_sgl_t) * n_sgl, cudaMemcpyHostToDevice, st));
-        CK(cudaMemcpyAsync(r->dev.obj_ptr + at, optr.data(), sizeof(uint64_t) * n_sgl,
+        CK(cudaMemcpyAsync(r->dev.obj_ptr + at, optr, sizeof(uint64_t) * n_sgl,
                            cudaMemcpyHostToDevice, st));
     }
     IocbHdr h;
@@ -705,6 +747,16 @@ int tutti_ring_read_sgl(tutti_ring_t *r, uint32_t iocb_idx, tutti_sgl_t *sgl, ui
     if (sgl && n)
         CK(cudaMemcpy(sgl, r->dev.sgl + (size_t)h.sgl_base + h.entry_first, sizeof(tutti_sgl_t) * n,
                       cudaMemcpyDeviceToHost));
+    return TUTTI_OK;
+}
+
+int tutti_ring_last_launch_sms(tutti_ring_t *r, uint32_t *smids, uint32_t max_ctas, uint32_t *n_ctas) {
+    if (!r || !n_ctas || (max_ctas && !smids)) return TUTTI_EINVAL;
+    DeviceGuard guard(r->ctx->device);
+    CK(cudaDeviceSynchronize());
+    *n_ctas = r->last_grid;
+    uint32_t n = r->last_grid < max_ctas ? r->last_grid : max_ctas;
+    if (n) CK(cudaMemcpy(smids, r->smid_log, sizeof(uint32_t) * n, cudaMemcpyDeviceToHost));
     return TUTTI_OK;
 }
 

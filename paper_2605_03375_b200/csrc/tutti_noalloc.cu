@@ -7,10 +7,13 @@
 // the plan arrays — in one file-scope device array that every GPU loading the
 // library holds until the process exits.
 #include <mutex>
+#include <string>
 
 #include "tutti_internal.h"
 
 using namespace tutti;
+
+extern "C" void tutti_set_cuda_error_(const char *msg);
 
 namespace {
 
@@ -45,18 +48,33 @@ std::mutex g_mu;
 unsigned char *g_scratch_addr[MAX_GPUS] = {nullptr};
 int g_sms[MAX_GPUS] = {0};
 
+int fail(cudaError_t e, const char *what) {
+    std::string m = std::string(what) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")";
+    tutti_set_cuda_error_(m.c_str());
+    return TUTTI_ECUDA;
+}
+
+// Header, counters and completion slot start from zero; the slot's status starts as
+// "timed out", so a launch that never posts its completion is not read as a success.
+__global__ void noalloc_reset_kernel(unsigned char *base) {
+    uint32_t *w = reinterpret_cast<uint32_t *>(base);
+    for (uint32_t i = threadIdx.x; i < CLEAR_BYTES / 4; i += blockDim.x) w[i] = 0;
+    __syncthreads();
+    if (threadIdx.x == 0) reinterpret_cast<CqSlot *>(base + OFF_CQ)->cqe.status = TUTTI_ETIMEDOUT;
+}
+
 // Once per device, with that device current: resolve the scratch address.
 int setup_device(int device, unsigned char **out, int *sms) {
     std::lock_guard<std::mutex> lock(g_mu);
     if (!g_scratch_addr[device]) {
         unsigned char *ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch);
-        if (e != cudaSuccess || !ptr) return TUTTI_ECUDA;
+        if (e != cudaSuccess || !ptr) return fail(e != cudaSuccess ? e : cudaErrorInvalidSymbol, "cudaGetSymbolAddress");
         int n = 0;
         e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device);
-        if (e != cudaSuccess) return TUTTI_ECUDA;
+        if (e != cudaSuccess) return fail(e, "cudaDeviceGetAttribute");
         e = copy_kernels_setup();
-        if (e != cudaSuccess) return TUTTI_ECUDA;
+        if (e != cudaSuccess) return fail(e, "kernel attributes");
         g_sms[device] = n;
         g_scratch_addr[device] = ptr;
     }
@@ -96,8 +114,9 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         sbytes[d] = store_bytes[d];
     }
     int prev = -1;
-    if (cudaGetDevice(&prev) != cudaSuccess) return TUTTI_ECUDA;
-    if (prev != device && cudaSetDevice(device) != cudaSuccess) return TUTTI_ECUDA;
+    cudaError_t e0 = cudaGetDevice(&prev);
+    if (e0 != cudaSuccess) return fail(e0, "cudaGetDevice");
+    if (prev != device && (e0 = cudaSetDevice(device)) != cudaSuccess) return fail(e0, "cudaSetDevice");
     unsigned char *base = nullptr;
     int sms = 0;
     rc = setup_device(device, &base, &sms);
@@ -135,11 +154,12 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         BatchDev b{batch->n_req, batch->n_obj, batch->n_blk, batch->hit_tokens, batch->obj_start,
                    batch->obj_slot, batch->blk_start, batch->block_ids};
         PoolLayer pool{(uint64_t)k_base, (uint64_t)v_base, block_stride, n_blocks, true};
-        CopyOptions opt{2, 2000000ull, 4, 0, 0, 0, 0};
+        CopyOptions opt{2, 2000000ull, 4, 0, 0, 0, 0, 0};
         uint32_t launches = 0;
         // header, completion slot and counters must start at zero: the array still holds
         // whatever the previous call left there
-        cudaError_t e = cudaMemsetAsync(base, 0, CLEAR_BYTES, st);
+        noalloc_reset_kernel<<<1, 256, 0, st>>>(base);
+        cudaError_t e = cudaGetLastError();
         if (e == cudaSuccess) e = launch_plan(r, g, b, st, nullptr);
         if (e == cudaSuccess)
             e = launch_emit(r, g, b, layer, 1, TUTTI_OP_READ, pool, nullptr, sbase, sbytes, 0, 1, 0,
@@ -148,10 +168,10 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
             e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, false,
                             PermGeom{geom->block_tokens, geom->n_kv_heads,
                                      geom->head_dim * geom->elem_bytes, (uint32_t)lo.token_bytes},
-                            nullptr, st, &launches);
+                            nullptr, nullptr, st, &launches, nullptr);
         if (e == cudaSuccess)
             e = cudaMemcpyAsync(cqe_out, base + OFF_CQ, sizeof(tutti_cqe_t), cudaMemcpyDefault, st);
-        if (e != cudaSuccess) rc = TUTTI_ECUDA;
+        if (e != cudaSuccess) rc = fail(e, "tutti_kv_restore_layer_noalloc");
     }
     if (prev != device) cudaSetDevice(prev);
     return rc;

@@ -19,7 +19,7 @@ LAYOUT_FILE_MAJOR, LAYOUT_LAYER_MAJOR = 0, 1
 OP_READ, OP_WRITE = 0, 1
 STORE_HBM, STORE_HOST_PINNED = 0, 1
 OPT_COPY_ENGINE, OPT_WAIT_NS, OPT_CTAS_PER_SM, OPT_BULK_WARPS, OPT_BULK_STAGES, OPT_CLAIM_CHUNKS, \
-    OPT_BULK_CHUNK_BYTES, OPT_POOL_LAYOUT = 1, 2, 3, 4, 5, 6, 7, 8
+    OPT_BULK_CHUNK_BYTES, OPT_POOL_LAYOUT, OPT_INJECT_BULK_TIMEOUT = 1, 2, 3, 4, 5, 6, 7, 8, 9
 POOL_NHD, POOL_HND = 0, 1
 OP_FLAG_HND = 0x100
 ENGINE_AUTO, ENGINE_LDST, ENGINE_BULK = 0, 1, 2
@@ -79,7 +79,7 @@ EXPORTS = [
     "tutti_filepool_create", "tutti_filepool_destroy", "tutti_filepool_insert",
     "tutti_filepool_lookup", "tutti_filepool_match_prefix", "tutti_filepool_pin",
     "tutti_filepool_remove", "tutti_filepool_stats", "tutti_build_sqes_layers",
-    "tutti_stream_wait_iocb",
+    "tutti_stream_wait_iocb", "tutti_ring_last_launch_sms",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -117,6 +117,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_ring_read_iocb": (C.c_int, [vp, u32, P(IocbInfo), vp, u32]),
         "tutti_ring_read_sgl": (C.c_int, [vp, u32, vp, u32, P(u32)]),
         "tutti_ring_stats": (C.c_int, [vp, P(u64), P(u64)]),
+        "tutti_ring_last_launch_sms": (C.c_int, [vp, vp, u32, P(u32)]),
         "tutti_sm_partition_create": (C.c_int, [vp, u32, P(vp), P(vp), P(u32), P(u32)]),
         "tutti_sm_partition_destroy": (C.c_int, [vp]),
         "tutti_hostring_create": (vp, [u32, u32]),
@@ -333,6 +334,14 @@ class Ring:
         _check(self.lib.tutti_ring_read_sgl(self.h, iocb_idx, sgl.ctypes.data, max_entries,
                                             C.byref(n)), "tutti_ring_read_sgl")
         return sgl[:min(n.value, max_entries)].copy()
+
+    def tutti_ring_last_launch_sms(self) -> np.ndarray:
+        """SM id of every CTA of the most recent copy launch (synchronises)."""
+        out = np.zeros(4096, dtype=np.uint32)
+        n = C.c_uint32()
+        _check(self.lib.tutti_ring_last_launch_sms(self.h, out.ctypes.data, len(out), C.byref(n)),
+               "tutti_ring_last_launch_sms")
+        return out[:min(n.value, len(out))].copy()
 
     def tutti_ring_stats(self) -> Tuple[int, int]:
         a, b = C.c_uint64(), C.c_uint64()

@@ -154,3 +154,94 @@ def test_bad_slot_in_a_large_batch_is_reported():
         assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
     finally:
         dc.close()
+
+
+def test_bulk_stage_wait_running_out_still_completes_every_iocb():
+    """The bulk engine's wait for a stage's bytes is made to report "ran out" from the host
+    (TUTTI_OPT_INJECT_BULK_TIMEOUT; nothing on the GPU faults or hangs).  Every IOCB of the
+    launch must still complete — with TUTTI_ETIMEDOUT — so that a poll never waits for ever,
+    and the ring must keep working afterwards."""
+    w = wl.config(2, 0.05, n_layers=3)
+    dc = DeviceCase(w, depth=16, capacity=8, sgl_capacity=2 * len(w.block_ids) * 4)
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, T.ENGINE_BULK)
+        for sm_count in (0, 8):
+            dc.ctx.tutti_set_option(T.OPT_INJECT_BULK_TIMEOUT, 1)
+            rc, first, per = dc.ring.tutti_build_sqes_layers(dc.batch, 0, 2, T.OP_READ)
+            assert per > 1                                          # several IOCBs per layer
+            infos = [dc.ring.tutti_ring_read_iocb(i)[0] for i in range(first, first + 2 * per)]
+            dc.ring.tutti_kv_restore_layer(first, 2 * per, sm_count)
+            cqes = dc.poll_all(first, 2 * per)
+            assert sorted(c[0] for c in cqes) == list(range(first, first + 2 * per))
+            for (idx, status, nbytes), info in zip(sorted(cqes), infos):
+                if info.total_entries:
+                    assert status == T.ETIMEDOUT, (idx, status)
+                else:
+                    assert status == 0 and nbytes == 0               # the empty tail of the reservation
+            # stream waits on those IOCBs are released too (they completed, with an error)
+            s2 = torch.cuda.Stream()
+            rc2, f2, n2 = dc.ring.tutti_build_sqes(dc.batch, 2, T.OP_READ)
+            dc.ring.tutti_kv_restore_layer(f2, n2, sm_count)
+            dc.ring.tutti_stream_wait_iocb(f2, s2)
+            s2.synchronize()
+            dc.poll_all(f2, n2)
+            # back to normal: the same ring moves the bytes
+            dc.ctx.tutti_set_option(T.OPT_INJECT_BULK_TIMEOUT, 0)
+            for layer in (0, 1):
+                dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
+                rc, f, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+                dc.ring.tutti_kv_restore_layer(f, n, sm_count)
+                assert all(c[1] == 0 for c in dc.poll_all(f, n))
+                assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+    finally:
+        dc.close()
+
+
+def test_stream_wait_refuses_an_iocb_that_was_not_issued():
+    """A stream wait is enqueued only for an IOCB whose copy launch is already in the stream:
+    for a built-but-unissued index the call answers TUTTI_EAGAIN and enqueues nothing (the
+    stream stays free), so no stream can be left waiting for a completion nobody produces."""
+    dc = DeviceCase(small())
+    s_use = torch.cuda.Stream()
+    try:
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        assert dc.ring.tutti_stream_wait_iocb(first, s_use, allow=(T.EAGAIN,)) == T.EAGAIN
+        rc, rsv = dc.ring.tutti_ring_reserve(1, 16)                 # reserved, never filled
+        assert dc.ring.tutti_stream_wait_iocb(rsv, s_use, allow=(T.EAGAIN,)) == T.EAGAIN
+        done = torch.zeros(1, device=dc.dev)
+        with torch.cuda.stream(s_use):
+            done.add_(1)                                            # runs at once: nothing is waited for
+        s_use.synchronize()
+        assert done.item() == 1
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert dc.ring.tutti_stream_wait_iocb(first, s_use) == T.OK  # issued: accepted
+        s_use.synchronize()
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        # the reserved IOCB is completed by a launch whose bounded wait runs out
+        dc.ctx.tutti_set_option(T.OPT_WAIT_NS, 100_000)
+        dc.ring.tutti_kv_restore_layer(rsv, 1)
+        assert dc.poll_all(rsv, 1)[0][1] == T.ETIMEDOUT
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
+@pytest.mark.parametrize("sm_count", [4, 8, 32])
+def test_capped_launch_stays_on_sm_count_sms(engine, sm_count):
+    """SM-capped mode on a plain stream (no green-context partition): the launch is exactly
+    sm_count CTAs and they sit on sm_count different SMs, with either copy engine."""
+    w = wl.config(2, 0.1, n_layers=1)
+    dc = DeviceCase(w)
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+        for op in (T.OP_READ, T.OP_WRITE):
+            rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, op)
+            (dc.ring.tutti_kv_restore_layer if op == T.OP_READ else dc.ring.tutti_kv_save_layer)(
+                first, n, sm_count)
+            assert all(c[1] == 0 for c in dc.poll_all(first, n))
+            smids = dc.ring.tutti_ring_last_launch_sms()
+            assert len(smids) == sm_count
+            assert len(set(smids.tolist())) == sm_count
+        assert np.array_equal(dc.pool_dev[0].cpu().numpy(), dc.oracle_restore(0))
+    finally:
+        dc.close()

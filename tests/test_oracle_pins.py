@@ -208,6 +208,19 @@ def test_restore_equals_numpy_indexing(case):
         assert rc == oracle.OK
         exp = _expected_pool_numpy(w, lo, store, pool0, layer)
         assert np.array_equal(pool, exp)
+        # the block-granular multi-threaded form (the all-cores baseline) gives the same bytes,
+        # and its save equals the plain save
+        pool_mt = pool0.copy()
+        assert oracle.move_layer_blocks_mt(g, layer, hc.batch_of(w), store, pool_mt, k_off, v_off,
+                                           stride, w.n_pool_blocks, True, 7, w.pool_hnd) == 0
+        assert np.array_equal(pool_mt, exp)
+        st_a = [np.zeros_like(x) for x in store]
+        st_b = [np.zeros_like(x) for x in store]
+        assert oracle.save_layer(g, layer, hc.batch_of(w), st_a, exp, k_off, v_off, stride,
+                                 w.n_pool_blocks, w.pool_hnd) == 0
+        assert oracle.move_layer_blocks_mt(g, layer, hc.batch_of(w), st_b, exp, k_off, v_off,
+                                           stride, w.n_pool_blocks, False, 7, w.pool_hnd) == 0
+        assert all(np.array_equal(a, b) for a, b in zip(st_a, st_b))
         # blocks not in the block table are byte-unchanged (canary / background)
         touched = np.zeros(w.n_pool_blocks, dtype=bool)
         touched[w.block_ids] = True

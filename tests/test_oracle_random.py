@@ -107,6 +107,17 @@ def test_restore_and_save_against_python_loops(seed):
                              c["hnd"]) == 0
     for a, b in zip(st_got, st_exp):
         assert np.array_equal(a, b)
+    # the block-granular, multi-threaded form used as the all-cores baseline: same bytes
+    for n_thr in (1, 2, 3, 5):
+        got_mt = pool0.copy()
+        assert oracle.move_layer_blocks_mt(g, layer, batch, store, got_mt, k_off, v_off, stride,
+                                           c["n_pool"], True, n_thr, c["hnd"]) == 0
+        assert np.array_equal(got_mt, exp)
+        st_mt = [s.copy() for s in store]
+        assert oracle.move_layer_blocks_mt(g, layer, batch, st_mt, pool1, k_off, v_off, stride,
+                                           c["n_pool"], False, n_thr, c["hnd"]) == 0
+        for a, b in zip(st_mt, st_exp):
+            assert np.array_equal(a, b)
     # descriptors executed = plain restore
     flag = oracle.OP_HND if c["hnd"] else 0
     base = 1 << 32

@@ -254,15 +254,17 @@ class Replica:
         self.saved_ev = {}          # duplex mode: last save of every layer
         # duplex mode: each direction on a few SMs, so that both kernels are resident at once
         # (the host link, not the SM count, bounds them)
-        self.duplex_sms = getattr(args, "e2e_sms", 8)
-        self.duplex_save_sms = getattr(args, "e2e_save_sms", 0) or self.duplex_sms
+        self.duplex_sms = getattr(args, "e2e_sms", 12)
+        self.duplex_save_sms = getattr(args, "e2e_save_sms", 8) or self.duplex_sms
         self.unpolled = []          # duplex mode: IOCBs of the previous pass
         self.two_streams = not getattr(args, "one_stream", False)
         G = getattr(args, "layers_per_launch", 0)
         if not G:
-            # one copy launch (and one build launch) spans enough layers to move ~4 GiB: 4 layers
-            # of a config-2 batch, a whole pass of a short prefix
-            G = max(4, min(w.n_layers, int(round(4 * GIB / max(self.payload_per_layer, 1)))))
+            # one build launch and one copy launch span the whole pass (measured on config 2:
+            # 0.978 of the copy peak with one layer per launch, 1.014 with 4, 1.024 with 32;
+            # for short prefixes the launches are the cost).  Every layer keeps its own IOCBs
+            # and completion entries, so a layer still completes as soon as its bytes landed.
+            G = w.n_layers
         G = min(G, w.n_layers, max(1, depth // (2 * n_iocb_layer)))
         self.layers_per_launch = max(1, G)
         self.epoch = 1
@@ -349,55 +351,62 @@ class Replica:
         T = self.T
         total = 0
         for first, n in issued:
-            for i in range(first, first + n):
-                rc, cqe = self.ring.tutti_ring_poll(i, 20_000_000_000)
-                if rc != T.OK or cqe.status != 0:
-                    raise RuntimeError(f"IOCB {i}: poll rc {rc}, status {cqe.status}")
-                total += cqe.bytes
+            rc, nbytes, err, done = self.ring.tutti_ring_poll_range(first, n, 20_000_000_000)
+            if rc != T.OK or err != 0:
+                raise RuntimeError(f"IOCBs {first}+{n}: poll rc {rc}, status {err}, {done} done")
+            total += nbytes
         return total
 
-    def step_duplex(self, upload_tables=False):
-        """One pass with both directions of the host link busy: layer l is saved on its own
-        stream as soon as it has been restored, while layer l+1 is being restored.  Ordering is
-        by events: a save waits for the restore of its layer, a restore waits for the previous
-        pass's save of its layer (same objects, same pool buffer).  Completions of a pass are
-        polled after the next pass has been issued, so the streams never run dry."""
+    def step_duplex(self, upload_tables=False, group=2, times=None):
+        """One pass with both directions of the host link busy: a group of layers is saved on
+        its own stream as soon as it has been restored, while the next group is being restored.
+        The READ and the WRITE descriptors of the whole pass are built with one call each; a
+        copy launch executes the IOCBs of `group` consecutive layers.  Ordering is by events: a
+        save waits for the restore of its layers, a restore waits for the previous pass's save
+        of its layers (same objects, same pool buffers).  Completions of a pass are polled
+        after the next pass has been issued, so the streams never run dry."""
         T, torch = self.T, self.torch
         sR, sW, sb = self.stream, self.write_stream, self.build_stream
-        assert self.R == self.w.n_layers, "duplex mode needs one pool buffer per layer"
+        L = self.w.n_layers
+        assert self.R == L, "duplex mode needs one pool buffer per layer"
         self.epoch += 1
         self.batch.plan_epoch = self.epoch
-        issued = []
-        start = torch.cuda.Event()
-        start.record(sR)
-        sb.wait_event(start)
         if upload_tables:
+            # the tables are read only by the build kernels, which run on this same stream:
+            # stream order alone keeps the upload behind the previous pass's builds
             with torch.cuda.stream(sb):
-                if self.saved_ev:       # the tables are read by builds still in flight
-                    for ev in self.saved_ev.values():
-                        sb.wait_event(ev)
                 for h, d in zip(self.tables_host, self.tables_dev):
                     d.copy_(h, non_blocking=True)
-        for l in range(self.w.n_layers):
-            rc, fr, nr = self.ring.tutti_build_sqes(self.batch, l, T.OP_READ, stream=sb)
-            rc, fw, nw = self.ring.tutti_build_sqes(self.batch, l, T.OP_WRITE, stream=sb)
-            built = torch.cuda.Event()
-            built.record(sb)
-            sR.wait_event(built)
-            if l in self.saved_ev:
-                sR.wait_event(self.saved_ev[l])
-            self.ring.tutti_kv_restore_layer(fr, nr, self.duplex_sms, stream=sR)
+        rc, fr, per_r = self.ring.tutti_build_sqes_layers(self.batch, 0, L, T.OP_READ, stream=sb)
+        rc, fw, per_w = self.ring.tutti_build_sqes_layers(self.batch, 0, L, T.OP_WRITE, stream=sb)
+        built = torch.cuda.Event()
+        built.record(sb)
+        sR.wait_event(built)
+        sW.wait_event(built)
+        if times is not None:
+            for key, st in (("r0", sR), ("w0", sW)):
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record(st)
+                times.setdefault(key, []).append(ev)
+        for l0 in range(0, L, group):
+            g = min(group, L - l0)
+            if l0 in self.saved_ev:
+                sR.wait_event(self.saved_ev[l0])
+            self.ring.tutti_kv_restore_layer(fr + l0 * per_r, g * per_r, self.duplex_sms, stream=sR)
             restored = torch.cuda.Event()
             restored.record(sR)
-            sW.wait_event(built)
             sW.wait_event(restored)
-            self.ring.tutti_kv_save_layer(fw, nw, self.duplex_save_sms, stream=sW)
+            self.ring.tutti_kv_save_layer(fw + l0 * per_w, g * per_w, self.duplex_save_sms, stream=sW)
             saved = torch.cuda.Event()
             saved.record(sW)
-            self.saved_ev[l] = saved
-            issued += [(fr, nr), (fw, nw)]
+            self.saved_ev[l0] = saved
+        if times is not None:
+            for key, st in (("r1", sR), ("w1", sW)):
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record(st)
+                times.setdefault(key, []).append(ev)
         total = self.poll_list(self.unpolled)
-        self.unpolled = issued
+        self.unpolled = [(fr, L * per_r), (fw, L * per_w)]
         return total
 
     def finish_duplex(self):
@@ -728,18 +737,23 @@ def run_e2e(args, local_rank, world):
     a2 = argparse.Namespace(**vars(args))
     L_host = min(args.e2e_host_layers, 32)
     a2.resident_layers = L_host
+    a2.layers_per_launch = 4
     rep = Replica(a2, local_rank, host_store=True, n_layers=L_host)
     passes = max(1, 32 // L_host) if args.config in (2, 5) else 1
     duplex = not args.e2e_serial
     if duplex:
         rep.ctx.tutti_set_option(rep.T.OPT_COPY_ENGINE, rep.T.ENGINE_BULK)
+    times = {}
 
     def one_pass():
-        return rep.step_duplex(upload_tables=True) if duplex else rep.step(upload_tables=True)
+        if duplex:
+            return rep.step_duplex(upload_tables=True, group=args.e2e_group, times=times)
+        return rep.step(upload_tables=True)
     one_pass()
     if duplex:
         rep.finish_duplex()
     torch.cuda.synchronize()
+    times.clear()
     barrier(world)
     steps = max(1, min(args.steps, 3))
     t0 = time.perf_counter()
@@ -759,19 +773,35 @@ def run_e2e(args, local_rank, world):
     payload = 2 * layers * rep.payload_per_layer
     assert moved == payload * steps, (moved, payload * steps)
     ok = rep.spot_check(64)
+    per_dir = None
+    if duplex and times:
+        # each direction's own rate: its bytes over the time its stream was busy with them
+        per_dir = {}
+        for key, a, b in (("restore_gbs", "r0", "r1"), ("save_gbs", "w0", "w1")):
+            busy = times[a][0].elapsed_time(times[b][-1])
+            per_dir[key] = round(steps * layers * rep.payload_per_layer / (busy * 1e-3) / 1e9, 2)
+    link = host_link_gbs(rep.dev) if world == 1 else None
     link_duplex = host_link_duplex_gbs(rep.dev) if world == 1 else None
     h2d = layers * rep.payload_per_layer + passes * rep.table_bytes
     d2h = layers * rep.payload_per_layer + 2 * layers * 32
     value = sum_over_ranks(float(payload), world, rep.dev) / (ms * 1e-3) / 1e9
     rep.close()
-    return {"value": round(value, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
-            "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms, 2),
-            "spot_check": bool(ok),
-            "host_link_duplex_gbs": None if link_duplex is None else round(link_duplex, 1),
-            "mode": "duplex: layer l saved while layer l+1 is restored (both directions of the "
-                    "host link busy)" if duplex else "serial: all restores, then all saves",
-            "store": f"pinned host memory, zero-copy; {L_host} layers resident, "
-                     f"{passes} passes per step = {layers} layer transfers each way"}
+    out = {"value": round(value, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms, 2),
+           "spot_check": bool(ok),
+           "host_link_duplex_gbs": None if link_duplex is None else round(link_duplex, 1),
+           "link_frac": None if link_duplex is None else round(value / link_duplex, 4),
+           "mode": f"duplex: groups of {args.e2e_group} layers saved while the next group is "
+                   f"restored (both directions of the host link busy); restore on "
+                   f"{rep.duplex_sms} SMs, save on {rep.duplex_save_sms} SMs"
+                   if duplex else "serial: all restores, then all saves",
+           "store": f"pinned host memory, zero-copy; {L_host} layers resident, "
+                    f"{passes} passes per step = {layers} layer transfers each way"}
+    if per_dir:
+        out.update(per_dir)
+    if link is not None:
+        out["host_link_h2d_gbs"], out["host_link_d2h_gbs"] = round(link[0], 2), round(link[1], 2)
+    return out
 
 
 def host_link_gbs(dev, nbytes=1 << 30, reps=10):
@@ -1230,10 +1260,12 @@ def main():
     ap.add_argument("--claim", type=int, default=0)
     ap.add_argument("--bulk-chunk", type=int, default=0)
     ap.add_argument("--e2e-host-layers", type=int, default=8)
-    ap.add_argument("--e2e-sms", type=int, default=8,
-                    help="e2e leg, duplex mode: SMs per direction")
-    ap.add_argument("--e2e-save-sms", type=int, default=0,
-                    help="e2e leg, duplex mode: SMs of the save direction (default: same)")
+    ap.add_argument("--e2e-sms", type=int, default=12,
+                    help="e2e leg, duplex mode: SMs of the restore direction")
+    ap.add_argument("--e2e-save-sms", type=int, default=8,
+                    help="e2e leg, duplex mode: SMs of the save direction")
+    ap.add_argument("--e2e-group", type=int, default=2,
+                    help="e2e leg, duplex mode: layers per copy launch")
     ap.add_argument("--e2e-serial", action="store_true",
                     help="e2e leg: restore pass then save pass instead of overlapping them")
     ap.add_argument("--gemm-iters", type=int, default=20)
@@ -1262,15 +1294,21 @@ def main():
                     help="skip the config 1/3/4/5 legs of the default line")
     ap.add_argument("--no-sched", action="store_true", help="skip the scheduler legs")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-only", action="store_true", help="run the end-to-end leg on its own")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.sched_demo or args.sweep_length or args.config != 2:
+    elif args.sched_demo or args.sweep_length or args.e2e_only or args.config != 2:
         # a single leg on its own (one GPU)
         rank, local_rank, world = init_dist("nccl")
         if args.sweep_length:
             run_length_sweep(args)
+            return
+        if args.e2e_only:
+            res = run_e2e(args, local_rank, world)
+            if rank == 0:
+                print(json.dumps(res), flush=True)
             return
         leg = (leg_sched_demo if args.sched_demo else
                {1: leg_config1, 3: leg_config3, 4: leg_config4, 5: leg_config5}[args.config])

@@ -273,6 +273,20 @@ int tutti_kv_save_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t first_ioc
 int tutti_ring_poll(tutti_ring_t *ring, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns);
 
 /*
+ * wait_cqe for a run of IOCBs (a layer's, or a whole pass's): polls first_iocb,
+ * first_iocb + 1, ... in order, as tutti_ring_poll does, with one budget of timeout_ns for
+ * all of them (0 never blocks).  TUTTI_OK when all n_iocb have completed (and are released);
+ * otherwise the code of the poll that stopped the walk (TUTTI_EAGAIN: that IOCB has not
+ * completed in time; TUTTI_EINVAL: not a live index) — the IOCBs before it were consumed, so
+ * the caller resumes at first_iocb + *n_done.  Host out (each may be NULL): *bytes_total sum
+ * of the completions' bytes, *first_error status of the first completion that carried one
+ * (0 if none), *n_done completions consumed by this call.
+ */
+int tutti_ring_poll_range(tutti_ring_t *ring, uint32_t first_iocb, uint32_t n_iocb,
+                          uint64_t *bytes_total, int32_t *first_error, uint32_t *n_done,
+                          uint64_t timeout_ns);
+
+/*
  * GPU-side dependency on one IOCB (Section 3.2: once enqueued, "GPU-side dependency
  * tracking" orders I/O and compute without the CPU): everything enqueued on `stream`
  * after this call starts only once IOCB iocb_idx has completed — for instance a layer's

@@ -115,18 +115,73 @@ __device__ void complete_empty(const RingDev &ring, IocbHdr *h, uint32_t idx) {
         post_cqe(ring, idx, h->status, 0);
 }
 
+constexpr int BULK_MAX_STAGES = 8;
+
+// Geometry of the chunks of one IOCB with uniform entry length.
+struct ChunkGeom {
+    uint32_t elen;       // entry length
+    uint32_t per_chunk;  // entries per chunk when elen <= chunk bytes (1..32), else 0
+    uint32_t pieces;     // pieces per entry when elen > chunk bytes, else 0
+    uint32_t n_chunks;
+    uint32_t total;
+};
+
+__device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen, uint32_t CB) {
+    ChunkGeom g;
+    g.elen = elen;
+    g.total = total;
+    if (elen <= CB) {
+        uint32_t pc = CB / elen;
+        g.per_chunk = pc > 32 ? 32 : pc;
+        g.pieces = 0;
+        g.n_chunks = (total + g.per_chunk - 1) / g.per_chunk;
+    } else {
+        g.per_chunk = 0;
+        g.pieces = (elen + CB - 1) / CB;
+        g.n_chunks = total * g.pieces;
+    }
+    return g;
+}
+
+
+// Number of claim units (what claim_cursor counts) of a published IOCB under this launch's
+// engine: tiles / chunks for uniform entries, entries for the per-entry paths.  0xffffffff for
+// an IOCB the engine will refuse (it must be opened, not skipped).  `bulk_chunk` is the bulk
+// engine's stage size, 0 for the ldst engine; `tm_valid` says whether head-major blocks can be
+// staged.  The copy loops use the very same function, so a look-ahead that skips IOCBs whose
+// cursor has passed this count can never skip unclaimed work.
+__device__ __forceinline__ uint32_t claim_units(const IocbHdr *h, const PermGeom &perm,
+                                                uint32_t bulk_chunk, bool tm_valid) {
+    const uint32_t total = h->total_entries, elen = h->entry_len;
+    const bool hnd = (h->opcode & TUTTI_OP_FLAG_HND) != 0;
+    if (hnd && (elen == 0 || elen != perm.block_tokens * perm.token_bytes)) return 0xffffffffu;
+    if (bulk_chunk) {
+        const bool hnd_staged = hnd && elen <= bulk_chunk && tm_valid && perm.n_heads <= 32;
+        if (elen == 0 || (hnd && !hnd_staged)) return total;      // per-entry vector path
+        if (hnd_staged) return total;                              // one block per stage
+        return chunk_geom(total, elen, bulk_chunk).n_chunks;
+    }
+    if (elen != 0 && (elen & 511u) == 0)
+        return (uint32_t)(((unsigned long long)total * elen + CHUNK_BYTES - 1) / CHUNK_BYTES);
+    return total;
+}
+
 // Warp-collective look-ahead over the IOCBs [bi, n_iocb) of a launch: 32 headers are read at
 // a time, and the leading ones that need no copying — already complete, or published with
 // nothing to move (the unused tail of a build's reservation, or a build error) — are
-// skipped without a round trip each.  The `designated` warp (one per launch) completes
-// the published-but-empty ones, one lane per IOCB.  Returns the first IOCB that is either
-// not published yet or has bytes to move (n_iocb if none).
+// skipped without a round trip each; so are IOCBs whose work has all been claimed already
+// (many small IOCBs in one launch: an agent does not open what others are finishing).  The
+// `designated` warp (one per launch) completes the published-but-empty ones, one lane per
+// IOCB.  Returns the first IOCB that is either not published yet or has unclaimed work
+// (n_iocb if none).
 __device__ uint32_t skip_idle_iocbs(const RingDev &ring, uint32_t first_iocb, uint32_t bi,
-                                    uint32_t n_iocb, bool designated) {
+                                    uint32_t n_iocb, bool designated, const PermGeom &perm,
+                                    uint32_t bulk_chunk, bool tm_valid, bool *ready_out = nullptr) {
     const uint32_t lane = threadIdx.x & 31;
+    bool ready_seen = false;
     while (bi < n_iocb) {
         const uint32_t k = bi + lane;
-        bool idle = false, empty_ready = false;
+        bool idle = false, empty_ready = false, ready = false;
         IocbHdr *h = nullptr;
         uint32_t idx = first_iocb + k;
         if (k < n_iocb) {
@@ -135,16 +190,25 @@ __device__ uint32_t skip_idle_iocbs(const RingDev &ring, uint32_t first_iocb, ui
             if (st == state_word(idx, PHASE_DONE)) {
                 idle = true;
             } else if (st == state_word(idx, PHASE_READY)) {
+                ready = true;
                 empty_ready = (h->total_entries == 0 || h->status != 0);
-                idle = empty_ready;
+                // every unit already claimed by other agents: nothing left to take here
+                idle = empty_ready ||
+                       *((volatile uint32_t *)&h->claim_cursor) >= claim_units(h, perm, bulk_chunk, tm_valid);
             }
         }
         const uint32_t mask = __ballot_sync(0xffffffffu, idle);
         const uint32_t lead = (mask == 0xffffffffu) ? 32u : (uint32_t)(__ffs(~mask) - 1);
         if (designated && empty_ready && lane < lead) complete_empty(ring, h, idx);
         bi += lead;
-        if (lead < 32u) break;
+        if (lead < 32u) {
+            // the IOCB the walk stops at was seen published (acquire): no second look needed
+            ready_seen = __shfl_sync(0xffffffffu, ready, lead);
+            __syncwarp();       // the other lanes read that header after this lane's acquire
+            break;
+        }
     }
+    if (ready_out) *ready_out = ready_seen && bi < n_iocb;
     return bi < n_iocb ? bi : n_iocb;
 }
 
@@ -199,7 +263,8 @@ copy_ldst_kernel(CopyParams p) {
     for (uint32_t bi = 0; bi < p.n_iocb; ++bi) {
         // warp 0 looks ahead past IOCBs that need no copying
         if (warp == 0) {
-            uint32_t nb = skip_idle_iocbs(p.ring, p.first_iocb, bi, p.n_iocb, blockIdx.x == 0 && grp == 0);
+            uint32_t nb = skip_idle_iocbs(p.ring, p.first_iocb, bi, p.n_iocb, blockIdx.x == 0 && grp == 0,
+                                          p.perm, 0, false);
             if (lane == 0) s_bi = nb;
         }
         group_sync(grp);
@@ -237,7 +302,7 @@ copy_ldst_kernel(CopyParams p) {
         if (elen != 0 && (elen & 511u) == 0) {
             // uniform entries, every 512-byte warp row lies inside one entry
             const unsigned long long total_bytes = (unsigned long long)total * elen;
-            const uint32_t n_tiles = (uint32_t)((total_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
+            const uint32_t n_tiles = claim_units(h, p.perm, 0, false);
             const bool pow2 = (elen & (elen - 1)) == 0;
             const uint32_t shift = 31 - __clz(elen);
             for (;;) {
@@ -430,34 +495,6 @@ __device__ __forceinline__ void tensor_s2g(const CUtensorMap *map, uint32_t head
         : "memory");
 }
 
-constexpr int BULK_MAX_STAGES = 8;
-
-// Geometry of the chunks of one IOCB with uniform entry length.
-struct ChunkGeom {
-    uint32_t elen;       // entry length
-    uint32_t per_chunk;  // entries per chunk when elen <= chunk bytes (1..32), else 0
-    uint32_t pieces;     // pieces per entry when elen > chunk bytes, else 0
-    uint32_t n_chunks;
-    uint32_t total;
-};
-
-__device__ __forceinline__ ChunkGeom chunk_geom(uint32_t total, uint32_t elen, uint32_t CB) {
-    ChunkGeom g;
-    g.elen = elen;
-    g.total = total;
-    if (elen <= CB) {
-        uint32_t pc = CB / elen;
-        g.per_chunk = pc > 32 ? 32 : pc;
-        g.pieces = 0;
-        g.n_chunks = (total + g.per_chunk - 1) / g.per_chunk;
-    } else {
-        g.per_chunk = 0;
-        g.pieces = (elen + CB - 1) / CB;
-        g.n_chunks = total * g.pieces;
-    }
-    return g;
-}
-
 // Each warp of the CTA is an independent agent with its own ring of stages, fed by a
 // stream of chunks that runs across the IOCBs of the launch without draining in between.
 // Shared memory: [warps][stages][chunk bytes] data, [warps][stages] mbarriers, then per
@@ -496,6 +533,9 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
 
     // ---- source side of the stream: the IOCB chunks are being claimed from
     uint32_t f_bi = 0;                      // next IOCB of the launch to open
+    uint32_t f_start = 0, f_limit = p.n_iocb;   // starting point and end of the current sweep
+    uint32_t claim = p.claim_chunks;            // chunks per work claim of this agent
+    bool f_wrapped = false;
     IocbHdr *f_h = nullptr;
     ChunkGeom cg{0, 0, 0, 0, 0};
     const tutti_sgl_t *sgl = nullptr;
@@ -559,17 +599,30 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
 
     // Open the next IOCB that has staged work; false when the launch has none left.
     auto open_next_iocb = [&]() -> bool {
-        while (f_bi < p.n_iocb) {
-            f_bi = skip_idle_iocbs(p.ring, p.first_iocb, f_bi, p.n_iocb,
-                                   blockIdx.x == 0 && warp == 0);
-            if (f_bi >= p.n_iocb) break;
+        for (;;) {
+            if (f_bi >= f_limit) {
+                // end of the launch's IOCBs: an agent that did not start at the first one goes
+                // round once, over the IOCBs before its starting point
+                if (f_wrapped || f_start == 0) break;
+                f_wrapped = true;
+                f_bi = 0;
+                f_limit = f_start;
+                continue;
+            }
+            bool seen_ready = false;
+            f_bi = skip_idle_iocbs(p.ring, p.first_iocb, f_bi, f_limit,
+                                   blockIdx.x == 0 && warp == 0, p.perm, CB, tm.valid != 0,
+                                   &seen_ready);
+            if (f_bi >= f_limit) continue;
             const uint32_t bi = f_bi++;
             const uint32_t idx = p.first_iocb + bi;
             IocbHdr *h = hdr_of(bi);
-            int mode = 0;
-            if (lane == 0) mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
-            mode = __shfl_sync(0xffffffffu, mode, 0);
-            if (mode == IOCB_SKIP) continue;
+            if (!seen_ready) {
+                int mode = 0;
+                if (lane == 0) mode = wait_iocb_ready(p.ring, h, idx, p.wait_ns);
+                mode = __shfl_sync(0xffffffffu, mode, 0);
+                if (mode == IOCB_SKIP) continue;
+            }
             const uint32_t total = h->total_entries;
             if (total == 0 || h->status != 0) {
                 if (lane == 0) complete_empty(p.ring, h, idx);
@@ -597,13 +650,43 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
             f_cur_bi = bi;
             f_hnd = hnd_staged;
             cg = chunk_geom(total, h->entry_len, CB);
-            if (f_hnd) { cg.per_chunk = 1; cg.n_chunks = total; }   // one block per stage
+            if (f_hnd) cg.per_chunk = 1;                            // one block per stage
+            cg.n_chunks = claim_units(h, p.perm, CB, tm.valid != 0);
             cur = cur_end = 0;
-            if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, p.claim_chunks);
+            if (lane == 0) pending_claim = atomicAdd(&h->claim_cursor, claim);
             return true;
         }
         return false;
     };
+
+    // A launch of many small IOCBs (a whole pass of a short prefix): opening an IOCB costs a
+    // few dependent round trips, so an agent should not have to open many for its share of the
+    // work, and the agents should not all queue up at the first one.  With the first IOCB's
+    // size as the estimate of all of them, a claim grows to about half an agent's share of the
+    // launch (never beyond the option's value when one IOCB alone can feed every agent), and
+    // agent a starts at the IOCB that this claim size assigns to it, walking on cyclically.
+    if (p.n_iocb > 1) {
+        uint32_t start = 0, cl = claim;
+        if (lane == 0) {
+            IocbHdr *h0 = hdr_of(0);
+            if (ld_acquire_u32(&h0->state) == state_word(p.first_iocb, PHASE_READY) &&
+                h0->total_entries != 0 && h0->status == 0) {
+                const uint32_t u = claim_units(h0, p.perm, CB, tm.valid != 0);
+                const uint32_t n_agents = gridDim.x * n_warps;
+                if (u != 0xffffffffu && u / claim < n_agents) {
+                    const unsigned long long share =
+                        ((unsigned long long)u * p.n_iocb + n_agents - 1) / n_agents;
+                    const unsigned long long half = (share + 1) / 2;
+                    if (half > cl) cl = (uint32_t)(half < u ? half : u);
+                    const uint32_t per = u / cl + (u % cl != 0);       // agents one IOCB feeds
+                    const uint32_t agent = warp * gridDim.x + blockIdx.x;
+                    start = min(agent / per, p.n_iocb - 1);
+                }
+            }
+        }
+        f_start = f_bi = __shfl_sync(0xffffffffu, start, 0);
+        claim = __shfl_sync(0xffffffffu, cl, 0);
+    }
 
     // Work claims are taken one ahead of need (the atomic's latency hides behind the
     // copies of the current claim), and the addresses of the next chunk are fetched as
@@ -619,8 +702,8 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
                 uint32_t c0 = __shfl_sync(0xffffffffu, pending_claim, 0);
                 if (c0 >= cg.n_chunks) { f_open = false; continue; }
                 cur = c0;
-                cur_end = min(c0 + p.claim_chunks, cg.n_chunks);
-                if (lane == 0) pending_claim = atomicAdd(&f_h->claim_cursor, p.claim_chunks);
+                cur_end = min(c0 + claim, cg.n_chunks);
+                if (lane == 0) pending_claim = atomicAdd(&f_h->claim_cursor, claim);
             }
             break;
         }

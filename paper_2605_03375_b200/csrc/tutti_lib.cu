@@ -587,6 +587,33 @@ int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64
     }
 }
 
+int tutti_ring_poll_range(tutti_ring_t *r, uint32_t first_iocb, uint32_t n_iocb, uint64_t *bytes_total,
+                          int32_t *first_error, uint32_t *n_done, uint64_t timeout_ns) {
+    if (!r || n_iocb == 0 || n_iocb > r->dev.depth) return TUTTI_EINVAL;
+    uint64_t bytes = 0;
+    int32_t err = 0;
+    uint32_t done = 0;
+    int rc = TUTTI_OK;
+    auto t0 = std::chrono::steady_clock::now();
+    for (; done < n_iocb; ++done) {
+        uint64_t left = 0;
+        if (timeout_ns) {
+            auto dt = std::chrono::duration_cast<std::chrono::nanoseconds>(
+                          std::chrono::steady_clock::now() - t0).count();
+            left = (uint64_t)dt < timeout_ns ? timeout_ns - (uint64_t)dt : 1;
+        }
+        tutti_cqe_t c;
+        rc = tutti_ring_poll(r, first_iocb + done, &c, left);
+        if (rc != TUTTI_OK) break;
+        bytes += c.bytes;
+        if (c.status != 0 && err == 0) err = c.status;
+    }
+    if (bytes_total) *bytes_total = bytes;
+    if (first_error) *first_error = err;
+    if (n_done) *n_done = done;
+    return rc;
+}
+
 int tutti_stream_wait_iocb(tutti_ring_t *r, uint32_t iocb_idx, void *stream) {
     if (!r || !r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
     r->host_calls++;

@@ -79,7 +79,7 @@ EXPORTS = [
     "tutti_filepool_create", "tutti_filepool_destroy", "tutti_filepool_insert",
     "tutti_filepool_lookup", "tutti_filepool_match_prefix", "tutti_filepool_pin",
     "tutti_filepool_remove", "tutti_filepool_stats", "tutti_build_sqes_layers",
-    "tutti_stream_wait_iocb", "tutti_ring_last_launch_sms",
+    "tutti_stream_wait_iocb", "tutti_ring_last_launch_sms", "tutti_ring_poll_range",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -105,6 +105,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_kv_save_layer": (C.c_int, [vp, vp, u32, u32, u32, vp]),
         "tutti_ring_poll": (C.c_int, [vp, u32, P(Cqe), u64]),
         "tutti_stream_wait_iocb": (C.c_int, [vp, u32, vp]),
+        "tutti_ring_poll_range": (C.c_int, [vp, u32, u32, P(u64), P(C.c_int32), P(u32), u64]),
         "tutti_ctx_create": (C.c_int, [P(Geom), C.c_int, P(vp)]),
         "tutti_ctx_destroy": (C.c_int, [vp]),
         "tutti_pool_register": (C.c_int, [vp, u32, vp, vp, u64, u64]),
@@ -299,6 +300,15 @@ class Ring:
         rc = self.lib.tutti_ring_poll(self.h, iocb_idx, C.byref(cqe), timeout_ns)
         _check(rc, "tutti_ring_poll", (EAGAIN, EINVAL))
         return rc, cqe
+
+    def tutti_ring_poll_range(self, first_iocb: int, n_iocb: int, timeout_ns: int = 0
+                              ) -> Tuple[int, int, int, int]:
+        """(rc, bytes_total, first_error, n_done) for the IOCBs [first_iocb, first_iocb + n_iocb)."""
+        b, e, n = C.c_uint64(), C.c_int32(), C.c_uint32()
+        rc = self.lib.tutti_ring_poll_range(self.h, first_iocb, n_iocb, C.byref(b), C.byref(e),
+                                            C.byref(n), timeout_ns)
+        _check(rc, "tutti_ring_poll_range", (EAGAIN, EINVAL))
+        return rc, b.value, e.value, n.value
 
     def tutti_stream_wait_iocb(self, iocb_idx: int, stream, allow: Sequence[int] = ()) -> int:
         """Work enqueued on `stream` after this call starts once the IOCB has completed."""

@@ -296,3 +296,45 @@ def test_mixed_hbm_and_pinned_host_storage_devices(hnd):
             assert np.array_equal(t.cpu().numpy(), s)
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
+@pytest.mark.parametrize("sm_count", [0, 8])
+@pytest.mark.parametrize("tokens", [1024, 4096 + 256 + 16])
+def test_whole_pass_of_a_short_prefix_in_one_launch(engine, sm_count, tokens):
+    """32 layers of a short prefix built by one launch and executed by one copy launch (both
+    directions): many small IOCBs, over which the copy agents spread instead of queueing at
+    the first one.  Completions are consumed with one tutti_ring_poll_range call."""
+    w = wl.config(2, 1.0, n_layers=32, hit_tokens=[tokens])
+    dc = DeviceCase(w, depth=64, capacity=2048, sgl_capacity=2 * len(w.block_ids) * 33)
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+        rc, first, per = dc.ring.tutti_build_sqes_layers(dc.batch, 0, 32, T.OP_READ)
+        assert per == 1
+        assert dc.ring.tutti_ring_poll_range(first, 32)[0] == T.EAGAIN      # nothing issued yet
+        dc.ring.tutti_kv_restore_layer(first, 32, sm_count)
+        rc, nbytes, err, done = dc.ring.tutti_ring_poll_range(first, 32, 5_000_000_000)
+        assert (rc, err, done) == (T.OK, 0, 32)
+        assert nbytes == 32 * tokens * 2 * int(dc.ctx.layout.token_bytes)
+        assert dc.ring.tutti_ring_poll_range(first, 1)[0] == T.EINVAL       # released: no longer live
+        want = {}
+        for layer in (0, 1, 13, 31):
+            want[layer] = dc.oracle_restore(layer)
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want[layer])
+        for t in dc.store_dev:
+            t.zero_()
+        rc, first, per = dc.ring.tutti_build_sqes_layers(dc.batch, 0, 32, T.OP_WRITE)
+        dc.ring.tutti_kv_save_layer(first, 32, sm_count)
+        rc, nbytes, err, done = dc.ring.tutti_ring_poll_range(first, 32, 5_000_000_000)
+        assert (rc, err, done) == (T.OK, 0, 32)
+        torch.cuda.synchronize()
+        st = [np.zeros_like(s) for s in dc.store_host]
+        for layer in range(32):
+            pool = want.get(layer)
+            if pool is None:
+                pool = dc.oracle_restore(layer)
+            dc.oracle_save(layer, pool, st)
+        for t, s in zip(dc.store_dev, st):
+            assert np.array_equal(t.cpu().numpy(), s)
+    finally:
+        dc.close()

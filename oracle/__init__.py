@@ -25,6 +25,7 @@ OK, EINVAL, ENOSPC = 0, -1, -2
 FILE_MAJOR, LAYER_MAJOR = 0, 1
 OP_READ, OP_WRITE = 0, 1
 OP_HND = 0x100       # opcode flag: head-major pool blocks
+SGL_DUP = 0x80000000  # SGL identifier flag: same object bytes as the entry before
 
 
 def build(force: bool = False) -> str:

@@ -35,9 +35,13 @@
  *
  * The paper gives no sorting/coalescing rule (only the motivation that small
  * scattered requests waste bandwidth, Section 2.3/2.4); the rule used here is
- * the reading recorded in the design notes: order by (device, offset), merge
- * exactly byte-adjacent neighbours on one device, stable on (request, chunk,
- * K-before-V).
+ * the reading recorded in the design notes: order by (device, offset, length), stable
+ * on (request, chunk, K-before-V); items that name exactly the same bytes (a stored
+ * chunk shared by several requests of the batch, Section 3.1 "Scalable GPU File
+ * Pool") form one source that is read once: its scatter-gather entries list, block
+ * by block, every request's destination, the second and later ones flagged as
+ * repeats; distinct sources that are exactly byte-adjacent on one device merge into
+ * one context.
  *
  * Parity pins (tests/test_oracle_*.py): brute force on tiny pools against an
  * independent Python byte loop, array-shaped (numpy advanced indexing)
@@ -60,6 +64,9 @@
 #define ORC_OP_READ 0  /* object store -> paged pool (restore) */
 #define ORC_OP_WRITE 1 /* paged pool -> object store (save)    */
 #define ORC_OP_HND 0x100 /* flag: pool blocks are [head][token][dim] instead of [token][head][dim] */
+/* Flag in the identifier of a scatter-gather entry: this entry takes (READ) the same object
+ * bytes as the entry before it, i.e. one stored chunk goes to several requests' blocks. */
+#define ORC_SGL_DUP 0x80000000u
 
 typedef struct {
     uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
@@ -293,6 +300,9 @@ static int item_cmp(const void *pa, const void *pb)
     const item_t *a = (const item_t *)pa, *b = (const item_t *)pb;
     if (a->dev != b->dev) return a->dev < b->dev ? -1 : 1;
     if (a->src_off != b->src_off) return a->src_off < b->src_off ? -1 : 1;
+    /* items that start at the same byte: the shorter (a prefix ending inside the object)
+     * first, so that items naming exactly the same bytes end up next to each other */
+    if (a->len != b->len) return a->len < b->len ? -1 : 1;
     /* equal keys keep generation order: this makes qsort behave as a stable sort */
     if (a->seq != b->seq) return a->seq < b->seq ? -1 : 1;
     return 0;
@@ -346,15 +356,23 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
         }
     }
 
-    /* step 2: order by (device, offset), stable */
+    /* step 2: order by (device, offset, length), stable */
     qsort(items, n_items, sizeof(item_t), item_cmp);
 
-    /* step 3 + 4: sweep, merging exactly adjacent neighbours; emit SGL entries */
+    /* step 3 + 4: sweep over the distinct sources.  A group = an item and the items right
+     * after it that name exactly the same bytes (same device, offset and length).  A group
+     * opens a new context unless it starts where the previous group's bytes end; its SGL
+     * entries go block by block, and for each block one entry per member of the group, in
+     * sorted order, all but the first flagged as repeats of the bytes just named. */
     uint32_t ns = 0, ne = 0;
-    for (uint64_t i = 0; i < n_items; ++i) {
+    const item_t *prev = NULL; /* first item of the previous group */
+    for (uint64_t i = 0; i < n_items;) {
         const item_t *it = &items[i];
-        int fresh = (i == 0) || items[i - 1].dev != it->dev ||
-                    items[i - 1].src_off + items[i - 1].len != it->src_off;
+        uint64_t k = 1;
+        while (i + k < n_items && items[i + k].dev == it->dev &&
+               items[i + k].src_off == it->src_off && items[i + k].len == it->len)
+            ++k;
+        int fresh = !prev || prev->dev != it->dev || prev->src_off + prev->len != it->src_off;
         if (fresh) {
             if (ns >= max_sqe) { free(items); return ORC_ENOSPC; }
             orc_sqe *s = &sqes[ns++];
@@ -367,17 +385,22 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
             s->layer = (uint16_t)layer;
         }
         orc_sqe *s = &sqes[ns - 1];
-        s->len += it->len;
-        s->sgl_count += it->n_blk;
+        s->len += it->len;                       /* the bytes are named once */
+        s->sgl_count += (uint32_t)(k * it->n_blk);
         for (uint32_t j = 0; j < it->n_blk; ++j) {
-            if (ne >= max_sgl) { free(items); return ORC_ENOSPC; }
-            int32_t id = block_ids[blk_start[it->r] + (uint64_t)it->c * lo.blocks_per_obj + j];
-            if (id < 0) { free(items); return ORC_EINVAL; }
-            sgl[ne].addr = (it->kv ? v_base_addr : k_base_addr) + (uint64_t)id * block_stride;
-            sgl[ne].len = (uint32_t)lo.block_bytes;
-            sgl[ne].id = (uint32_t)id;
-            ++ne;
+            for (uint64_t c = 0; c < k; ++c) {
+                const item_t *m = &items[i + c];
+                if (ne >= max_sgl) { free(items); return ORC_ENOSPC; }
+                int32_t id = block_ids[blk_start[m->r] + (uint64_t)m->c * lo.blocks_per_obj + j];
+                if (id < 0) { free(items); return ORC_EINVAL; }
+                sgl[ne].addr = (m->kv ? v_base_addr : k_base_addr) + (uint64_t)id * block_stride;
+                sgl[ne].len = (uint32_t)lo.block_bytes;
+                sgl[ne].id = (uint32_t)id | (c ? ORC_SGL_DUP : 0u);
+                ++ne;
+            }
         }
+        prev = it;
+        i += k;
     }
     free(items);
 
@@ -398,7 +421,8 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
 /*
  * Execute descriptors: for each context, walk its SGL entries with a cursor
  * on the object side.  READ moves object bytes to the entry's address, WRITE
- * the other way.  Pool addresses are translated to the host copy of the pool
+ * the other way.  An entry flagged as a repeat uses the object bytes of the entry
+ * before it and does not advance the cursor.  Pool addresses are translated to the host copy of the pool
  * by  host = pool_host + (addr - pool_base_addr).
  */
 int orc_exec(const orc_sqe *sqes, uint32_t n_sqe, const orc_sgl *sgl, uint32_t n_sgl,
@@ -411,13 +435,20 @@ int orc_exec(const orc_sqe *sqes, uint32_t n_sqe, const orc_sgl *sgl, uint32_t n
         if (s->dev >= n_devices) return ORC_EINVAL;
         if ((uint64_t)s->sgl_first + s->sgl_count > n_sgl) return ORC_EINVAL;
         int to_pool = (s->opcode & 0xff) == ORC_OP_READ;
-        uint64_t cursor = s->src_off;
+        uint64_t cursor = s->src_off, at = s->src_off;
         for (uint32_t e = s->sgl_first; e < s->sgl_first + s->sgl_count; ++e) {
             if (sgl[e].addr < pool_base_addr) return ORC_EINVAL;
             uint64_t poff = sgl[e].addr - pool_base_addr;
             if (poff + sgl[e].len > pool_bytes) return ORC_EINVAL;
-            if (cursor + sgl[e].len > store_bytes[s->dev]) return ORC_EINVAL;
-            uint8_t *obj = store[s->dev] + cursor, *blk = pool_host + poff;
+            if (sgl[e].id & ORC_SGL_DUP) {
+                /* the bytes of the entry before: the cursor stays where it is */
+                if (e == s->sgl_first || sgl[e].len != sgl[e - 1].len) return ORC_EINVAL;
+            } else {
+                at = cursor;
+                cursor += sgl[e].len;
+            }
+            if (at + sgl[e].len > store_bytes[s->dev]) return ORC_EINVAL;
+            uint8_t *obj = store[s->dev] + at, *blk = pool_host + poff;
             if (!(s->opcode & ORC_OP_HND)) {
                 if (to_pool) memcpy(blk, obj, sgl[e].len); else memcpy(obj, blk, sgl[e].len);
             } else {
@@ -433,7 +464,6 @@ int orc_exec(const orc_sqe *sqes, uint32_t n_sqe, const orc_sgl *sgl, uint32_t n
                         if (to_pool) memcpy(q, o, row_bytes); else memcpy(o, q, row_bytes);
                     }
             }
-            cursor += sgl[e].len;
         }
         if (cursor - s->src_off != s->len) return ORC_EINVAL;
     }

@@ -235,7 +235,7 @@ def make_workload(name: str, *, seed: int, n_layers: int, hit_tokens, block_toke
                   pool_round: int = 1024, pool_interleaved: bool = False,
                   store_kind: str = "hbm", n_pool_blocks: Optional[int] = None,
                   consecutive_slots: bool = False, pool_hnd: bool = False,
-                  pool_pad_bytes: int = 0) -> Workload:
+                  pool_pad_bytes: int = 0, shared_prefix_frac: float = 0.0) -> Workload:
     rng = np.random.default_rng(seed)
     hit = np.asarray(hit_tokens, dtype=np.uint32)
     assert np.all(hit % block_tokens == 0)
@@ -262,6 +262,12 @@ def make_workload(name: str, *, seed: int, n_layers: int, hit_tokens, block_toke
         n_slots = max(int(math.ceil(n_obj * slot_space_factor)), 1)
         n_slots = ((n_slots + n_devices - 1) // n_devices) * n_devices
         per_req = _assign_slots(rng, [int(k) for k in objs], n_slots, slot_mean_run)
+    if shared_prefix_frac > 0.0 and len(per_req) > 1:
+        # requests with a common prefix: the leading objects of every request are the very
+        # objects of request 0 (stored once, shared by all), the rest stays private
+        n_share = int(min(len(p) for p in per_req) * shared_prefix_frac)
+        for p in per_req[1:]:
+            p[:n_share] = per_req[0][:n_share]
     obj_slot = np.concatenate(per_req) if per_req else np.zeros(0, dtype=np.uint32)
     return Workload(name=name, seed=seed, n_layers=n_layers, n_kv_heads=n_kv_heads,
                     head_dim=head_dim, elem_bytes=elem_bytes, block_tokens=block_tokens,

@@ -361,6 +361,76 @@ def test_descriptors(case, capacity):
         assert np.array_equal(a, b)
 
 
+SHARED = [
+    dict(index=2, scale=0.05, n_layers=2, shared_prefix_frac=0.75),
+    dict(index=2, scale=0.05, n_layers=2, shared_prefix_frac=1.0, n_devices=2,
+         layout=wl.LAYOUT_FILE_MAJOR),
+    dict(index=4, scale=0.04, n_layers=2, shared_prefix_frac=1.0),
+    dict(index=2, scale=0.05, n_layers=2, shared_prefix_frac=0.75, pool_hnd=True),
+]
+
+
+@pytest.mark.parametrize("case", SHARED, ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
+@pytest.mark.parametrize("capacity", [2048, 3])
+def test_descriptors_of_requests_with_a_shared_prefix(case, capacity):
+    """Several requests of a batch hit the same stored objects: each distinct source is named
+    once, every destination still appears exactly once, and executing the descriptors is the
+    plain restore."""
+    w, g, lo = _mk(case)
+    nbytes, k_off, v_off, stride = hc.pool_geometry(w, lo)
+    base = 0x7F0000000000
+    layer = w.n_layers - 1
+    batch = hc.batch_of(w)
+    flag = oracle.OP_HND if w.pool_hnd else 0
+    rowb = w.head_dim * w.elem_bytes
+    rc, sqes, sgl, num = oracle.build_descriptors(g, layer, oracle.OP_READ | flag, batch,
+                                                  base + k_off, base + v_off, stride, capacity)
+    assert rc == 0
+    tb, bb = int(lo.token_bytes), int(lo.block_bytes)
+    # distinct sources, counted from the inputs alone: (slot, tokens of it that are hit)
+    distinct = set()
+    for r in range(w.n_req):
+        hit = int(w.hit_tokens[r])
+        for c in range(-(-hit // w.obj_tokens)):
+            distinct.add((int(w.obj_slot[int(w.obj_start[r]) + c]), min(w.obj_tokens, hit - c * w.obj_tokens)))
+    unique_bytes = sum(2 * v * tb for _, v in distinct)
+    payload = w.total_tokens * 2 * tb
+    assert unique_bytes < payload                               # the batch does share objects
+    assert int(sqes["len"].sum()) == unique_bytes
+    assert len(sgl) == 2 * len(w.block_ids) == int(sqes["sgl_count"].sum())
+    dup = (sgl["id"] & oracle.SGL_DUP) != 0
+    assert int((~dup).sum()) * bb == unique_bytes and int(dup.sum()) * bb == payload - unique_bytes
+    assert np.array_equal(sqes["sgl_first"], np.cumsum(sqes["sgl_count"]) - sqes["sgl_count"])
+    for s_ in sqes:
+        e0, e1 = int(s_["sgl_first"]), int(s_["sgl_first"]) + int(s_["sgl_count"])
+        assert not dup[e0]                                      # a context never opens with a repeat
+        assert int((~dup[e0:e1]).sum()) * bb == int(s_["len"])
+    # contexts in (device, offset) order, a context never starts exactly where its predecessor
+    # ends (they would have merged); contexts overlap only where prefixes of different length of
+    # one object are hit (1-token pages with ragged hits)
+    for a, b in zip(sqes[:-1], sqes[1:]):
+        assert (int(a["dev"]), int(a["src_off"])) <= (int(b["dev"]), int(b["src_off"]))
+        if a["dev"] == b["dev"]:
+            assert int(a["src_off"]) + int(a["len"]) != int(b["src_off"])
+    # every destination block (K and V of every request's table) exactly once
+    want = {base + off + int(b) * stride for off in (k_off, v_off) for b in w.block_ids}
+    got = [int(a) for a in sgl["addr"]]
+    assert len(got) == len(set(got)) and set(got) == want
+    assert np.array_equal(sgl["id"] & 0x7FFFFFFF,
+                          ((sgl["addr"] - np.uint64(base)) % np.uint64(v_off if v_off > stride else stride)
+                           // np.uint64(stride)).astype(np.uint32)) or w.pool_interleaved
+    assert int(num.sum()) == len(sqes) and len(num) == max(1, -(-len(sqes) // capacity))
+    # executing the descriptors reproduces the plain restore, byte for byte
+    store = hc.make_store(w, lo)
+    pool_a = hc.make_pool_layer(w, lo, layer)
+    pool_b = pool_a.copy()
+    assert oracle.restore_layer(g, layer, batch, store, pool_a, k_off, v_off, stride,
+                                w.n_pool_blocks, w.pool_hnd) == 0
+    assert oracle.exec_descriptors(sqes, sgl, store, pool_b, base, w.n_kv_heads, rowb) == 0
+    assert np.array_equal(pool_a, pool_b)
+    assert not np.array_equal(pool_a, hc.make_pool_layer(w, lo, layer))
+
+
 def test_config1_closed_form_counts():
     """Config 1: 16 items, 256 SGL entries; consecutive slots give one 8 MiB context,
     pairwise non-adjacent slots give eight 1 MiB contexts (K and V halves always merge)."""
@@ -391,8 +461,8 @@ def test_config1_closed_form_counts():
 
 def test_partial_last_object_and_duplicates():
     """A prefix that ends inside an object: its K and V halves are not adjacent, so they stay
-    separate contexts.  The same object hit by two requests gives two contexts with the same
-    offset, kept in request order."""
+    separate contexts.  The same object hit by two requests is read once (one source, two
+    destinations per block)."""
     g = oracle.geom(2, 8, 128, 2, 16, 256, 1, oracle.LAYER_MAJOR, 8)
     batch = ([256 + 64], [0, 2], [3, 4], [0, 20], list(range(20)))
     rc, sqes, sgl, num = oracle.build_descriptors(g, 1, 0, batch, 0, 1 << 30, 32768, 2048)
@@ -402,16 +472,32 @@ def test_partial_last_object_and_duplicates():
     assert [(int(s["src_off"]), int(s["len"])) for s in sqes] == [
         (base, lo.obj_bytes + 64 * 2048), (base + lo.obj_bytes + lo.obj_kv_bytes, 64 * 2048)]
     assert list(sqes["sgl_count"]) == [36, 4]
+    # the same object hit by two requests is one source, read once: sorted items K(req 0),
+    # K(req 1), V(req 0), V(req 1) are two groups of two; K and V are byte-adjacent, so one
+    # context names the object's bytes once and lists, block by block, both destinations
     batch = ([256, 256], [0, 1, 2], [5, 5], [0, 16, 32], list(range(32)))
     rc, sqes, sgl, num = oracle.build_descriptors(g, 0, 0, batch, 0, 1 << 30, 32768, 2048)
     assert rc == 0
-    # sorted items: K(req 0), K(req 1), V(req 0), V(req 1).  K(req 1) is followed in bytes by
-    # V(req 0), so those two merge; the byte-adjacency rule knows nothing about requests.
     kvb = int(lo.obj_kv_bytes)
-    assert [(int(s["src_off"]) - 5 * lo.obj_bytes, int(s["len"])) for s in sqes] == [
-        (0, kvb), (0, 2 * kvb), (kvb, kvb)]
-    assert list(sgl["id"][:16]) == list(range(16)) and list(sgl["id"][16:32]) == list(range(16, 32))
-    assert list(sgl["id"][32:48]) == list(range(16)) and np.all(sgl["addr"][32:48] >= 1 << 30)
+    assert [(int(s["src_off"]) - 5 * lo.obj_bytes, int(s["len"]), int(s["sgl_count"]))
+            for s in sqes] == [(0, 2 * kvb, 64)]
+    D = oracle.SGL_DUP
+    want_ids = [x for j in range(16) for x in (j, (16 + j) | D)]
+    assert list(sgl["id"][:32]) == want_ids and list(sgl["id"][32:]) == want_ids
+    assert np.all(sgl["addr"][:32] < 1 << 30) and np.all(sgl["addr"][32:] >= 1 << 30)
+    assert [int(a) for a in sgl["addr"][:4]] == [0, 16 * 32768, 32768, 17 * 32768]
+    # a partial hit of the same object is a different source (other length), read on its own.
+    # Sorted by (offset, length): K of the 64-token hit [0, 128K), K of the full hit [0, 512K),
+    # V of the 64-token hit [512K, 640K), V of the full hit [512K, 1M).  The full K ends where
+    # the short V starts, so those two merge; the full V starts before its predecessor ends.
+    batch = ([256, 64], [0, 1, 2], [5, 5], [0, 16, 20], list(range(20)))
+    rc, sqes, sgl, num = oracle.build_descriptors(g, 0, 0, batch, 0, 1 << 30, 32768, 2048)
+    assert rc == 0
+    p64 = 64 * 2048
+    assert [(int(s["src_off"]) - 5 * lo.obj_bytes, int(s["len"]), int(s["sgl_count"]))
+            for s in sqes] == [(0, p64, 4), (0, kvb + p64, 20), (kvb, kvb, 16)]
+    assert not np.any(sgl["id"] & D)
+    assert list(sgl["id"]) == [16, 17, 18, 19] + list(range(16)) + [16, 17, 18, 19] + list(range(16))
 
 
 def test_empty_and_invalid():

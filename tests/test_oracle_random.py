@@ -22,6 +22,15 @@ def _case(seed):
     n_objs = [-(-h // ot) for h in hits]
     n_slots = max(sum(n_objs) + int(rng.integers(0, 4)), 1)
     slots = rng.permutation(n_slots)[:sum(n_objs)].tolist()
+    # half of the multi-request cases share leading objects with request 0 (a common prefix
+    # stored once): the same slot is then hit by several requests
+    shared = False
+    if n_req > 1 and rng.random() < 0.5:
+        pos = np.concatenate([[0], np.cumsum(n_objs)]).tolist()
+        for r in range(1, n_req):
+            k = int(rng.integers(0, min(n_objs[0], n_objs[r]) + 1))
+            slots[pos[r]:pos[r] + k] = slots[pos[0]:pos[0] + k]
+            shared = shared or k > 0
     n_blks = [h // bt for h in hits]
     n_pool = sum(n_blks) + int(rng.integers(1, 5))
     blocks = rng.permutation(n_pool)[:sum(n_blks)].tolist()
@@ -30,7 +39,7 @@ def _case(seed):
     pad = int(rng.choice([0, 0, 8]))
     return dict(H=H, row=row, bt=bt, ot=ot, L=L, n_dev=n_dev, layout=layout, hits=hits,
                 n_objs=n_objs, n_slots=n_slots, slots=slots, n_blks=n_blks, n_pool=n_pool,
-                blocks=blocks, hnd=hnd, interleaved=interleaved, pad=pad, rng=rng)
+                blocks=blocks, hnd=hnd, interleaved=interleaved, pad=pad, rng=rng, shared=shared)
 
 
 def _store_as_dict(c, store):
@@ -97,6 +106,28 @@ def test_restore_and_save_against_python_loops(seed):
     assert oracle.restore_layer(g, layer, batch, store, got, k_off, v_off, stride, c["n_pool"],
                                 c["hnd"]) == 0
     assert np.array_equal(got, exp)
+    # the block-granular multi-threaded form restores the same bytes
+    for n_thr in (1, 2, 3, 5):
+        got_mt = pool0.copy()
+        assert oracle.move_layer_blocks_mt(g, layer, batch, store, got_mt, k_off, v_off, stride,
+                                           c["n_pool"], True, n_thr, c["hnd"]) == 0
+        assert np.array_equal(got_mt, exp)
+    # descriptors executed = plain restore (shared objects are named once, with repeat entries)
+    flag = oracle.OP_HND if c["hnd"] else 0
+    base = 1 << 32
+    rc, sq, sg, num = oracle.build_descriptors(g, layer, oracle.OP_READ | flag, batch, base + k_off,
+                                               base + v_off, stride, 3)
+    assert rc == 0
+    got2 = pool0.copy()
+    assert oracle.exec_descriptors(sq, sg, store, got2, base, c["H"], c["row"]) == 0
+    assert np.array_equal(got2, exp)
+    n_dup = int(((sg["id"] & oracle.SGL_DUP) != 0).sum())
+    distinct = {(c["slots"][os_[r] + t // c["ot"]], min(c["ot"], hit - (t // c["ot"]) * c["ot"]))
+                for r, hit in enumerate(c["hits"]) for t in range(0, hit, c["ot"])}
+    assert int(sq["len"].sum()) == sum(2 * v * c["H"] * c["row"] for _, v in distinct)
+    assert (n_dup > 0) == (int(sq["len"].sum()) < 2 * sum(c["hits"]) * c["H"] * c["row"])
+    if c["shared"]:
+        return          # saving several requests' blocks into one object is the caller's error
     # expected save from a fresh random pool
     pool1 = rng.integers(0, 256, pool0.nbytes, dtype=np.uint8)
     st_exp = [s.copy() for s in store]
@@ -109,21 +140,8 @@ def test_restore_and_save_against_python_loops(seed):
         assert np.array_equal(a, b)
     # the block-granular, multi-threaded form used as the all-cores baseline: same bytes
     for n_thr in (1, 2, 3, 5):
-        got_mt = pool0.copy()
-        assert oracle.move_layer_blocks_mt(g, layer, batch, store, got_mt, k_off, v_off, stride,
-                                           c["n_pool"], True, n_thr, c["hnd"]) == 0
-        assert np.array_equal(got_mt, exp)
         st_mt = [s.copy() for s in store]
         assert oracle.move_layer_blocks_mt(g, layer, batch, st_mt, pool1, k_off, v_off, stride,
                                            c["n_pool"], False, n_thr, c["hnd"]) == 0
         for a, b in zip(st_mt, st_exp):
             assert np.array_equal(a, b)
-    # descriptors executed = plain restore
-    flag = oracle.OP_HND if c["hnd"] else 0
-    base = 1 << 32
-    rc, sq, sg, num = oracle.build_descriptors(g, layer, oracle.OP_READ | flag, batch, base + k_off,
-                                               base + v_off, stride, 3)
-    assert rc == 0
-    got2 = pool0.copy()
-    assert oracle.exec_descriptors(sq, sg, store, got2, base, c["H"], c["row"]) == 0
-    assert np.array_equal(got2, exp)

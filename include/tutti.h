@@ -156,7 +156,12 @@ typedef struct tutti_sqe {
 } tutti_sqe_t;
 
 /* Scatter-gather entry, 16 bytes (Section 3.1: address 8 B, length 4 B, identifier
- * 4 B).  addr is the pool-side device address, id the pool block id. */
+ * 4 B).  addr is the pool-side device address, id the pool block id.  A stored chunk that
+ * several requests of the batch hit (Section 3.1: a chunk is shared by every request with
+ * that prefix) is named once in its context; the entries of the second and later requests
+ * carry TUTTI_SGL_FLAG_DUP in id: "the object bytes of the entry before this one", so the
+ * walk over the context's byte range does not advance for them. */
+#define TUTTI_SGL_FLAG_DUP 0x80000000u
 typedef struct tutti_sgl {
     uint64_t addr;
     uint32_t len;
@@ -207,10 +212,12 @@ int tutti_obj_layout(const tutti_geom_t *geom, tutti_layout_t *out);
  * Build one layer's I/O contexts on the GPU (Section 3.1 "block lookup and P2P
  * table lookup to generate a batch of lightweight GPU I/O contexts"; Section 3.2
  * step 2, get_iocb).  GPU threads turn (object slot, layer) into (device, offset,
- * length) items, order them by (device, offset), merge exactly byte-adjacent
- * neighbours into one context, emit one 16-byte SGL entry per pool block in
- * object byte order, pack contexts into IOCBs of ioctx_per_iocb entries and
- * publish them in the ring.
+ * length) items, order them by (device, offset, length), treat items that name
+ * exactly the same bytes as one source (read once, TUTTI_SGL_FLAG_DUP), merge
+ * exactly byte-adjacent sources into one context, emit one 16-byte SGL entry per
+ * pool block in object byte order, pack contexts into IOCBs of ioctx_per_iocb
+ * entries and publish them in the ring.  A context's len is the bytes it names in
+ * the store; a completion's bytes are the bytes that landed (entries x length).
  *   batch        host pointer to the struct; its arrays are device pointers.
  *   first_iocb,  host out: indices of the reserved IOCBs, known without waiting
  *   n_iocb       for the GPU: ceil(2*n_obj / ioctx_per_iocb), at least 1.  IOCBs

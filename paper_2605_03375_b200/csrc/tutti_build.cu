@@ -75,8 +75,12 @@ __device__ void bitonic_sort(unsigned long long *key, uint32_t *idx, uint32_t n)
     }
 }
 
-// Sort key of item q = 2 * object + kv: (device << 56) | byte offset at layer 0, or KEY_NONE
-// when the object holds no hit token (or q is padding).  A slot out of range is reported.
+// Sort key of item q = 2 * object + kv, or KEY_NONE when the object holds no hit token (or q
+// is padding).  Items are ordered by (device, offset, length): the key is
+// (device << 56) | (offset at layer 0 in blocks + blocks of the item - 1).  Offsets of items are
+// multiples of an object half (blocks_per_obj blocks) and an item has 1..blocks_per_obj blocks,
+// so the sum orders by offset first, then by length, and equal keys mean exactly the same
+// bytes (a stored chunk hit by several requests).  A slot out of range is reported.
 __device__ unsigned long long item_key(const GeomDev &g, const BatchDev &b, uint32_t q,
                                        int32_t &err) {
     if (q >= 2u * b.n_obj || b.n_req == 0) return KEY_NONE;
@@ -84,7 +88,8 @@ __device__ unsigned long long item_key(const GeomDev &g, const BatchDev &b, uint
     const uint32_t r = find_request(b.obj_start, b.n_req, o);
     if (o < b.obj_start[r] || o >= b.obj_start[r + 1]) return KEY_NONE;
     const uint32_t c = o - b.obj_start[r];
-    if (valid_tokens(b.hit_tokens[r], c, g.obj_tokens) == 0) return KEY_NONE;
+    const uint32_t n_blk = valid_tokens(b.hit_tokens[r], c, g.obj_tokens) / g.block_tokens;
+    if (n_blk == 0) return KEY_NONE;
     const unsigned long long slot = b.obj_slot[o];
     if (slot >= g.n_slots) {
         err = TUTTI_EFAULT;
@@ -93,7 +98,7 @@ __device__ unsigned long long item_key(const GeomDev &g, const BatchDev &b, uint
     const unsigned long long dev = slot % g.n_devices;
     const unsigned long long off = (slot / g.n_devices) * g.stride_slot +
                                    (unsigned long long)kv * g.stride_kv;
-    return (dev << 56) | off;
+    return (dev << 56) | (off / g.block_bytes + (n_blk - 1));
 }
 
 // ---- batches too large for one CTA's shared memory: the same bitonic network, run as a
@@ -162,19 +167,22 @@ bitonic_global_kernel(unsigned long long *key, uint32_t *idx, uint32_t np, uint3
     cmp_exchange(key, idx, i, i | j, (i & k) == 0);
 }
 
-struct ScanPair {
-    uint32_t a, b;
+struct ScanVals {
+    uint32_t a;   // sum: blocks
+    uint32_t b;   // sum of a 0/1 flag: context heads
+    uint32_t m;   // running maximum: index of the latest group start
 };
 
-// Inclusive scan of (a, b) across the CTA for one element per thread, plus carry.  `a`
-// (block counts) goes through shuffles; `b` is a 0/1 flag (run head), so its warp-level
-// prefix is a ballot and a population count.
-__device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &carry) {
+// Inclusive scan of (a, b, m) across the CTA for one element per thread, plus carry.  `a`
+// (block counts) and `m` go through shuffles; `b` is a 0/1 flag (context head), so its
+// warp-level prefix is a ballot and a population count.
+__device__ ScanVals block_scan_incl(ScanVals v, ScanVals *warp_tot, ScanVals &carry) {
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
         uint32_t ua = __shfl_up_sync(0xffffffffu, v.a, d);
-        if (lane >= (uint32_t)d) v.a += ua;
+        uint32_t um = __shfl_up_sync(0xffffffffu, v.m, d);
+        if (lane >= (uint32_t)d) { v.a += ua; v.m = max(v.m, um); }
     }
     const uint32_t heads = __ballot_sync(0xffffffffu, v.b != 0);
     v.b = __popc(heads & (0xffffffffu >> (31 - lane)));
@@ -182,22 +190,27 @@ __device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &ca
     if (lane == 31) warp_tot[warp] = v;
     __syncthreads();
     if (warp == 0) {
-        ScanPair w = lane < n_warps ? warp_tot[lane] : ScanPair{0, 0};
+        ScanVals w = lane < n_warps ? warp_tot[lane] : ScanVals{0, 0, 0};
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             uint32_t ua = __shfl_up_sync(0xffffffffu, w.a, d);
             uint32_t ub = __shfl_up_sync(0xffffffffu, w.b, d);
-            if (lane >= (uint32_t)d) { w.a += ua; w.b += ub; }
+            uint32_t um = __shfl_up_sync(0xffffffffu, w.m, d);
+            if (lane >= (uint32_t)d) { w.a += ua; w.b += ub; w.m = max(w.m, um); }
         }
         if (lane < n_warps) warp_tot[lane] = w;
     }
     __syncthreads();
-    ScanPair off = carry;
-    if (warp > 0) { off.a += warp_tot[warp - 1].a; off.b += warp_tot[warp - 1].b; }
-    v.a += off.a; v.b += off.b;
-    ScanPair tot = warp_tot[n_warps - 1];
+    ScanVals off = carry;
+    if (warp > 0) {
+        off.a += warp_tot[warp - 1].a;
+        off.b += warp_tot[warp - 1].b;
+        off.m = max(off.m, warp_tot[warp - 1].m);
+    }
+    v.a += off.a; v.b += off.b; v.m = max(v.m, off.m);
+    ScanVals tot = warp_tot[n_warps - 1];
     __syncthreads();
-    if (threadIdx.x == 0) { carry.a += tot.a; carry.b += tot.b; }
+    if (threadIdx.x == 0) { carry.a += tot.a; carry.b += tot.b; carry.m = max(carry.m, tot.m); }
     __syncthreads();
     return v;
 }
@@ -205,8 +218,8 @@ __device__ ScanPair block_scan_incl(ScanPair v, ScanPair *warp_tot, ScanPair &ca
 __global__ void __launch_bounds__(PLAN_THREADS, 1)
 plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int presorted) {
     extern __shared__ __align__(16) unsigned char dyn_smem[];
-    __shared__ ScanPair warp_tot[32];
-    __shared__ ScanPair carry;
+    __shared__ ScanVals warp_tot[32];
+    __shared__ ScanVals carry;
     __shared__ int32_t s_status;
     __shared__ uint32_t s_nact;
 
@@ -214,7 +227,7 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
                                        : ring.plan_key;
     uint32_t *idx = use_smem ? reinterpret_cast<uint32_t *>(dyn_smem + (size_t)np * 8)
                              : ring.plan_idx;
-    if (threadIdx.x == 0) { s_status = 0; s_nact = 0; carry.a = 0; carry.b = 0; }
+    if (threadIdx.x == 0) { s_status = 0; s_nact = 0; carry.a = 0; carry.b = 0; carry.m = 0; }
     __syncthreads();
 
     // per-request preconditions
@@ -253,55 +266,66 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
     __syncthreads();
     const uint32_t n_act = s_status ? 0 : s_nact;
 
-    // blocks per item (kept in plan_sqe_of until the scans have run)
+    const unsigned long long OFF_MASK = (1ull << 56) - 1;
+    // blocks per item (kept in plan_sqe_of until the scans have run), byte offset, item id
     for (uint32_t i = threadIdx.x; i < n_act; i += blockDim.x) {
         uint32_t q = idx[i], o = q >> 1;
         uint32_t r = find_request(b.obj_start, b.n_req, o);
         uint32_t valid = valid_tokens(b.hit_tokens[r], o - b.obj_start[r], g.obj_tokens);
-        ring.plan_sqe_of[i] = valid / g.block_tokens;
+        const uint32_t n_blk = valid / g.block_tokens;
+        const unsigned long long k = key[i];
+        ring.plan_sqe_of[i] = n_blk;
         ring.plan_item[i] = q;
+        ring.plan_off[i] = (k & ~OFF_MASK) | (((k & OFF_MASK) - (n_blk - 1)) * g.block_bytes);
     }
     __syncthreads();
 
-    // steps 3-4: adjacency flags (an item starts a new context unless it begins exactly
-    // where its predecessor on the same device ends); packed with the block count
+    // steps 3-4: flags.  An item repeats its predecessor when the keys are equal (the same
+    // bytes, hit by another request): such a group is one source.  A group starts a new
+    // context unless it begins exactly where the previous group's bytes end on the same
+    // device.  Packed with the block count: bit 31 context head, bit 30 repeat.
     for (uint32_t i = threadIdx.x; i < n_act; i += blockDim.x) {
-        uint32_t head = 1;
+        uint32_t head = 1, rep = 0;
         if (i > 0) {
-            unsigned long long k = key[i], kp = key[i - 1];
-            unsigned long long end_prev = (kp & ((1ull << 56) - 1)) +
-                                          (unsigned long long)ring.plan_sqe_of[i - 1] * g.block_bytes;
-            head = ((kp >> 56) != (k >> 56)) || (end_prev != (k & ((1ull << 56) - 1)));
+            const unsigned long long k = key[i], kp = key[i - 1];
+            rep = (k == kp);
+            // end of the previous item = end of its group (all members name the same bytes)
+            const unsigned long long end_prev = (kp & OFF_MASK) + 1;          // in blocks
+            const unsigned long long start = (k & OFF_MASK) - (ring.plan_sqe_of[i] - 1);
+            head = !rep && (((kp >> 56) != (k >> 56)) || (end_prev != start));
         }
-        ring.plan_cumblk[i] = (head << 31) | ring.plan_sqe_of[i];
+        ring.plan_cumblk[i] = (head << 31) | (rep << 30) | ring.plan_sqe_of[i];
     }
     __syncthreads();
 
-    // step 5: prefix sums of (blocks, run heads); every thread touches only its own item
+    // step 5: prefix sums of (blocks, context heads) and the running group start; every
+    // thread touches only its own item
     for (uint32_t base = 0; base < n_act; base += blockDim.x) {
         uint32_t i = base + threadIdx.x;
-        ScanPair v{0, 0};
-        uint32_t nblk = 0, head = 0;
+        ScanVals v{0, 0, 0};
+        uint32_t nblk = 0, head = 0, rep = 0;
         if (i < n_act) {
             uint32_t packed = ring.plan_cumblk[i];
-            nblk = packed & 0x7fffffffu;
+            nblk = packed & 0x3fffffffu;
             head = packed >> 31;
-            v.a = nblk; v.b = head;
+            rep = (packed >> 30) & 1u;
+            v.a = nblk; v.b = head; v.m = rep ? 0u : i;
         }
-        ScanPair s = block_scan_incl(v, warp_tot, carry);
+        ScanVals s = block_scan_incl(v, warp_tot, carry);
         if (i < n_act) {
             uint32_t excl = s.a - nblk;
             uint32_t sq = s.b - 1;
             ring.plan_cumblk[i] = excl;
             ring.plan_sqe_of[i] = sq;
+            ring.plan_grp[i] = s.m;                  // index of the first item of this group
             if (head) {
-                unsigned long long k = key[i];
+                const unsigned long long po = ring.plan_off[i];
                 tutti_sqe_t e;
-                e.src_off = k & ((1ull << 56) - 1);
+                e.src_off = po & OFF_MASK;
                 e.len = 0;
                 e.sgl_first = excl;
                 e.sgl_count = 0;
-                e.dev = (uint32_t)(k >> 56);
+                e.dev = (uint32_t)(po >> 56);
                 e.opcode = 0;
                 e.layer = 0;
                 ring.plan_sqe[sq] = e;
@@ -313,14 +337,19 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
     if (threadIdx.x == 0) ring.plan_cumblk[n_act] = n_entries;
     __syncthreads();
 
-    // close every run: length and entry count
+    // group sizes (written at every group's first item) and the end of every context: its
+    // entries cover all members of its groups, its length names the bytes once
     for (uint32_t i = threadIdx.x; i < n_act; i += blockDim.x) {
+        const bool group_ends = (i + 1 == n_act) || (ring.plan_grp[i + 1] == i + 1);
+        if (group_ends) ring.plan_k[ring.plan_grp[i]] = i + 1 - ring.plan_grp[i];
         uint32_t sq = ring.plan_sqe_of[i];
         bool last = (i + 1 == n_act) || (ring.plan_sqe_of[i + 1] != sq);
         if (last) {
-            uint32_t cnt = ring.plan_cumblk[i + 1] - ring.plan_sqe[sq].sgl_first;
-            ring.plan_sqe[sq].sgl_count = cnt;
-            ring.plan_sqe[sq].len = (unsigned long long)cnt * g.block_bytes;
+            const uint32_t n_blk = ring.plan_cumblk[i + 1] - ring.plan_cumblk[i];
+            const unsigned long long end = (ring.plan_off[i] & OFF_MASK) +
+                                           (unsigned long long)n_blk * g.block_bytes;
+            ring.plan_sqe[sq].sgl_count = ring.plan_cumblk[i + 1] - ring.plan_sqe[sq].sgl_first;
+            ring.plan_sqe[sq].len = end - ring.plan_sqe[sq].src_off;
         }
     }
     if (threadIdx.x == 0) {
@@ -414,40 +443,43 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
     for (uint32_t i0 = gwarp * per_warp; i0 < n_items; i0 += nwarps * per_warp) {
         const uint32_t i = i0 + sub;
         const bool live = i < n_items;
-        uint32_t q = 0, e_first = 0, e_next = 0;
-        unsigned long long meta0 = 0, meta1 = 0;   // (row start in block table, object-side address)
+        // leader: the item, its place in its group (copy c of k), the group's first entry,
+        // its row in the block table and the object-side address of its first byte
+        uint32_t q = 0, n_blk = 0, g_first = 0, k_copies = 1, c_copy = 0;
+        unsigned long long meta0 = 0, meta1 = 0;
         if (live && sl == 0) {
             q = ring.plan_item[i];
-            e_first = ring.plan_cumblk[i];
-            e_next = ring.plan_cumblk[i + 1];
-            const uint32_t sq = ring.plan_sqe_of[i];
+            n_blk = ring.plan_cumblk[i + 1] - ring.plan_cumblk[i];
+            const uint32_t gs = ring.plan_grp[i];
+            g_first = ring.plan_cumblk[gs];
+            k_copies = ring.plan_k[gs];
+            c_copy = i - gs;
             const uint32_t o = q >> 1;
             uint32_t r = find_request(b.obj_start, b.n_req, o);
             uint32_t c = o - b.obj_start[r];
             meta0 = (unsigned long long)b.blk_start[r] + (unsigned long long)c * g.blocks_per_obj;
-            // object-side address of the item's first byte: context start + bytes of the
-            // items that precede it in the same run
-            tutti_sqe_t run = ring.plan_sqe[sq];
-            unsigned long long off = run.src_off + layer_off +
-                                     (unsigned long long)(e_first - run.sgl_first) * g.block_bytes;
-            unsigned long long end = off + (unsigned long long)(e_next - e_first) * g.block_bytes;
-            if (end > p.store_bytes[run.dev]) {
+            const unsigned long long po = ring.plan_off[i];
+            const uint32_t dev = (uint32_t)(po >> 56);
+            const unsigned long long off = (po & ((1ull << 56) - 1)) + layer_off;
+            const unsigned long long end = off + (unsigned long long)n_blk * g.block_bytes;
+            if (end > p.store_bytes[dev]) {
                 note_error(&hdr0->emit_status, TUTTI_EFAULT);
                 meta1 = 0;
-                e_next = e_first;                      // nothing is emitted for this item
+                n_blk = 0;                             // nothing is emitted for this item
             } else {
-                meta1 = p.store_base[run.dev] + off;
+                meta1 = p.store_base[dev] + off;
             }
         }
         // the group leader read the item; its lanes get it by shuffle
         q = __shfl_sync(0xffffffffu, q, leader);
-        e_first = __shfl_sync(0xffffffffu, e_first, leader);
-        e_next = __shfl_sync(0xffffffffu, e_next, leader);
+        n_blk = __shfl_sync(0xffffffffu, n_blk, leader);
+        g_first = __shfl_sync(0xffffffffu, g_first, leader);
+        k_copies = __shfl_sync(0xffffffffu, k_copies, leader);
+        c_copy = __shfl_sync(0xffffffffu, c_copy, leader);
         const unsigned long long row0 = __shfl_sync(0xffffffffu, meta0, leader);
         const unsigned long long obj0 = __shfl_sync(0xffffffffu, meta1, leader);
         if (!live) continue;
         const unsigned long long pool_base = (q & 1) ? p.v_base : p.k_base;
-        const uint32_t n_blk = e_next - e_first;
         for (uint32_t j = sl; j < n_blk; j += G) {
             unsigned long long bi = row0 + j;
             tutti_sgl_t ent;
@@ -461,9 +493,11 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
                 note_error(&hdr0->emit_status, TUTTI_EFAULT);
                 continue;
             }
+            // block j of the source: one entry per member of the group, side by side; all
+            // but the first are flagged as taking the bytes of the entry before them
             ent.addr = pool_base + (unsigned long long)id * p.block_stride;
-            ent.id = (uint32_t)id;
-            size_t at = (size_t)p.sgl_base + e_first + j;
+            ent.id = (uint32_t)id | (c_copy ? TUTTI_SGL_FLAG_DUP : 0u);
+            size_t at = (size_t)p.sgl_base + g_first + (size_t)j * k_copies + c_copy;
             ring.sgl[at] = ent;
             ring.obj_ptr[at] = obj0 + (unsigned long long)j * g.block_bytes;
         }

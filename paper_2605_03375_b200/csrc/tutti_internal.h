@@ -84,6 +84,10 @@ struct RingDev {
     uint32_t *plan_item;      // [max_items]  item id (2*object + kv) in sorted order
     uint32_t *plan_cumblk;    // [max_items+1] exclusive prefix of blocks per item
     uint32_t *plan_sqe_of;    // [max_items]  context index of each item
+    uint64_t *plan_off;       // [max_items]  (device << 56) | byte offset of the item at layer 0
+    uint32_t *plan_grp;       // [max_items]  index of the first item of the item's group (items
+                              //              that name exactly the same bytes form a group)
+    uint32_t *plan_k;         // [max_items]  at a group's first item: members of the group
     tutti_sqe_t *plan_sqe;    // [max_items]  contexts for layer 0, opcode unset
     unsigned long long *plan_key;  // [pow2(max_items)] sort keys when they do not fit in shared memory
     uint32_t *plan_idx;       // [pow2(max_items)] sort payload, same

@@ -369,6 +369,9 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
     A((void **)&d.plan_item, sizeof(uint32_t) * (size_t)max_items, false);
     A((void **)&d.plan_cumblk, sizeof(uint32_t) * ((size_t)max_items + 1), false);
     A((void **)&d.plan_sqe_of, sizeof(uint32_t) * (size_t)max_items, false);
+    A((void **)&d.plan_off, sizeof(uint64_t) * (size_t)max_items, false);
+    A((void **)&d.plan_grp, sizeof(uint32_t) * (size_t)max_items, false);
+    A((void **)&d.plan_k, sizeof(uint32_t) * (size_t)max_items, false);
     A((void **)&d.plan_sqe, sizeof(tutti_sqe_t) * (size_t)max_items, false);
     A((void **)&d.plan_key, sizeof(unsigned long long) * (size_t)np, false);
     A((void **)&d.plan_idx, sizeof(uint32_t) * (size_t)np, false);
@@ -694,14 +697,20 @@ int tutti_ring_fill_host(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t iocb_idx,
         for (uint32_t e = s.sgl_first; e < s.sgl_first + s.sgl_count; ++e) {
             if (seen[e] || (sgl[e].len & 15) || (sgl[e].addr & 15) || sgl[e].len == 0) return TUTTI_EINVAL;
             seen[e] = 1;
-            if (cursor + sgl[e].len > ctx->store[s.dev].bytes) return TUTTI_EFAULT;
-            optr[e] = ctx->store[s.dev].base + cursor;
-            if (optr[e] & 15) return TUTTI_EINVAL;
-            cursor += sgl[e].len;
+            if (sgl[e].id & TUTTI_SGL_FLAG_DUP) {
+                // the object bytes of the entry before: same address, the walk stays put
+                if (e == s.sgl_first || sgl[e].len != sgl[e - 1].len) return TUTTI_EINVAL;
+                optr[e] = optr[e - 1];
+            } else {
+                if (cursor + sgl[e].len > ctx->store[s.dev].bytes) return TUTTI_EFAULT;
+                optr[e] = ctx->store[s.dev].base + cursor;
+                if (optr[e] & 15) return TUTTI_EINVAL;
+                cursor += sgl[e].len;
+            }
+            total += sgl[e].len;
             if (sgl[e].len != common) common = 0;
         }
         if (cursor - s.src_off != s.len) return TUTTI_EINVAL;
-        total += s.len;
     }
     for (uint32_t e = 0; e < n_sgl; ++e)
         if (!seen[e]) return TUTTI_EINVAL;

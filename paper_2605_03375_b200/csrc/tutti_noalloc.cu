@@ -32,7 +32,10 @@ constexpr size_t OFF_PLAN_SQE = OFF_SQES + sizeof(tutti_sqe_t) * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_ITEM = OFF_PLAN_SQE + sizeof(tutti_sqe_t) * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_CUM = OFF_PLAN_ITEM + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_SQE_OF = OFF_PLAN_CUM + 4 * (NA_MAX_ITEMS + 64);
-constexpr size_t OFF_PLAN_KEY = OFF_PLAN_SQE_OF + 4 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_OFF = OFF_PLAN_SQE_OF + 4 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_GRP = OFF_PLAN_OFF + 8 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_K = OFF_PLAN_GRP + 4 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_KEY = OFF_PLAN_K + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_IDX = OFF_PLAN_KEY + 8 * NA_POW2_ITEMS;
 constexpr size_t OFF_SGL = OFF_PLAN_IDX + 4 * NA_POW2_ITEMS;
 constexpr size_t OFF_OBJ = OFF_SGL + sizeof(tutti_sgl_t) * NA_MAX_ENTRIES;
@@ -135,6 +138,9 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         r.plan_cumblk = reinterpret_cast<uint32_t *>(base + OFF_PLAN_CUM);
         r.plan_sqe_of = reinterpret_cast<uint32_t *>(base + OFF_PLAN_SQE_OF);
         r.plan_sqe = reinterpret_cast<tutti_sqe_t *>(base + OFF_PLAN_SQE);
+        r.plan_off = reinterpret_cast<uint64_t *>(base + OFF_PLAN_OFF);
+        r.plan_grp = reinterpret_cast<uint32_t *>(base + OFF_PLAN_GRP);
+        r.plan_k = reinterpret_cast<uint32_t *>(base + OFF_PLAN_K);
         r.plan_key = reinterpret_cast<unsigned long long *>(base + OFF_PLAN_KEY);
         r.plan_idx = reinterpret_cast<uint32_t *>(base + OFF_PLAN_IDX);
         r.plan_counts = reinterpret_cast<PlanCounts *>(base + OFF_COUNTS);

@@ -34,7 +34,9 @@ def random_workload(seed):
         layout=int(rng.choice([wl.LAYOUT_FILE_MAJOR, wl.LAYOUT_LAYER_MAJOR])),
         slot_mean_run=float(rng.choice([1.0, 2.0, 6.0])), slot_space_factor=float(rng.choice([1.1, 2.0])),
         pool_round=64, pool_interleaved=bool(rng.random() < 0.4), pool_hnd=hnd,
-        pool_pad_bytes=int(rng.choice([0, 0, 16, 256]))), rng
+        pool_pad_bytes=int(rng.choice([0, 0, 16, 256])),
+        # a third of the cases: requests share leading objects (read once, repeat entries)
+        shared_prefix_frac=float(np.random.default_rng(9000 + seed).choice([0.0, 0.0, 0.5, 1.0]))), rng
 
 
 @pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("TUTTI_FUZZ_CASES", "40"))))
@@ -61,7 +63,7 @@ def test_random_case(seed):
         dc.ring.tutti_kv_restore_layer(first, n, sm_count)
         cqes = dc.poll_all(first, n)
         assert all(c[1] == 0 for c in cqes)
-        assert sum(c[2] for c in cqes) == int(osq["len"].sum())
+        assert sum(c[2] for c in cqes) == int(osg["len"].astype(np.uint64).sum())
         want = dc.oracle_restore(layer)
         assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
         for t in dc.store_dev:
@@ -222,7 +224,7 @@ def test_random_host_prepared_descriptors(seed):
         sm = int(rng.choice([0, 5]))
         (dc.ring.tutti_kv_restore_layer if op == T.OP_READ else dc.ring.tutti_kv_save_layer)(first, 1, sm)
         (idx, status, nbytes), = dc.poll_all(first, 1)
-        assert status == 0 and nbytes == int(osq["len"].sum())
+        assert status == 0 and nbytes == int(osg["len"].astype(np.uint64).sum())
         if op == T.OP_READ:
             assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
         else:

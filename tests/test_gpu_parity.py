@@ -36,6 +36,14 @@ CASES = {
                                   head_dim=64, block_tokens=2, obj_tokens=32),
     "hnd-pool-interleaved-2dev": dict(index=2, scale=0.04, n_layers=2, pool_hnd=True, n_devices=2,
                                       pool_interleaved=True, layout=wl.LAYOUT_FILE_MAJOR),
+    # requests with a common prefix: the shared objects are read once (repeat entries)
+    "shared-prefix-8-requests": dict(index=2, scale=0.25, n_layers=2, hit_tokens=[2048] * 8,
+                                     shared_prefix_frac=0.75),
+    "shared-prefix-1-token-pages": dict(index=4, scale=0.05, n_layers=2, shared_prefix_frac=1.0),
+    "shared-prefix-hnd-2dev": dict(index=2, scale=0.05, n_layers=2, hit_tokens=[1024] * 3,
+                                   shared_prefix_frac=0.5, pool_hnd=True, n_devices=2),
+    "shared-prefix-one-block-objects": dict(index=2, scale=0.02, n_layers=2, obj_tokens=16,
+                                            hit_tokens=[512, 512, 256], shared_prefix_frac=1.0),
 }
 
 
@@ -69,7 +77,7 @@ def test_restore_and_save_match_oracle(name, engine):
             cqes = dc.poll_all(first, n)
             assert sorted(c[0] for c in cqes) == list(range(first, first + n))
             assert all(c[1] == 0 for c in cqes)
-            assert sum(c[2] for c in cqes) == int(osq["len"].sum())
+            assert sum(c[2] for c in cqes) == int(osg["len"].astype(np.uint64).sum())
             got = dc.pool_dev[layer].cpu().numpy()
             want = dc.oracle_restore(layer)
             assert np.array_equal(got, want)
@@ -116,7 +124,7 @@ def test_small_iocbs_ring_wrap_and_capped_mode(engine, sm_count):
             dc.ring.tutti_kv_restore_layer(first, n, sm_count)
             cqes = dc.poll_all(first, n)
             assert sorted(c[0] for c in cqes) == list(range(first, first + n))
-            assert sum(c[2] for c in cqes) == int(osq["len"].sum())
+            assert sum(c[2] for c in cqes) == int(osg["len"].astype(np.uint64).sum())
             assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
             seen.append(first)
         assert seen[-1] >= 64          # the index counter ran past the ring depth
@@ -156,7 +164,7 @@ def test_host_prepared_descriptors():
         dc.ring.tutti_ring_fill_host(first, sq2, sg2)
         dc.ring.tutti_kv_restore_layer(first, 1)
         (idx, status, nbytes), = dc.poll_all(first, 1)
-        assert status == 0 and nbytes == int(osq["len"].sum())
+        assert status == 0 and nbytes == int(osg["len"].astype(np.uint64).sum())
         assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
     finally:
         dc.close()

@@ -25,10 +25,11 @@ def _case(seed):
     # half of the multi-request cases share leading objects with request 0 (a common prefix
     # stored once): the same slot is then hit by several requests
     shared = False
-    if n_req > 1 and rng.random() < 0.5:
+    if n_req > 1 and rng.random() < 0.7:
         pos = np.concatenate([[0], np.cumsum(n_objs)]).tolist()
         for r in range(1, n_req):
-            k = int(rng.integers(0, min(n_objs[0], n_objs[r]) + 1))
+            m = min(n_objs[0], n_objs[r])
+            k = int(rng.integers(min(1, m), m + 1))
             slots[pos[r]:pos[r] + k] = slots[pos[0]:pos[0] + k]
             shared = shared or k > 0
     n_blks = [h // bt for h in hits]

@@ -164,7 +164,7 @@ class Replica:
     """Config-2-shaped workload resident on one GPU, registered with the library."""
 
     def __init__(self, args, device_index: int, host_store: bool = False, n_layers=None,
-                 hit_tokens=None, ring_depth=None):
+                 hit_tokens=None, ring_depth=None, shared_prefix_frac=0.0):
         import torch
         from paper_2605_03375_b200 import tutti as T
         from paper_2605_03375_b200 import workload as wl
@@ -183,6 +183,8 @@ class Replica:
             over["n_layers"] = n_layers
         if hit_tokens is not None:
             over["hit_tokens"] = hit_tokens
+        if shared_prefix_frac:
+            over["shared_prefix_frac"] = shared_prefix_frac
         self.w = w = wl.config(args.config, args.scale, **over)
         self.geom = T.geom_of(w)
         self.ctx = T.Context(self.geom, device_index)
@@ -624,6 +626,7 @@ def run_ours(args):
                 "cfg3": run_leg(leg_config3, args, local_rank),
                 "cfg4": run_leg(leg_config4, args, local_rank),
                 "cfg5": run_leg(leg_config5, args, local_rank),
+                "shared_prefix": run_leg(leg_shared_prefix, args, local_rank),
             }
         if not args.no_sched:
             out["sched"] = {"hbm": run_leg(leg_sched_demo, args, local_rank, False),
@@ -691,6 +694,56 @@ def leg_config1(args, local_rank):
                    "16 MiB of traffic stays in L2, so no HBM fraction is quoted")
     out["spot_check"] = bool(rep.spot_check(64))
     rep.close()
+    return out
+
+
+def leg_shared_prefix(args, local_rank):
+    """Requests of one batch with a common prefix (Section 3.1: a stored chunk is shared by every
+    request with that prefix): the config-2 batch with the first 75 % of every request's objects
+    being the same stored objects.  The descriptors name each shared object once; the copy
+    kernels load it once per stage and store it to every request's blocks.  Restore only (a
+    save of several requests into one object is the caller's race)."""
+    import torch
+    from paper_2605_03375_b200 import tutti as T
+    peak, _ = measured_peak()
+    out = {"batch": "config-2 shape, 8 requests x 32768 tokens, first 75 % of the objects shared"}
+    for store, host, layers in (("hbm", False, 8), ("pinned_host", True, 4)):
+        res = {}
+        for frac in (0.75, 0.0):
+            a2 = argparse.Namespace(**vars(args))
+            a2.config, a2.scale, a2.set, a2.layers = 2, 1.0, None, 0
+            a2.ioctx_per_iocb = 2048
+            a2.layers_per_launch = 0
+            a2.resident_layers = layers
+            rep = Replica(a2, local_rank, host_store=host, n_layers=layers, shared_prefix_frac=frac)
+            if host:
+                rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, T.ENGINE_BULK)
+            sm = 16 if host else 0
+            ms = timed_passes(rep, (T.OP_READ,), 2 if host else 4, sm_count=sm)
+            gbs = rep.payload_per_layer / (ms * 1e-3) / 1e9
+            key = "shared" if frac else "private"
+            res[key] = {"landed_gbs": round(gbs, 1), "ms_per_layer": round(ms, 4)}
+            if frac:
+                # bytes the descriptors name in the store, from the library's own contexts
+                rep.epoch += 1
+                rep.batch.plan_epoch = rep.epoch
+                rc, first, n = rep.ring.tutti_build_sqes(rep.batch, 0, T.OP_READ, stream=rep.stream)
+                named = 0
+                for i in range(first, first + n):
+                    info, sq = rep.ring.tutti_ring_read_iocb(i)
+                    named += int(sq["len"].sum())
+                rep.ring.tutti_kv_restore_layer(first, n, 0, stream=rep.stream)
+                rep.poll_list([(first, n)])
+                res["store_bytes_named_per_landed_byte"] = round(named / rep.payload_per_layer, 4)
+                res["spot_check"] = bool(rep.spot_check(64))
+            rep.close()
+            del rep
+            torch.cuda.empty_cache()
+        res["speedup_from_sharing"] = round(res["shared"]["landed_gbs"] / res["private"]["landed_gbs"], 3)
+        if not host:
+            res["shared"]["pool_write_hbm_frac"] = round(res["shared"]["landed_gbs"] / peak, 4)
+        res["sm_count"] = 16 if host else 0
+        out[store] = res
     return out
 
 
@@ -1293,13 +1346,16 @@ def main():
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the config 1/3/4/5 legs of the default line")
     ap.add_argument("--no-sched", action="store_true", help="skip the scheduler legs")
+    ap.add_argument("--shared-prefix", action="store_true",
+                    help="run the shared-prefix leg on its own")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-only", action="store_true", help="run the end-to-end leg on its own")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    elif args.sched_demo or args.sweep_length or args.e2e_only or args.config != 2:
+    elif (args.sched_demo or args.sweep_length or args.e2e_only or args.shared_prefix or
+          args.config != 2):
         # a single leg on its own (one GPU)
         rank, local_rank, world = init_dist("nccl")
         if args.sweep_length:
@@ -1310,7 +1366,7 @@ def main():
             if rank == 0:
                 print(json.dumps(res), flush=True)
             return
-        leg = (leg_sched_demo if args.sched_demo else
+        leg = (leg_sched_demo if args.sched_demo else leg_shared_prefix if args.shared_prefix else
                {1: leg_config1, 3: leg_config3, 4: leg_config4, 5: leg_config5}[args.config])
         extra = (args.sched_host,) if args.sched_demo else ()
         res = run_leg(leg, args, local_rank, *extra)

@@ -333,6 +333,26 @@ copy_ldst_kernel(CopyParams p) {
                             for (int k = 0; k < 8; ++k) v[k] = ld_stream(src + k * 512);
 #pragma unroll
                             for (int k = 0; k < 8; ++k) st_stream(dst + k * 512, v[k]);
+                            // restore of an object shared by several requests: the following
+                            // entries of this claim that repeat these bytes (one entry per
+                            // tile, so every warp of the group sees the same flags) are stored
+                            // from the registers just loaded, and their tiles are skipped
+                            while (TO_POOL && elen == CHUNK_BYTES && t + 1 < t1) {
+                                unsigned long long a_next = 0;
+                                uint32_t id_next = 0;
+                                if (lane == 0) {
+                                    const tutti_sgl_t ent = sgl[t + 1];
+                                    a_next = ent.addr;
+                                    id_next = ent.id;
+                                }
+                                id_next = __shfl_sync(0xffffffffu, id_next, 0);
+                                if (!(id_next & TUTTI_SGL_FLAG_DUP)) break;
+                                a_next = __shfl_sync(0xffffffffu, a_next, 0);
+                                char *dst2 = reinterpret_cast<char *>(a_next) + o_obj;
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) st_stream(dst2 + k * 512, v[k]);
+                                ++t;
+                            }
                         } else {
                             // head-major pool block: every 16-byte vector keeps its place in the
                             // object and goes to the transposed row of the block
@@ -712,48 +732,126 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
         n_bi = f_cur_bi;
         n_hnd = f_hnd;
         ld_bytes = 0; st_bytes = 0; st_off = 0; ld_addr = 0; st_addr = 0;
-        if (f_hnd) {
-            // one block: every lane needs both addresses (the rows are spread over the lanes)
+        if (cg.per_chunk == 1) {
+            // one entry per stage (a whole block; also every head-major block).  On a restore
+            // the entries right after it that repeat its bytes (the same stored chunk going to
+            // other requests' blocks) share the stage: one load, one store per destination.
+            const uint32_t n_in = min(32u, cur_end - c);         // entries of this claim from c on
             unsigned long long a_obj = 0, a_pool = 0;
-            if (lane == 0) { a_obj = obj[c]; a_pool = sgl[c].addr; }
+            uint32_t id_flags = 0;
+            if (lane < n_in) {
+                const tutti_sgl_t ent = sgl[c + lane];
+                a_pool = ent.addr;
+                id_flags = ent.id;
+            }
+            if (lane == 0) a_obj = obj[c];
             a_obj = __shfl_sync(0xffffffffu, a_obj, 0);
-            a_pool = __shfl_sync(0xffffffffu, a_pool, 0);
-            // object side as (device, token row) for the tensor map
-            uint32_t dv = 0;
-            for (uint32_t d = 1; d < tm.n_devices; ++d)
-                if (a_obj >= tm.base[d] && a_obj < tm.base[d] + tm.bytes[d]) dv = d;
-            const unsigned long long rowi = (a_obj - tm.base[dv]) / p.perm.token_bytes;
-            const unsigned long long packed = (rowi << 8) | dv;
-            ld_addr = TO_POOL ? packed : a_pool;
-            st_addr = TO_POOL ? a_pool : packed;
-            ld_bytes = st_bytes = (lane == 0) ? cg.elen : 0;
+            const bool rep = TO_POOL && lane > 0 && lane < n_in && (id_flags & TUTTI_SGL_FLAG_DUP);
+            const uint32_t reps = __ballot_sync(0xffffffffu, rep) | 1u;
+            const uint32_t m = (reps == 0xffffffffu) ? 32u : (uint32_t)(__ffs(~reps) - 1);
+            cur += m - 1;                                         // the repeats are consumed too
+            if (f_hnd) {
+                // object side as (device, token row) for the tensor map; the rows are spread
+                // over the lanes, so every lane carries the packed source
+                uint32_t dv = 0;
+                for (uint32_t d = 1; d < tm.n_devices; ++d)
+                    if (a_obj >= tm.base[d] && a_obj < tm.base[d] + tm.bytes[d]) dv = d;
+                const unsigned long long rowi = (a_obj - tm.base[dv]) / p.perm.token_bytes;
+                const unsigned long long packed = (rowi << 8) | dv;
+                const unsigned long long pool0 = __shfl_sync(0xffffffffu, a_pool, 0);
+                if (TO_POOL) {
+                    ld_addr = packed;
+                    ld_bytes = (lane == 0) ? cg.elen : 0;
+                    st_addr = a_pool;
+                    st_bytes = (lane < m) ? cg.elen : 0;
+                } else {
+                    ld_addr = pool0;
+                    ld_bytes = (lane == 0) ? cg.elen : 0;
+                    st_addr = packed;
+                    st_bytes = (lane == 0) ? cg.elen : 0;
+                }
+            } else if (TO_POOL) {
+                ld_addr = a_obj;
+                ld_bytes = (lane == 0) ? cg.elen : 0;
+                st_addr = a_pool;
+                st_bytes = (lane < m) ? cg.elen : 0;
+            } else {
+                ld_addr = a_pool;
+                ld_bytes = (lane == 0) ? cg.elen : 0;
+                st_addr = a_obj;
+                st_bytes = (lane == 0) ? cg.elen : 0;
+            }
         } else if (cg.per_chunk) {
             const uint32_t e0 = c * cg.per_chunk;
             const uint32_t n_e = min(cg.per_chunk, cg.total - e0);
             unsigned long long a_obj = 0, a_pool = 0;
-            if (lane < n_e) { a_obj = obj[e0 + lane]; a_pool = sgl[e0 + lane].addr; }
+            uint32_t id_flags = 0;
+            if (lane < n_e) {
+                const tutti_sgl_t ent = sgl[e0 + lane];
+                a_obj = obj[e0 + lane];
+                a_pool = ent.addr;
+                id_flags = ent.id;
+            }
+            // restore: an entry that repeats the bytes of the entry before it brings nothing
+            // into the stage and is stored from its predecessor's place (the first entry of a
+            // chunk always loads: its predecessor sits in another chunk)
+            const bool rep = TO_POOL && lane > 0 && lane < n_e && (id_flags & TUTTI_SGL_FLAG_DUP);
+            const uint32_t live = (n_e >= 32u) ? 0xffffffffu : ((1u << n_e) - 1u);
+            const uint32_t uniq = live & ~__ballot_sync(0xffffffffu, rep);
+            const uint32_t upto = 0xffffffffu >> (31 - lane);     // lanes 0..lane
+            const uint32_t slot = (lane < n_e) ? (uint32_t)__popc(uniq & upto) - 1u : 0u;
             // the object side is contiguous in runs: one bulk copy per run
             unsigned long long prev = __shfl_up_sync(0xffffffffu, a_obj, 1);
-            bool is_head = lane < n_e && (lane == 0 || a_obj != prev + cg.elen);
+            bool is_head = ((uniq >> lane) & 1u) && (lane == 0 || a_obj != prev + cg.elen);
             uint32_t heads = __ballot_sync(0xffffffffu, is_head);
             uint32_t run_bytes = 0;
             if (is_head) {
                 uint32_t above = lane < 31 ? heads >> (lane + 1) : 0u;
                 uint32_t next = above ? lane + __ffs(above) : n_e;
-                run_bytes = (next - lane) * cg.elen;
+                const uint32_t below_next = (next >= 32u) ? 0xffffffffu : ((1u << next) - 1u);
+                run_bytes = (uint32_t)__popc(uniq & below_next & ~(upto >> 1)) * cg.elen;
             }
             const uint32_t one = lane < n_e ? cg.elen : 0;
-            st_off = lane * cg.elen;
+            st_off = slot * cg.elen;
             if (TO_POOL) { ld_addr = a_obj; ld_bytes = run_bytes; st_addr = a_pool; st_bytes = one; }
             else         { ld_addr = a_pool; ld_bytes = one; st_addr = a_obj; st_bytes = run_bytes; }
         } else {
-            const uint32_t e = c / cg.pieces, piece = c % cg.pieces;
+            // entries longer than a stage are moved in pieces.  Chunks are numbered piece-major
+            // inside blocks of 32 entries (piece 0 of entries 0..31, then piece 1 of them, ...),
+            // so that consecutive chunks are the same piece of consecutive entries: on a
+            // restore, entries that repeat their predecessor's bytes share the stage here too.
+            // (A save has no repeats to fold and keeps entry-major order, which writes the
+            // object side sequentially.)
+            const uint32_t PB = TO_POOL ? 32u : 1u;               // entries per block
+            const uint32_t span = PB * cg.pieces;
+            const uint32_t blk = c / span, rem = c - blk * span;
+            const uint32_t e_base = blk * PB;
+            const uint32_t n_b = min(PB, cg.total - e_base);      // entries of this block
+            const uint32_t piece = rem / n_b, ei = rem - piece * n_b;
+            const uint32_t e = e_base + ei;
             const uint32_t off = piece * CB;
             const uint32_t bytes = min(CB, cg.elen - off);
-            if (lane == 0) {
-                unsigned long long a_obj = obj[e] + off, a_pool = sgl[e].addr + off;
-                ld_addr = TO_POOL ? a_obj : a_pool;
-                st_addr = TO_POOL ? a_pool : a_obj;
+            const uint32_t n_in = min(min(32u, cur_end - c), n_b - ei);
+            unsigned long long a_obj = 0, a_pool = 0;
+            uint32_t id_flags = 0;
+            if (lane < n_in) {
+                const tutti_sgl_t ent = sgl[e + lane];
+                a_pool = ent.addr + off;
+                id_flags = ent.id;
+            }
+            if (lane == 0) a_obj = obj[e] + off;
+            const bool rep = TO_POOL && lane > 0 && lane < n_in && (id_flags & TUTTI_SGL_FLAG_DUP);
+            const uint32_t reps = __ballot_sync(0xffffffffu, rep) | 1u;
+            const uint32_t m = (reps == 0xffffffffu) ? 32u : (uint32_t)(__ffs(~reps) - 1);
+            cur += m - 1;
+            if (TO_POOL) {
+                ld_addr = a_obj;
+                ld_bytes = (lane == 0) ? bytes : 0;
+                st_addr = a_pool;
+                st_bytes = (lane < m) ? bytes : 0;
+            } else if (lane == 0) {
+                ld_addr = a_pool;
+                st_addr = a_obj;
                 ld_bytes = bytes; st_bytes = bytes;
             }
         }
@@ -772,6 +870,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
             const uint32_t bar = smem_u32(&bars[s]);
             const uint32_t sbase = smem_u32(data + (size_t)s * CB);
             const uint32_t total_bytes = __reduce_add_sync(0xffffffffu, ld_bytes);
+            const uint32_t landed_bytes = __reduce_add_sync(0xffffffffu, st_bytes);
             if (lane == 0) mbar_expect_tx(bar, total_bytes);
             __syncwarp();
             if (n_hnd && TO_POOL) {
@@ -787,7 +886,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
             st_bytes_of[s * 32 + lane] = st_bytes;
             st_off_of[s * 32 + lane] = st_off;
             if (lane == 0) {
-                chunk_bytes_of[s] = total_bytes;
+                chunk_bytes_of[s] = landed_bytes;       // completion is counted in bytes landed
                 chunk_iocb_of[s] = n_bi | (n_hnd ? 0x80000000u : 0u);
             }
             __syncwarp();
@@ -806,7 +905,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
                     acct_bi = n_bi;
                 }
                 if (lane == 0) atomicCAS(&hdr_of(n_bi)->status, 0, TUTTI_ETIMEDOUT);
-                moved += __reduce_add_sync(0xffffffffu, ld_bytes);
+                moved += __reduce_add_sync(0xffffffffu, st_bytes);
                 fetch_next();
             } while (have_next);
             break;
@@ -899,12 +998,13 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     if (engine == 2) {
         // measured on B200: all SMs -> 2 warps x 3 stages x 32 KiB; a capped launch gets
         // closest to the per-SM ceiling (~49 GB/s each way) with 4 warps x 3 stages x 16 KiB
-        uint32_t warps = opt.bulk_warps ? opt.bulk_warps : (sm_count ? 4 : 2);
+        const bool capped_hbm = sm_count != 0;
+        uint32_t warps = opt.bulk_warps ? opt.bulk_warps : (capped_hbm ? 4 : 2);
         uint32_t stages = opt.bulk_stages ? opt.bulk_stages : 3;
         if (warps > 8) warps = 8;
         if (stages < 2) stages = 2;
         if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
-        uint32_t cb = opt.bulk_chunk ? opt.bulk_chunk : (sm_count ? 16384u : CHUNK_BYTES);
+        uint32_t cb = opt.bulk_chunk ? opt.bulk_chunk : (capped_hbm ? 16384u : CHUNK_BYTES);
         const size_t per_stage = cb + 8 + 32 * 16 + 8;
         while ((size_t)warps * stages * per_stage > 224u * 1024u) {
             if (stages > 2) --stages; else --warps;

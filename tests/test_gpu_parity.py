@@ -346,3 +346,33 @@ def test_whole_pass_of_a_short_prefix_in_one_launch(engine, sm_count, tokens):
             assert np.array_equal(t.cpu().numpy(), s)
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
+@pytest.mark.parametrize("sm_count", [0, 8])
+@pytest.mark.parametrize("chunk", [0, 8192])
+def test_shared_prefix_batch_grid_and_capped(engine, sm_count, chunk):
+    """8 requests sharing 75 % of their prefix: the shared objects are named once in the
+    descriptors and go to all eight requests' blocks, on all SMs and SM-capped, with stages
+    that hold a whole block and with stages that hold a piece of one."""
+    w = mk("shared-prefix-8-requests")
+    dc = DeviceCase(w, capacity=16)
+    try:
+        dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+        if chunk:
+            dc.ctx.tutti_set_option(T.OPT_BULK_CHUNK_BYTES, chunk)
+        layer = 1
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+        sq, sg, num, infos = dc.read_build(first, n)
+        orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 16)
+        assert same_records(sq, osq) and same_records(sg, osg)
+        n_dup = int(((sg["id"] & oracle.SGL_DUP) != 0).sum())
+        assert n_dup > len(sg) // 2                                  # most entries are repeats
+        assert int(sq["len"].sum()) < int(sg["len"].astype(np.uint64).sum()) // 2
+        dc.ring.tutti_kv_restore_layer(first, n, sm_count)
+        cqes = dc.poll_all(first, n)
+        assert all(c[1] == 0 for c in cqes)
+        assert sum(c[2] for c in cqes) == int(sg["len"].astype(np.uint64).sum())   # bytes landed
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+    finally:
+        dc.close()

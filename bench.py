@@ -1052,22 +1052,25 @@ def leg_config5(args, local_rank):
 def leg_sched_demo(args, local_rank, sched_host):
     """Layer-wise pipelining under the slack-aware scheduler (Section 3.3), with GEMMs standing
     in for a layer's compute: restores of the next layers are sized from the profiled tables
-    and issued on the I/O partition while the current layer computes on the other SMs."""
+    and issued on the I/O partition while the current layer computes on the other SMs.
+    IOCBs are cut by bytes (equal work), the I/O table is filled by the library's own
+    profiling pass, and the table's estimate is checked against launches it did not time."""
     import torch
     from paper_2605_03375_b200 import tutti as T
     a2 = argparse.Namespace(**vars(args))
     a2.config, a2.scale, a2.set = 2, 1.0, None
-    a2.ioctx_per_iocb = args.sched_ioctx
+    a2.ioctx_per_iocb = 2048
     a2.one_stream = True
     a2.layers_per_launch = 1
     a2.resident_layers = 8
+    n_layers = (args.layers or 6) if sched_host else (args.layers or 32)
+    rep = Replica(a2, local_rank, host_store=sched_host, n_layers=n_layers, ring_depth=2048)
     if sched_host:
         # objects in pinned host memory: the restore is bound by the host link, so a few
         # SMs carry it while the rest of the GPU computes
-        rep = Replica(a2, local_rank, host_store=True, n_layers=args.layers or 6)
         rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, T.ENGINE_BULK)
-    else:
-        rep = Replica(a2, local_rank, n_layers=args.layers or 32)
+    iocb_bytes = args.sched_iocb_mib << 20
+    rep.ring.tutti_ring_set_iocb_bytes(iocb_bytes)
     w, dev = rep.w, rep.dev
     io_sms = 8 if sched_host else args.sched_sms
     io_s, comp_s, got_io, got_comp = rep.ctx.tutti_sm_partition_create(io_sms)
@@ -1077,11 +1080,6 @@ def leg_sched_demo(args, local_rank, sched_host):
     A = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
     B = torch.randn(n, n, device=dev, dtype=torch.bfloat16)
     Cm = torch.empty(n, n, device=dev, dtype=torch.bfloat16)
-    gemms_per_layer = args.sched_gemms
-
-    def layer_compute():
-        for _ in range(gemms_per_layer):
-            torch.matmul(A, B, out=Cm)
 
     def timed(fn, stream):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -1093,21 +1091,22 @@ def leg_sched_demo(args, local_rank, sched_host):
         return a.elapsed_time(b)
 
     def build_all(stream):
-        built = []
         rep.epoch += 1
         rep.batch.plan_epoch = rep.epoch
-        for l in range(w.n_layers):
-            rc, first, cnt = rep.ring.tutti_build_sqes(rep.batch, l, T.OP_READ, stream=stream)
-            built.append((first, cnt))
-        return built
+        rc, first, per = rep.ring.tutti_build_sqes_layers(rep.batch, 0, w.n_layers, T.OP_READ,
+                                                          stream=stream)
+        return [(first + l * per, per) for l in range(w.n_layers)]
 
     def poll(built):
-        for first, cnt in built:
-            for i in range(first, first + cnt):
-                rc, cqe = rep.ring.tutti_ring_poll(i, 20_000_000_000)
-                assert rc == T.OK and cqe.status == 0
+        rep.poll_list(built)
 
-    # how many IOCBs does a layer really use (the rest of the reservation is empty)?
+    # warm-up profiling inside the library: restore time against the IOCB count on the I/O
+    # partition (1, 2, 4, ... and all IOCBs of a layer)
+    sched = T.Scheduler(w.n_layers, 32, 65536, 65536)
+    rep.epoch += 1
+    rep.batch.plan_epoch = rep.epoch
+    n_points = sched.tutti_sched_profile(rep.ring, rep.batch, 0, T.OP_READ, [got_io], reps=2,
+                                         stream=io_stream)
     built = build_all(io_stream)
     torch.cuda.synchronize()
     used = sum(1 for i in range(built[0][0], built[0][0] + built[0][1])
@@ -1115,23 +1114,39 @@ def leg_sched_demo(args, local_rank, sched_host):
     for first, cnt in built:
         rep.ring.tutti_kv_restore_layer(first, cnt, got_io, stream=io_stream)
     poll(built)
-
-    # offline profiles: (1) I/O kernel time against IOCB count on the I/O partition
-    sched = T.Scheduler(w.n_layers, 32, 65536, 65536)
-    profile = {}
-    for k in sorted({1, 2, max(1, used // 2), used}):
+    profile = {k: round(sched.tutti_sched_io_time(T.OP_READ, got_io, k), 1)
+               for k in sorted({1, 2, 4, 8, used})}
+    # the table against launches it has not seen: IOCB counts between the profiled points
+    est_err = {}
+    for k in sorted({3, 5, max(1, used - 3)}):
+        if k >= used:
+            continue
         built = build_all(io_stream)
         first = built[0][0]
         ms = timed(lambda: rep.ring.tutti_kv_restore_layer(first, k, got_io, stream=io_stream),
                    io_stream)
-        for f, c in built:
+        rep.ring.tutti_kv_restore_layer(first + k, built[0][1] - k, got_io, stream=io_stream)
+        for f, c in built[1:]:
             rep.ring.tutti_kv_restore_layer(f, c, got_io, stream=io_stream)
         poll(built)
-        sched.tutti_sched_set_io_time(T.OP_READ, got_io, k, ms * 1e3)
-        profile[k] = round(ms * 1e3, 1)
-    # (2) the layer's window: its compute time on the compute partition
+        est = sched.tutti_sched_io_time(T.OP_READ, got_io, k)
+        est_err[k] = {"measured_us": round(ms * 1e3, 1), "estimated_us": round(est, 1),
+                      "error": round(abs(est - ms * 1e3) / (ms * 1e3), 4)}
+    layer_restore_ms = profile[used] / 1e3
+    # the layer's window: its compute time on the compute partition.  From HBM a layer's KV
+    # arrives in a fraction of a 3-GEMM layer; from pinned host memory the link needs ~20 ms
+    # per GiB layer, so the stand-in layer is made that long (a long prefill chunk)
     with torch.cuda.stream(comp_stream):
-        layer_compute()
+        torch.matmul(A, B, out=Cm)
+        gemm_ms = timed(lambda: [torch.matmul(A, B, out=Cm) for _ in range(4)], comp_stream) / 4
+    gemms_per_layer = args.sched_gemms
+    if sched_host:
+        gemms_per_layer = max(gemms_per_layer, int(1.15 * layer_restore_ms / gemm_ms) + 1)
+
+    def layer_compute():
+        for _ in range(gemms_per_layer):
+            torch.matmul(A, B, out=Cm)
+    with torch.cuda.stream(comp_stream):
         layer_ms = timed(layer_compute, comp_stream)
     l_in, l_pre = 8192, 32768
     sched.tutti_sched_set_slack(l_in, l_pre, layer_ms * 1e3, got_io)
@@ -1153,8 +1168,7 @@ def leg_sched_demo(args, local_rank, sched_host):
                     layer_compute()
         else:
             for l, (first, cnt) in enumerate(built):
-                sched.tutti_sched_enqueue(T.OP_READ, l, first, cnt)
-            done_ev = {}
+                sched.tutti_sched_enqueue(T.OP_READ, l, first, used)
             for l in range(w.n_layers):
                 # before layer l begins: launch what the window holds (at least layer l's reads)
                 for (op, first, cnt, sms, lay, est) in sched.tutti_sched_next(
@@ -1162,26 +1176,21 @@ def leg_sched_demo(args, local_rank, sched_host):
                     rep.ring.tutti_kv_restore_layer(first, cnt, sms, stream=io_stream)
                 # layer l may start once its own IOCBs are done (they were launched now or
                 # earlier); reads launched ahead for later layers do not hold it back
-                if used <= 8:
-                    for i in range(built[l][0], built[l][0] + used):
-                        rep.ring.tutti_stream_wait_iocb(i, comp_stream)
-                else:
-                    # many small IOCBs per layer: one event after everything launched so far
-                    # costs less than a stream wait per IOCB
-                    ev = torch.cuda.Event()
-                    ev.record(io_stream)
-                    comp_stream.wait_event(ev)
+                for i in range(built[l][0], built[l][0] + used):
+                    rep.ring.tutti_stream_wait_iocb(i, comp_stream)
                 with torch.cuda.stream(comp_stream):
                     layer_compute()
             assert sched.tutti_sched_pending() == (0, 0)
+            # the empty tail of every layer's reservation completes too
+            for first, cnt in built:
+                if cnt > used:
+                    rep.ring.tutti_kv_restore_layer(first + used, cnt - used, got_io, stream=io_stream)
         t1.record(comp_stream)
         torch.cuda.synchronize()
-        if mode != "compute_only":
-            poll(built)
-        else:
+        if mode == "compute_only":
             for f, c in built:
                 rep.ring.tutti_kv_restore_layer(f, c, 0, stream=io_stream)
-            poll(built)
+        poll(built)
         return t0.elapsed_time(t1)
 
     res = {m: round(min(run(m) for _ in range(3)), 3) for m in ("compute_only", "serial", "scheduled")}
@@ -1189,9 +1198,12 @@ def leg_sched_demo(args, local_rank, sched_host):
     out = {"demo": "slack-aware layer-wise pipelining, config-2 batch, GEMMs as layer compute",
            "store": "pinned host, zero-copy" if sched_host else "hbm", "layers": w.n_layers,
            "io_partition_sms": got_io, "compute_partition_sms": got_comp,
-           "ioctx_per_iocb": args.sched_ioctx, "iocbs_per_layer_used": used,
-           "io_profile_us_by_iocbs": profile, "layer_compute_ms": round(layer_ms, 3),
-           "restore_ms_per_layer_on_partition": round(profile[used] / 1e3, 3),
+           "iocb_mib": args.sched_iocb_mib, "iocbs_per_layer_used": used,
+           "profile": "tutti_sched_profile (library), %d table entries" % n_points,
+           "io_profile_us_by_iocbs": profile,
+           "estimate_vs_measured": est_err,
+           "gemms_per_layer": gemms_per_layer, "layer_compute_ms": round(layer_ms, 3),
+           "restore_ms_per_layer_on_partition": round(layer_restore_ms, 3),
            "total_ms": res,
            "bubble_ms_scheduled": round(res["scheduled"] - res["compute_only"], 3),
            "bubble_ms_serial": round(res["serial"] - res["compute_only"], 3),
@@ -1329,7 +1341,8 @@ def main():
                     help="layer-wise pipelining under the slack-aware scheduler")
     ap.add_argument("--sched-host", action="store_true")
     ap.add_argument("--sched-sms", type=int, default=16)
-    ap.add_argument("--sched-ioctx", type=int, default=16)
+    ap.add_argument("--sched-iocb-mib", type=int, default=64,
+                    help="scheduler legs: bytes per IOCB (IOCBs cut by bytes)")
     ap.add_argument("--sched-gemms", type=int, default=3)
     ap.add_argument("--layers-per-launch", type=int, default=0,
                     help="consecutive layers whose IOCBs one copy launch executes "

@@ -220,8 +220,9 @@ int tutti_obj_layout(const tutti_geom_t *geom, tutti_layout_t *out);
  * the store; a completion's bytes are the bytes that landed (entries x length).
  *   batch        host pointer to the struct; its arrays are device pointers.
  *   first_iocb,  host out: indices of the reserved IOCBs, known without waiting
- *   n_iocb       for the GPU: ceil(2*n_obj / ioctx_per_iocb), at least 1.  IOCBs
- *                the build does not need are published with num_ioctx = 0.
+ *   n_iocb       for the GPU: ceil(2*n_obj / ioctx_per_iocb), at least 1 (or the
+ *                count tutti_ring_set_iocb_bytes states).  IOCBs the build does
+ *                not need are published with num_ioctx = 0.
  * Asynchronous on `stream`.  TUTTI_EAGAIN if the ring or the SGL arena has no
  * room (poll completed IOCBs first); TUTTI_EINVAL for layer >= n_layers, unknown
  * opcode, unregistered pool layer / store device, or a batch larger than the ring
@@ -344,6 +345,18 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
                       uint32_t sgl_capacity, uint32_t max_items, tutti_ring_t **out);
 int tutti_ring_destroy(tutti_ring_t *ring);
 
+/* IOCBs of equal work (Section 3.2: the paper's IOCB is a uniform batch of 2048 equal I/O
+ * contexts, which is what lets Section 3.3 profile kernel time against the IOCB count).  Here
+ * contexts are coalesced runs of very different length, so by default an IOCB (ioctx_per_iocb
+ * contexts) is not a unit of time.  With bytes != 0, builds made afterwards on this ring cut
+ * IOCBs by bytes instead: IOCB k of a build takes the scatter-gather entries from entry
+ * k * (bytes / block_bytes) to entry (k + 1) * (bytes / block_bytes), each boundary moved back
+ * so that a TUTTI_SGL_FLAG_DUP entry stays with the entry it repeats; a context that crosses
+ * a boundary is cut there into two.  A build then reserves ceil(2 * n_blk * block_bytes /
+ * bytes) IOCBs per layer.  bytes / block_bytes must be 1..ioctx_per_iocb (TUTTI_EINVAL);
+ * bytes = 0 goes back to IOCBs of ioctx_per_iocb contexts. */
+int tutti_ring_set_iocb_bytes(tutti_ring_t *ring, uint64_t bytes);
+
 /* get_iocb(nums) for descriptors prepared by the CPU (the paper's own split,
  * Section 3.2: "CPU-prepared, GPU-executed"): reserve n IOCBs and n_sgl arena
  * entries without building anything. */
@@ -455,6 +468,21 @@ int tutti_sched_set_io_time(tutti_sched_t *sched, uint32_t opcode, uint32_t sm_c
                             uint32_t n_iocb, float us);
 int tutti_sched_io_time(const tutti_sched_t *sched, uint32_t opcode, uint32_t sm_count,
                         uint32_t n_iocb, float *us);
+/* The profiling pass itself (Section 3.3 "offline profiling ... kernel time and SM occupancy
+ * vs IOCB count"; Section 3.4: done once at warm-up).  For every SM count in sm_counts[0..n_sm)
+ * (0 = all SMs) it times launches of 1, 2, 4, ... and all of the IOCBs that one layer's build
+ * of `batch` fills, with CUDA events on `stream` (minimum of `reps` launches per point), and
+ * enters the times into the scheduler's I/O table.  opcode TUTTI_OP_READ times
+ * tutti_kv_restore_layer, TUTTI_OP_WRITE tutti_kv_save_layer.  The transfers really run:
+ * layer `layer` of the pool (READ) or the batch's objects of that layer (WRITE) are
+ * overwritten as by any restore / save.  Blocks the host until done: a warm-up call, not for
+ * the per-layer path.  With IOCBs cut by bytes (tutti_ring_set_iocb_bytes) every IOCB is the
+ * same work and the table is exact; otherwise it is an average over unequal IOCBs.
+ * *n_points (may be NULL): table entries written. */
+int tutti_sched_profile(tutti_ctx_t *ctx, tutti_ring_t *ring, tutti_sched_t *sched,
+                        const tutti_batch_t *batch, uint32_t layer, uint32_t opcode,
+                        const uint32_t *sm_counts, uint32_t n_sm, uint32_t reps, void *stream,
+                        uint32_t *n_points);
 /* Queue built IOCBs: reads when a request arrives, writes when a layer's KV is produced. */
 int tutti_sched_enqueue(tutti_sched_t *sched, uint32_t opcode, uint32_t layer, uint32_t first_iocb,
                         uint32_t n_iocb);

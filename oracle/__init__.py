@@ -195,21 +195,26 @@ def row_location(g: Geom, layer: int, batch, r: int, t: int, kv: int, head: int,
 
 
 def build_descriptors(g: Geom, layer: int, opcode: int, batch, k_base_addr: int,
-                      v_base_addr: int, block_stride: int, capacity: int):
+                      v_base_addr: int, block_stride: int, capacity: int,
+                      entries_per_iocb: int = 0):
     """Returns (rc, sqes, sgl, num_ioctx) — structured arrays SQE_DTYPE / SGL_DTYPE and the
-    per-IOCB context counts."""
+    per-IOCB context counts.  entries_per_iocb != 0: IOCBs are cut every that many
+    scatter-gather entries (equal work) instead of every `capacity` contexts."""
     keep, bargs = _batch(*batch)
     hit, os_, osl, bs, bi = keep
-    max_sqe = 2 * int(osl.shape[0]) + 1
     max_sgl = 2 * int(bi.shape[0]) + 1
-    max_iocb = max_sqe // max(capacity, 1) + 2
+    max_iocb = (2 * int(osl.shape[0]) + 1) // max(capacity, 1) + 2
+    if entries_per_iocb:
+        max_iocb = max_sgl // entries_per_iocb + 2
+    max_sqe = 2 * int(osl.shape[0]) + 1 + max_iocb
     sqes = np.zeros(max_sqe, dtype=SQE_DTYPE)
     sgl = np.zeros(max_sgl, dtype=SGL_DTYPE)
     num = np.zeros(max_iocb, dtype=np.uint32)
     n_sqe, n_sgl, n_iocb = C.c_uint32(), C.c_uint32(), C.c_uint32()
-    rc = lib().orc_build(C.byref(g), C.c_uint32(layer), C.c_uint32(opcode), *bargs,
+    rc = lib().orc_build_budget(C.byref(g), C.c_uint32(layer), C.c_uint32(opcode), *bargs,
                          C.c_uint64(k_base_addr), C.c_uint64(v_base_addr),
                          C.c_uint64(block_stride), C.c_uint32(capacity),
+                         C.c_uint32(entries_per_iocb),
                          C.c_void_p(sqes.ctypes.data), C.c_uint32(max_sqe),
                          C.c_void_p(sgl.ctypes.data), C.c_uint32(max_sgl), _p(num, C.c_uint32),
                          C.c_uint32(max_iocb), C.byref(n_sqe), C.byref(n_sgl), C.byref(n_iocb))

@@ -309,18 +309,80 @@ static int item_cmp(const void *pa, const void *pb)
 }
 
 /*
+ * Step 5, second form: IOCBs of (nearly) equal work instead of equal context count, so that
+ * "n IOCBs" is a unit of transfer time as it is with the paper's uniform IOCBs (Section 3.2:
+ * an IOCB is a batch of 2048 equal I/O contexts; Section 3.3 profiles kernel time against the
+ * IOCB count).  IOCB k takes the scatter-gather entries from boundary k to boundary k + 1,
+ * where boundary k is entry k * entries_per_iocb moved back to the first entry of its source
+ * block (a repeat is never separated from the bytes it repeats); a context that crosses a
+ * boundary is cut there into two contexts.  The contexts are rewritten in place.
+ */
+static int pack_by_entries(orc_sqe *sqes, uint32_t ns, uint32_t max_sqe, const orc_sgl *sgl,
+                           uint32_t ne, uint32_t capacity, uint32_t per, uint32_t *num_ioctx,
+                           uint32_t max_iocb, uint32_t *n_sqe, uint32_t *n_sgl, uint32_t *n_iocb)
+{
+    uint32_t nb = (ne + per - 1) / per;
+    if (nb == 0) nb = 1;
+    if (nb > max_iocb) return ORC_ENOSPC;
+    orc_sqe *whole = (orc_sqe *)malloc((ns ? ns : 1) * sizeof(orc_sqe));
+    if (!whole) return ORC_ENOSPC;
+    memcpy(whole, sqes, ns * sizeof(orc_sqe));
+    uint32_t out = 0, s = 0;
+    for (uint32_t k = 0; k < nb; ++k) {
+        uint64_t y0 = (uint64_t)k * per, y1 = (uint64_t)(k + 1) * per;
+        uint32_t lo = y0 < ne ? (uint32_t)y0 : ne, hi = y1 < ne ? (uint32_t)y1 : ne;
+        while (lo < ne && lo > 0 && (sgl[lo].id & ORC_SGL_DUP)) --lo;
+        while (hi < ne && hi > 0 && (sgl[hi].id & ORC_SGL_DUP)) --hi;
+        uint32_t count = 0;
+        /* the contexts that have entries in [lo, hi) */
+        while (s < ns && whole[s].sgl_first + whole[s].sgl_count <= lo) ++s;
+        for (uint32_t t = s; t < ns && whole[t].sgl_first < hi; ++t) {
+            uint32_t a = whole[t].sgl_first > lo ? whole[t].sgl_first : lo;
+            uint32_t b = whole[t].sgl_first + whole[t].sgl_count < hi
+                             ? whole[t].sgl_first + whole[t].sgl_count : hi;
+            if (a >= b) continue;
+            if (out >= max_sqe) { free(whole); return ORC_ENOSPC; }
+            orc_sqe *p = &sqes[out++];
+            *p = whole[t];
+            /* object bytes named before entry a, and by the entries [a, b) */
+            uint64_t before = 0, named = 0;
+            for (uint32_t e = whole[t].sgl_first; e < a; ++e)
+                if (!(sgl[e].id & ORC_SGL_DUP)) before += sgl[e].len;
+            for (uint32_t e = a; e < b; ++e)
+                if (!(sgl[e].id & ORC_SGL_DUP)) named += sgl[e].len;
+            p->src_off = whole[t].src_off + before;
+            p->len = named;
+            p->sgl_first = a;
+            p->sgl_count = b - a;
+            ++count;
+        }
+        if (count > capacity) { free(whole); return ORC_EINVAL; }
+        num_ioctx[k] = count;
+    }
+    free(whole);
+    *n_sqe = out;
+    *n_sgl = ne;
+    *n_iocb = nb;
+    return ORC_OK;
+}
+
+/*
  * Build one layer's descriptors.
  *   sqes[max_sqe], sgl[max_sgl], num_ioctx[max_iocb] are outputs; *n_sqe, *n_sgl,
  *   *n_iocb the counts produced.  SQE k belongs to IOCB k / capacity at position
  *   k % capacity.  n_iocb = ceil(n_sqe / capacity), at least 1 (an empty batch
- *   yields one IOCB with num_ioctx = 0).
+ *   yields one IOCB with num_ioctx = 0).  With entries_per_iocb != 0 the IOCBs are cut by
+ *   scatter-gather entries instead (see pack_by_entries): n_iocb = ceil(n_sgl /
+ *   entries_per_iocb), IOCB b holds num_ioctx[b] consecutive contexts of the output.
  */
-int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req,
-              const uint32_t *hit_tokens, const uint32_t *obj_start, const uint32_t *obj_slot,
-              const uint32_t *blk_start, const int32_t *block_ids, uint64_t k_base_addr,
-              uint64_t v_base_addr, uint64_t block_stride, uint32_t capacity, orc_sqe *sqes,
-              uint32_t max_sqe, orc_sgl *sgl, uint32_t max_sgl, uint32_t *num_ioctx,
-              uint32_t max_iocb, uint32_t *n_sqe, uint32_t *n_sgl, uint32_t *n_iocb)
+int orc_build_budget(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req,
+                     const uint32_t *hit_tokens, const uint32_t *obj_start,
+                     const uint32_t *obj_slot, const uint32_t *blk_start,
+                     const int32_t *block_ids, uint64_t k_base_addr, uint64_t v_base_addr,
+                     uint64_t block_stride, uint32_t capacity, uint32_t entries_per_iocb,
+                     orc_sqe *sqes, uint32_t max_sqe, orc_sgl *sgl, uint32_t max_sgl,
+                     uint32_t *num_ioctx, uint32_t max_iocb, uint32_t *n_sqe, uint32_t *n_sgl,
+                     uint32_t *n_iocb)
 {
     orc_layout lo;
     int rc = orc_obj_layout(g, &lo);
@@ -404,6 +466,10 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
     }
     free(items);
 
+    if (entries_per_iocb != 0)
+        return pack_by_entries(sqes, ns, max_sqe, sgl, ne, capacity, entries_per_iocb, num_ioctx,
+                               max_iocb, n_sqe, n_sgl, n_iocb);
+
     /* step 5: pack into IOCBs of `capacity` contexts */
     uint32_t nb = (ns + capacity - 1) / capacity;
     if (nb == 0) nb = 1;
@@ -416,6 +482,18 @@ int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req
     *n_sgl = ne;
     *n_iocb = nb;
     return ORC_OK;
+}
+
+int orc_build(const orc_geom *g, uint32_t layer, uint32_t opcode, uint32_t n_req,
+              const uint32_t *hit_tokens, const uint32_t *obj_start, const uint32_t *obj_slot,
+              const uint32_t *blk_start, const int32_t *block_ids, uint64_t k_base_addr,
+              uint64_t v_base_addr, uint64_t block_stride, uint32_t capacity, orc_sqe *sqes,
+              uint32_t max_sqe, orc_sgl *sgl, uint32_t max_sgl, uint32_t *num_ioctx,
+              uint32_t max_iocb, uint32_t *n_sqe, uint32_t *n_sgl, uint32_t *n_iocb)
+{
+    return orc_build_budget(g, layer, opcode, n_req, hit_tokens, obj_start, obj_slot, blk_start,
+                            block_ids, k_base_addr, v_base_addr, block_stride, capacity, 0, sqes,
+                            max_sqe, sgl, max_sgl, num_ioctx, max_iocb, n_sqe, n_sgl, n_iocb);
 }
 
 /*

@@ -370,8 +370,39 @@ struct EmitParams {
     uint64_t store_base[TUTTI_MAX_DEVICES];
     uint64_t store_bytes[TUTTI_MAX_DEVICES];
     uint32_t first_iocb, n_iocb, sgl_base, sgl_reserved;
+    uint32_t entries_per_iocb;   // 0: IOCBs of `capacity` contexts; else IOCBs cut by entries
     const PoolLayerDev *pools;   // per-layer pool table for launches that cover several layers
 };
+
+// IOCBs of equal work: boundary k of a build is scatter-gather entry k * entries_per_iocb moved
+// back to the first entry of its source block (a repeat is never separated from the bytes it
+// repeats).  A cut: the boundary's entry index, the context that holds it and the object-side
+// offset (layer 0) its source block starts at.
+struct Cut {
+    uint32_t entry;
+    uint32_t sq;
+    unsigned long long src;
+};
+
+__device__ Cut cut_at(const RingDev &ring, const GeomDev &g, uint32_t n_items, uint32_t n_entries,
+                      unsigned long long y) {
+    Cut c{n_entries, 0xffffffffu, 0};
+    if (y >= n_entries) return c;
+    // the item whose share of the entries, [cumblk[i], cumblk[i + 1]), holds y
+    uint32_t lo = 0, hi = n_items;
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (ring.plan_cumblk[mid] <= y) lo = mid; else hi = mid;
+    }
+    // its group lists block j of the source k_copies times in a row
+    const uint32_t gs = ring.plan_grp[lo];
+    const uint32_t first = ring.plan_cumblk[gs], k_copies = ring.plan_k[gs];
+    const uint32_t j = ((uint32_t)y - first) / k_copies;
+    c.entry = first + j * k_copies;
+    c.sq = ring.plan_sqe_of[gs];
+    c.src = (ring.plan_off[gs] & ((1ull << 56) - 1)) + (unsigned long long)j * g.block_bytes;
+    return c;
+}
 
 // blockIdx.y selects the layer of a multi-layer launch: layer p.layer + y, whose IOCBs and
 // arena range follow those of the layer before it.
@@ -397,38 +428,84 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
     const unsigned long long layer_off = (unsigned long long)p.layer * g.stride_layer;
 
     // IOCB headers (step 7 of the path): CTA 0
+    const uint32_t per = p.entries_per_iocb;
     if (blockIdx.x == 0) {
         for (uint32_t k = threadIdx.x; k < p.n_iocb; k += blockDim.x) {
             uint32_t idx = p.first_iocb + k;
             IocbHdr *h = &ring.hdrs[idx & (ring.depth - 1)];
-            unsigned long long s0 = (unsigned long long)k * ring.capacity;
-            unsigned long long s1 = s0 + ring.capacity;
-            uint32_t e0 = s0 < n_sqe ? ring.plan_sqe[s0].sgl_first : n_entries;
-            uint32_t e1 = s1 < n_sqe ? ring.plan_sqe[s1].sgl_first : n_entries;
-            h->num_ioctx = s0 < n_sqe ? (uint32_t)((s1 < n_sqe ? s1 : n_sqe) - s0) : 0;
+            uint32_t e0, e1, n_ctx;
+            if (per == 0) {
+                unsigned long long s0 = (unsigned long long)k * ring.capacity;
+                unsigned long long s1 = s0 + ring.capacity;
+                e0 = s0 < n_sqe ? ring.plan_sqe[s0].sgl_first : n_entries;
+                e1 = s1 < n_sqe ? ring.plan_sqe[s1].sgl_first : n_entries;
+                n_ctx = s0 < n_sqe ? (uint32_t)((s1 < n_sqe ? s1 : n_sqe) - s0) : 0;
+            } else {
+                const Cut a = cut_at(ring, g, n_items, n_entries, (unsigned long long)k * per);
+                const Cut b = cut_at(ring, g, n_items, n_entries, (unsigned long long)(k + 1) * per);
+                e0 = a.entry;
+                e1 = b.entry;
+                n_ctx = 0;
+                if (e1 > e0) {
+                    // contexts with entries in [e0, e1): from the one holding e0 to the one
+                    // holding e1 - 1
+                    const uint32_t last = (b.sq == 0xffffffffu) ? n_sqe - 1
+                                          : (e1 > ring.plan_sqe[b.sq].sgl_first ? b.sq : b.sq - 1);
+                    n_ctx = last - a.sq + 1;
+                }
+            }
+            h->num_ioctx = n_ctx;
             h->opcode = p.opcode;
             h->layer = p.layer;
-            h->status = status;
+            h->status = (n_ctx > ring.capacity && status == 0) ? TUTTI_EINVAL : status;
             h->sgl_base = p.sgl_base;
             h->entry_first = e0;
-            h->total_entries = e1 - e0;
+            h->total_entries = (n_ctx > ring.capacity) ? 0 : e1 - e0;
             h->entry_len = (uint32_t)g.block_bytes;
             h->claim_cursor = 0;
             h->done_bytes = 0;
-            h->bytes = (unsigned long long)(e1 - e0) * g.block_bytes;
+            h->bytes = (n_ctx > ring.capacity) ? 0 : (unsigned long long)(e1 - e0) * g.block_bytes;
         }
     }
 
     // contexts, rebased to this layer and packed into IOCBs
     const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t gthreads = gridDim.x * blockDim.x;
-    for (uint32_t k = gtid; k < n_sqe; k += gthreads) {
-        tutti_sqe_t e = ring.plan_sqe[k];
-        e.src_off += layer_off;
-        e.opcode = (uint16_t)p.opcode;
-        e.layer = (uint16_t)p.layer;
-        uint32_t slot = (p.first_iocb + k / ring.capacity) & (ring.depth - 1);
-        ring.sqes[(size_t)slot * ring.capacity + k % ring.capacity] = e;
+    if (per == 0) {
+        for (uint32_t k = gtid; k < n_sqe; k += gthreads) {
+            tutti_sqe_t e = ring.plan_sqe[k];
+            e.src_off += layer_off;
+            e.opcode = (uint16_t)p.opcode;
+            e.layer = (uint16_t)p.layer;
+            uint32_t slot = (p.first_iocb + k / ring.capacity) & (ring.depth - 1);
+            ring.sqes[(size_t)slot * ring.capacity + k % ring.capacity] = e;
+        }
+    } else {
+        // one IOCB per CTA at a time; a context that crosses a boundary is cut there
+        for (uint32_t k = blockIdx.x; k < p.n_iocb; k += gridDim.x) {
+            const Cut a = cut_at(ring, g, n_items, n_entries, (unsigned long long)k * per);
+            const Cut b = cut_at(ring, g, n_items, n_entries, (unsigned long long)(k + 1) * per);
+            if (b.entry <= a.entry) continue;
+            const uint32_t last = (b.sq == 0xffffffffu) ? n_sqe - 1
+                                  : (b.entry > ring.plan_sqe[b.sq].sgl_first ? b.sq : b.sq - 1);
+            const uint32_t n_ctx = last - a.sq + 1;
+            if (n_ctx > ring.capacity) continue;                 // reported in the header
+            const uint32_t slot = (p.first_iocb + k) & (ring.depth - 1);
+            for (uint32_t q = threadIdx.x; q < n_ctx; q += blockDim.x) {
+                const tutti_sqe_t whole = ring.plan_sqe[a.sq + q];
+                const uint32_t w_end = whole.sgl_first + whole.sgl_count;
+                tutti_sqe_t e = whole;
+                const unsigned long long src0 = whole.sgl_first >= a.entry ? whole.src_off : a.src;
+                const unsigned long long src1 = w_end <= b.entry ? whole.src_off + whole.len : b.src;
+                e.src_off = src0 + layer_off;
+                e.len = src1 - src0;
+                e.sgl_first = max(whole.sgl_first, a.entry);
+                e.sgl_count = min(w_end, b.entry) - e.sgl_first;
+                e.opcode = (uint16_t)p.opcode;
+                e.layer = (uint16_t)p.layer;
+                ring.sqes[(size_t)slot * ring.capacity + q] = e;
+            }
+        }
     }
 
     // SGL entries: a group of G lanes per item, lanes over the item's blocks.  G is the
@@ -595,9 +672,10 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
                         uint32_t layer, uint32_t n_layers, uint32_t opcode, const PoolLayer &pool,
                         const PoolLayerDev *pools, const uint64_t *store_base,
                         const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
-                        uint32_t sgl_base, uint32_t sgl_reserved, int device_sms,
-                        cudaStream_t stream) {
+                        uint32_t sgl_base, uint32_t sgl_reserved, uint32_t entries_per_iocb,
+                        int device_sms, cudaStream_t stream) {
     EmitParams p;
+    p.entries_per_iocb = entries_per_iocb;
     p.layer = layer;
     p.opcode = opcode;
     p.k_base = pool.k_base;

@@ -140,8 +140,8 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
                         uint32_t layer, uint32_t n_layers, uint32_t opcode, const PoolLayer &pool,
                         const PoolLayerDev *pools, const uint64_t *store_base,
                         const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
-                        uint32_t sgl_base, uint32_t sgl_reserved, int device_sms,
-                        cudaStream_t stream);
+                        uint32_t sgl_base, uint32_t sgl_reserved, uint32_t entries_per_iocb,
+                        int device_sms, cudaStream_t stream);
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
                         bool pool_hnd, const PermGeom &perm, const StoreTensorMaps *maps,

@@ -87,6 +87,7 @@ struct tutti_ring {
     std::vector<uint8_t> issued;          // per slot: a copy launch that executes it was enqueued
     std::vector<uint64_t> fill_optr;      // tutti_ring_fill_host scratch (sized at create)
     std::vector<uint8_t> fill_seen;
+    uint32_t entries_per_iocb = 0;        // IOCBs cut by entries (0: by context count)
     uint32_t *smid_log = nullptr;         // device: SM of every CTA of the last copy launch
     uint32_t smid_cap = 0, last_grid = 0;
     uint32_t sgl_capacity;
@@ -407,6 +408,16 @@ int tutti_ring_destroy(tutti_ring_t *r) {
     return TUTTI_OK;
 }
 
+int tutti_ring_set_iocb_bytes(tutti_ring_t *r, uint64_t bytes) {
+    if (!r) return TUTTI_EINVAL;
+    if (bytes == 0) { r->entries_per_iocb = 0; return TUTTI_OK; }
+    const uint64_t per = bytes / r->ctx->layout.block_bytes;
+    // every context of an IOCB holds at least one entry, so `per` contexts always fit
+    if (per == 0 || per > r->dev.capacity) return TUTTI_EINVAL;
+    r->entries_per_iocb = (uint32_t)per;
+    return TUTTI_OK;
+}
+
 int tutti_ring_stats(tutti_ring_t *r, uint64_t *kernel_launches, uint64_t *host_calls) {
     if (!r) return TUTTI_EINVAL;
     if (kernel_launches) *kernel_launches = r->kernel_launches;
@@ -439,7 +450,9 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
     if (batch->n_obj > r->dev.max_items / 2 || batch->n_blk > 0x7fffffffu / 2) return TUTTI_EINVAL;
     const uint32_t items = 2u * batch->n_obj;
     const uint32_t need_sgl = 2u * batch->n_blk;
-    uint32_t need_iocb = (items + r->dev.capacity - 1) / r->dev.capacity;
+    uint32_t need_iocb = r->entries_per_iocb
+                             ? (need_sgl + r->entries_per_iocb - 1) / r->entries_per_iocb
+                             : (items + r->dev.capacity - 1) / r->dev.capacity;
     if (need_iocb == 0) need_iocb = 1;
     if ((uint64_t)need_sgl * n_layers > r->sgl_capacity) return TUTTI_EINVAL;
     if ((uint64_t)need_iocb * n_layers > r->dev.depth) return TUTTI_EINVAL;
@@ -482,7 +495,7 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
     const uint32_t op_flags = opcode | (ctx->pool_hnd ? TUTTI_OP_FLAG_HND : 0u);
     CK_OR_CANCEL(launch_emit(r->dev, ctx->gdev, b, layer, n_layers, op_flags, ctx->pool[layer],
                              n_layers > 1 ? ctx->d_pools : nullptr, sbase, sbytes, first, need_iocb,
-                             sgl_base, need_sgl, ctx->device_sms, st));
+                             sgl_base, need_sgl, r->entries_per_iocb, ctx->device_sms, st));
 #undef CK_OR_CANCEL
     r->kernel_launches++;
     *first_iocb = first;
@@ -614,6 +627,75 @@ int tutti_ring_poll_range(tutti_ring_t *r, uint32_t first_iocb, uint32_t n_iocb,
     if (bytes_total) *bytes_total = bytes;
     if (first_error) *first_error = err;
     if (n_done) *n_done = done;
+    return rc;
+}
+
+int tutti_sched_profile(tutti_ctx_t *ctx, tutti_ring_t *r, tutti_sched_t *sched,
+                        const tutti_batch_t *batch, uint32_t layer, uint32_t opcode,
+                        const uint32_t *sm_counts, uint32_t n_sm, uint32_t reps, void *stream,
+                        uint32_t *n_points) {
+    if (!ctx || !r || r->ctx != ctx || !sched || !batch || !sm_counts || n_sm == 0 || reps == 0 ||
+        (opcode != TUTTI_OP_READ && opcode != TUTTI_OP_WRITE))
+        return TUTTI_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    CK(cudaEventCreate(&e0));
+    cudaError_t ce = cudaEventCreate(&e1);
+    if (ce != cudaSuccess) { cudaEventDestroy(e0); return cuda_fail(ce, "cudaEventCreate"); }
+    uint32_t points = 0;
+    int rc = TUTTI_OK;
+    // one build to learn how many IOCBs of a layer carry work (the rest of a reservation is empty)
+    uint32_t first = 0, n = 0, used = 0;
+    rc = tutti_build_sqes(ctx, r, batch, layer, opcode, stream, &first, &n);
+    if (rc == TUTTI_OK) {
+        for (uint32_t k = 0; k < n && rc == TUTTI_OK; ++k) {
+            tutti_iocb_info_t info;
+            rc = tutti_ring_read_iocb(r, first + k, &info, nullptr, 0);
+            if (rc == TUTTI_OK && info.status != 0) rc = info.status;
+            if (rc == TUTTI_OK && info.total_entries) used = k + 1;
+        }
+        int rc2 = issue(ctx, r, first, n, 0, stream, opcode);
+        if (rc == TUTTI_OK) rc = rc2;
+        if (rc2 == TUTTI_OK) tutti_ring_poll_range(r, first, n, nullptr, nullptr, nullptr, 5000000000ull);
+    }
+    for (uint32_t si = 0; si < n_sm && rc == TUTTI_OK && used; ++si) {
+        const uint32_t sms = sm_counts[si];
+        for (uint32_t cnt = 1; rc == TUTTI_OK; cnt = (cnt * 2 < used || cnt == used) ? cnt * 2 : used) {
+            if (cnt > used) break;
+            float best = 0.f;
+            for (uint32_t rep = 0; rep < reps && rc == TUTTI_OK; ++rep) {
+                rc = tutti_build_sqes(ctx, r, batch, layer, opcode, stream, &first, &n);
+                if (rc != TUTTI_OK) break;
+                // the launch under test, alone on the stream, between two events
+                ce = cudaStreamSynchronize(st);
+                if (ce == cudaSuccess) ce = cudaEventRecord(e0, st);
+                if (ce != cudaSuccess) { rc = cuda_fail(ce, "cudaEventRecord"); break; }
+                rc = issue(ctx, r, first, cnt, sms, stream, opcode);
+                if (rc != TUTTI_OK) break;
+                ce = cudaEventRecord(e1, st);
+                // the rest of the build runs too, so that every reserved IOCB completes
+                if (cnt < n) rc = issue(ctx, r, first + cnt, n - cnt, sms, stream, opcode);
+                if (ce == cudaSuccess) ce = cudaEventSynchronize(e1);
+                float ms = 0.f;
+                if (ce == cudaSuccess) ce = cudaEventElapsedTime(&ms, e0, e1);
+                if (ce != cudaSuccess) { rc = cuda_fail(ce, "cudaEventElapsedTime"); break; }
+                int32_t err = 0;
+                int prc = tutti_ring_poll_range(r, first, n, nullptr, &err, nullptr, 5000000000ull);
+                if (rc == TUTTI_OK && prc != TUTTI_OK) rc = prc;
+                if (rc == TUTTI_OK && err != 0) rc = err;
+                if (rep == 0 || ms < best) best = ms;
+            }
+            if (rc == TUTTI_OK) {
+                rc = tutti_sched_set_io_time(sched, opcode, sms, cnt, best * 1e3f);
+                ++points;
+            }
+            if (cnt == used) break;
+        }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (n_points) *n_points = points;
     return rc;
 }
 

@@ -169,7 +169,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         if (e == cudaSuccess) e = launch_plan(r, g, b, st, nullptr);
         if (e == cudaSuccess)
             e = launch_emit(r, g, b, layer, 1, TUTTI_OP_READ, pool, nullptr, sbase, sbytes, 0, 1, 0,
-                            NA_MAX_ENTRIES, sms, st);
+                            NA_MAX_ENTRIES, 0, sms, st);
         if (e == cudaSuccess)
             e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, false,
                             PermGeom{geom->block_tokens, geom->n_kv_heads,

@@ -80,6 +80,7 @@ EXPORTS = [
     "tutti_filepool_lookup", "tutti_filepool_match_prefix", "tutti_filepool_pin",
     "tutti_filepool_remove", "tutti_filepool_stats", "tutti_build_sqes_layers",
     "tutti_stream_wait_iocb", "tutti_ring_last_launch_sms", "tutti_ring_poll_range",
+    "tutti_ring_set_iocb_bytes", "tutti_sched_profile",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -118,6 +119,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_ring_read_iocb": (C.c_int, [vp, u32, P(IocbInfo), vp, u32]),
         "tutti_ring_read_sgl": (C.c_int, [vp, u32, vp, u32, P(u32)]),
         "tutti_ring_stats": (C.c_int, [vp, P(u64), P(u64)]),
+        "tutti_ring_set_iocb_bytes": (C.c_int, [vp, u64]),
         "tutti_ring_last_launch_sms": (C.c_int, [vp, vp, u32, P(u32)]),
         "tutti_sm_partition_create": (C.c_int, [vp, u32, P(vp), P(vp), P(u32), P(u32)]),
         "tutti_sm_partition_destroy": (C.c_int, [vp]),
@@ -139,6 +141,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_sched_enqueue": (C.c_int, [vp, u32, u32, u32, u32]),
         "tutti_sched_next": (C.c_int, [vp, u32, u32, u32, u32, P(Launch), u32, P(u32)]),
         "tutti_sched_pending": (C.c_int, [vp, P(u32), P(u32)]),
+        "tutti_sched_profile": (C.c_int, [vp, vp, vp, P(Batch), u32, u32, P(u32), u32, u32, vp, P(u32)]),
         "tutti_filepool_create": (C.c_int, [u64, P(vp)]),
         "tutti_filepool_destroy": (C.c_int, [vp]),
         "tutti_filepool_insert": (C.c_int, [vp, u64, P(u32), P(C.c_int)]),
@@ -345,6 +348,11 @@ class Ring:
                                             C.byref(n)), "tutti_ring_read_sgl")
         return sgl[:min(n.value, max_entries)].copy()
 
+    def tutti_ring_set_iocb_bytes(self, nbytes: int, allow: Sequence[int] = ()) -> int:
+        """IOCBs of (nearly) equal work: cut by bytes instead of by context count (0 = off)."""
+        return _check(self.lib.tutti_ring_set_iocb_bytes(self.h, nbytes),
+                      "tutti_ring_set_iocb_bytes", allow)
+
     def tutti_ring_last_launch_sms(self) -> np.ndarray:
         """SM id of every CTA of the most recent copy launch (synchronises)."""
         out = np.zeros(4096, dtype=np.uint32)
@@ -412,6 +420,18 @@ class Scheduler:
         _check(self.lib.tutti_sched_io_time(self.h, opcode, sm_count, n_iocb, C.byref(us)),
                "tutti_sched_io_time")
         return us.value
+
+    def tutti_sched_profile(self, ring: "Ring", batch: Batch, layer: int, opcode: int,
+                            sm_counts: Sequence[int], reps: int = 3, stream=None) -> int:
+        """Time the I/O kernels against the IOCB count on every SM count and fill the table;
+        returns the number of table entries written."""
+        arr = (C.c_uint32 * len(sm_counts))(*sm_counts)
+        n = C.c_uint32()
+        _check(self.lib.tutti_sched_profile(ring.ctx.h, ring.h, self.h, C.byref(batch), layer,
+                                            opcode, arr, len(sm_counts), reps,
+                                            _stream_ptr(stream), C.byref(n)),
+               "tutti_sched_profile")
+        return n.value
 
     def tutti_sched_enqueue(self, opcode, layer, first_iocb, n_iocb, allow: Sequence[int] = ()):
         return _check(self.lib.tutti_sched_enqueue(self.h, opcode, layer, first_iocb, n_iocb),

@@ -68,12 +68,12 @@ class DeviceCase:
         self.ctx.close()
 
     # ---- oracle side -----------------------------------------------------
-    def oracle_descriptors(self, layer, opcode, capacity):
+    def oracle_descriptors(self, layer, opcode, capacity, entries_per_iocb=0):
         base = self.pool_dev[layer].data_ptr()
         if self.hnd:
             opcode |= oracle.OP_HND
         return oracle.build_descriptors(self.og, layer, opcode, self.obatch, base + self.k_off,
-                                        base + self.v_off, self.stride, capacity)
+                                        base + self.v_off, self.stride, capacity, entries_per_iocb)
 
     def oracle_restore(self, layer):
         pool = self.pool_host[layer].copy()

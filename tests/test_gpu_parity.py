@@ -376,3 +376,60 @@ def test_shared_prefix_batch_grid_and_capped(engine, sm_count, chunk):
         assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2-small", "shared-prefix-8-requests", "cfg4-small",
+                                  "shared-prefix-1-token-pages", "hnd-pool"])
+@pytest.mark.parametrize("per", [5, 64, 2048])
+def test_iocbs_cut_by_bytes(name, per):
+    """tutti_ring_set_iocb_bytes: IOCBs of equal work.  Contexts, entries and per-IOCB counts
+    equal the oracle's, every IOCB moves at most its budget, and the bytes land as always —
+    single-layer and multi-layer builds, both engines, capped and on all SMs."""
+    w = mk(name)
+    n_ent = 2 * len(w.block_ids)
+    per_layer = max(1, -(-n_ent // per))
+    depth = 1
+    while depth < 2 * per_layer * w.n_layers:
+        depth *= 2
+    cap = 64 if per <= 64 else 2048
+    dc = DeviceCase(w, depth=depth, capacity=cap, sgl_capacity=n_ent * (w.n_layers + 2))
+    try:
+        bb = int(dc.ctx.layout.block_bytes)
+        assert dc.ring.tutti_ring_set_iocb_bytes(4096 * bb, allow=(T.EINVAL,)) == T.EINVAL
+        assert dc.ring.tutti_ring_set_iocb_bytes(bb - 16, allow=(T.EINVAL,)) == T.EINVAL
+        dc.ring.tutti_ring_set_iocb_bytes(per * bb)
+        for engine, sm_count in ((T.ENGINE_BULK, 0), (T.ENGINE_LDST, 8)):
+            dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
+            for l in range(w.n_layers):
+                dc.pool_dev[l].copy_(torch.from_numpy(dc.pool_host[l]))
+            rc, first, n = dc.ring.tutti_build_sqes_layers(dc.batch, 0, w.n_layers, T.OP_READ)
+            assert n == per_layer
+            for layer in range(w.n_layers):
+                sq, sg, num, infos = dc.read_build(first + layer * n, n)
+                orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, cap, per)
+                assert orc == 0
+                assert same_records(sq, osq) and same_records(sg, osg)
+                assert list(num[:len(onum)]) == list(onum) and not num[len(onum):].any()
+                assert all(i.status == 0 and i.bytes <= per * bb + 64 * bb for i in infos)
+                assert sum(i.bytes for i in infos) == int(osg["len"].astype(np.uint64).sum())
+            # issue the IOCBs of every layer in two launches, out of order
+            half = (n * w.n_layers) // 2
+            if half:
+                dc.ring.tutti_kv_restore_layer(first + half, n * w.n_layers - half, sm_count)
+                dc.ring.tutti_kv_restore_layer(first, half, sm_count)
+            else:
+                dc.ring.tutti_kv_restore_layer(first, n * w.n_layers, sm_count)
+            rc, nbytes, err, done = dc.ring.tutti_ring_poll_range(first, n * w.n_layers, 5_000_000_000)
+            assert (rc, err, done) == (T.OK, 0, n * w.n_layers)
+            for layer in range(w.n_layers):
+                assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        # back to IOCBs of a fixed number of contexts
+        dc.ring.tutti_ring_set_iocb_bytes(0)
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        sq, sg, num, infos = dc.read_build(first, n)
+        orc, osq, osg, onum = dc.oracle_descriptors(0, oracle.OP_READ, cap)
+        assert same_records(sq, osq) and n == max(1, -(-2 * len(w.obj_slot) // cap))
+        dc.ring.tutti_kv_restore_layer(first, n)
+        dc.poll_all(first, n)
+    finally:
+        dc.close()

@@ -431,6 +431,91 @@ def test_descriptors_of_requests_with_a_shared_prefix(case, capacity):
     assert not np.array_equal(pool_a, hc.make_pool_layer(w, lo, layer))
 
 
+def test_iocbs_cut_by_entries_hand_worked():
+    """IOCBs of equal work: boundaries every `per` scatter-gather entries, moved back so that a
+    repeat stays with the bytes it repeats; a context crossing a boundary is cut in two."""
+    g = oracle.geom(2, 8, 128, 2, 16, 256, 1, oracle.LAYER_MAJOR, 8)
+    lo = oracle.obj_layout(g)
+    bb = int(lo.block_bytes)
+    # one request, 512 tokens in the consecutive slots 3 and 4: one context of 64 entries
+    batch = ([512], [0, 2], [3, 4], [0, 32], list(range(32)))
+    rc, sqes, sgl, num = oracle.build_descriptors(g, 1, 0, batch, 0, 1 << 30, bb, 2048, 24)
+    assert rc == 0 and len(sgl) == 64
+    base = int(lo.stride_layer) + 3 * int(lo.obj_bytes)
+    assert [(int(s["src_off"]) - base, int(s["len"]), int(s["sgl_first"]), int(s["sgl_count"]))
+            for s in sqes] == [(0, 24 * bb, 0, 24), (24 * bb, 24 * bb, 24, 24), (48 * bb, 16 * bb, 48, 16)]
+    assert list(num) == [1, 1, 1]
+    # a budget that covers everything: one IOCB, the context as it is
+    rc, sq1, sg1, num1 = oracle.build_descriptors(g, 1, 0, batch, 0, 1 << 30, bb, 2048, 1000)
+    rc, sq0, sg0, num0 = oracle.build_descriptors(g, 1, 0, batch, 0, 1 << 30, bb, 2048)
+    assert sq1.tobytes() == sq0.tobytes() and sg1.tobytes() == sg0.tobytes() and list(num1) == [1]
+    # two requests sharing slot 5: entries go (block j of request 0, its repeat for request 1);
+    # with 5 entries per IOCB the odd boundaries 5, 15, ... fall on repeats and move back by one
+    batch = ([256, 256], [0, 1, 2], [5, 5], [0, 16, 32], list(range(32)))
+    rc, sqes, sgl, num = oracle.build_descriptors(g, 0, 0, batch, 0, 1 << 30, bb, 2048, 5)
+    assert rc == 0 and len(sgl) == 64
+    firsts = [int(s["sgl_first"]) for s in sqes]
+    assert firsts == [0, 4, 10, 14, 20, 24, 30, 34, 40, 44, 50, 54, 60]
+    assert list(num) == [1] * 13
+    assert [int(s["sgl_count"]) for s in sqes] == [4, 6, 4, 6, 4, 6, 4, 6, 4, 6, 4, 6, 4]
+    # the bytes are named once: 2, 3, 2, 3, ... source blocks per piece, back to back
+    assert [int(s["len"]) // bb for s in sqes] == [2, 3] * 6 + [2]
+    off5 = 5 * int(lo.obj_bytes)
+    assert [int(s["src_off"]) - off5 for s in sqes] == [bb * x for x in (0, 2, 5, 7, 10, 12, 15, 17, 20, 22, 25, 27, 30)]
+
+
+@pytest.mark.parametrize("case", [CASES[0], CASES[2], CASES[3]] + SHARED,
+                         ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
+@pytest.mark.parametrize("per", [7, 64, 1000])
+def test_iocbs_cut_by_entries_invariants(case, per):
+    w, g, lo = _mk(case)
+    nbytes, k_off, v_off, stride = hc.pool_geometry(w, lo)
+    base = 0x7F0000000000
+    layer = w.n_layers - 1
+    batch = hc.batch_of(w)
+    flag = oracle.OP_HND if w.pool_hnd else 0
+    rowb = w.head_dim * w.elem_bytes
+    bb = int(lo.block_bytes)
+    rc, sq0, sg0, num0 = oracle.build_descriptors(g, layer, oracle.OP_READ | flag, batch,
+                                                  base + k_off, base + v_off, stride, 1 << 20)
+    rc, sqes, sgl, num = oracle.build_descriptors(g, layer, oracle.OP_READ | flag, batch,
+                                                  base + k_off, base + v_off, stride, 1 << 20, per)
+    assert rc == 0
+    assert sgl.tobytes() == sg0.tobytes()                       # the entries do not change
+    ne = len(sgl)
+    assert len(num) == max(1, -(-ne // per)) and int(num.sum()) == len(sqes)
+    dup = (sgl["id"] & oracle.SGL_DUP) != 0
+    # the contexts, IOCB by IOCB, partition the entries in order
+    assert int(sqes["sgl_first"][0]) == 0
+    ends = sqes["sgl_first"].astype(np.int64) + sqes["sgl_count"].astype(np.int64)
+    assert np.array_equal(ends[:-1], sqes["sgl_first"][1:]) and int(ends[-1]) == ne
+    at = 0
+    for k, n in enumerate(num):
+        first = int(sqes["sgl_first"][at]) if n else None
+        last = int(ends[at + n - 1]) if n else None
+        if n:
+            # an IOCB starts at its boundary moved back over repeats, and holds at most `per`
+            # entries more than that
+            want = min(k * per, ne)
+            while 0 < want < ne and dup[want]:
+                want -= 1
+            assert first == want and last - first <= per + (k * per - want)
+            assert not dup[first]
+        at += n
+    for s_ in sqes:
+        e0, e1 = int(s_["sgl_first"]), int(s_["sgl_first"]) + int(s_["sgl_count"])
+        assert not dup[e0] and int((~dup[e0:e1]).sum()) * bb == int(s_["len"])
+    assert int(sqes["len"].sum()) == int(sq0["len"].sum())       # the same bytes are named
+    # executing the cut contexts is the plain restore
+    store = hc.make_store(w, lo)
+    pool_a = hc.make_pool_layer(w, lo, layer)
+    pool_b = pool_a.copy()
+    assert oracle.restore_layer(g, layer, batch, store, pool_a, k_off, v_off, stride,
+                                w.n_pool_blocks, w.pool_hnd) == 0
+    assert oracle.exec_descriptors(sqes, sgl, store, pool_b, base, w.n_kv_heads, rowb) == 0
+    assert np.array_equal(pool_a, pool_b)
+
+
 def test_config1_closed_form_counts():
     """Config 1: 16 items, 256 SGL entries; consecutive slots give one 8 MiB context,
     pairwise non-adjacent slots give eight 1 MiB contexts (K and V halves always merge)."""

@@ -153,7 +153,7 @@ def measured_peak():
 # entries of 32 KiB; traffic is proportional to the payload because every entry is an
 # independent copy).  A constant of the kernel version it was captured on: it has to be
 # re-captured on that small case whenever copy_bulk_kernel changes.
-NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore_copy": 1.957, "save_copy": 1.953}
+NCU_DRAM_BYTES_PER_PAYLOAD_BYTE = {"restore_copy": 1.955, "save_copy": 1.952}
 
 
 def ncu_traffic(kernel: str):
@@ -315,8 +315,12 @@ class Replica:
                         ba = torch.cuda.Event(enable_timing=True)
                         bb_ = torch.cuda.Event(enable_timing=True)
                         ba.record(sb)
+                    h0 = time.perf_counter()
                     rc, first, per = self.ring.tutti_build_sqes_layers(self.batch, l0, g, op, stream=sb,
                                                                        allow=(T.EAGAIN,))
+                    if events is not None:
+                        events["host_s"]["build"] += time.perf_counter() - h0
+                        events["host_s"]["n_build"] += 1
                     if rc == T.EAGAIN:
                         # the ring is full: consume the completions of what was issued, retry
                         polled += self.poll_list(issued)
@@ -335,11 +339,14 @@ class Replica:
                         a = torch.cuda.Event(enable_timing=True)
                         b = torch.cuda.Event(enable_timing=True)
                         a.record(s)
+                    h0 = time.perf_counter()
                     if op == T.OP_READ:
                         self.ring.tutti_kv_restore_layer(first, n, sm_count, stream=s)
                     else:
                         self.ring.tutti_kv_save_layer(first, n, sm_count, stream=s)
                     if events is not None:
+                        events["host_s"]["issue"] += time.perf_counter() - h0
+                        events["host_s"]["n_issue"] += 1
                         b.record(s)
                         events["copy"][op].append((a, b, min(G, self.w.n_layers - l0)))
                     issued.append((first, n))
@@ -527,7 +534,8 @@ def run_ours(args):
     k0, _ = rep.ring.tutti_ring_stats()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    events = {"pass": [], "build": [], "copy": {T.OP_READ: [], T.OP_WRITE: []}}
+    events = {"pass": [], "build": [], "copy": {T.OP_READ: [], T.OP_WRITE: []},
+              "host_s": {"build": 0.0, "n_build": 0, "issue": 0.0, "n_issue": 0}}
     barrier(world)
     torch.cuda.synchronize()
     e0 = torch.cuda.Event(enable_timing=True)
@@ -596,6 +604,14 @@ def run_ours(args):
             "blocks_per_s": restore["blocks_per_s"],
             "restore": restore, "save": save,
             "build_ms_per_layer": round(build_ms, 4),
+            # host side of the submission path: the ring indices and the SGL range of a build
+            # are reserved on the CPU (O(1) per call), the rest of the call is kernel launches
+            "host_us_per_build_call": round(events["host_s"]["build"] * 1e6 /
+                                            max(1, events["host_s"]["n_build"]), 1),
+            "host_us_per_issue_call": round(events["host_s"]["issue"] * 1e6 /
+                                            max(1, events["host_s"]["n_issue"]), 1),
+            "host_calls_per_step": (events["host_s"]["n_build"] + events["host_s"]["n_issue"]) //
+            max(1, args.steps),
             "gpu_launches": int(k1 - k0),
             "spot_check": bool(verified),
             "clocks": clocks,

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 
 def _args(**kw):
     d = dict(config=2, scale=1.0, layers=0, engine=0, resident_layers=3, ioctx_per_iocb=2048,
-             ctas_per_sm=0, bulk_warps=0, bulk_stages=0, claim=0, layers_per_launch=4)
+             ctas_per_sm=0, bulk_warps=0, bulk_stages=0, claim=0, layers_per_launch=0)
     d.update(kw)
     return argparse.Namespace(**d)
 
@@ -68,6 +68,42 @@ def test_config2_full_size(engine):
         assert np.array_equal(got_store, want_store[0])
         cov = want_store[0] != 0
         assert np.array_equal(got_store[cov], orig.cpu().numpy()[cov])     # round trip
+    finally:
+        rep.close()
+
+
+def test_config2_full_size_every_layer_resident():
+    """The bench's own residency: all 32 pool layers and the whole store in HBM, one build
+    launch and one copy launch for the whole pass.  The oracle names, token by token, the
+    store bytes and pool bytes that must be equal — sampled from every layer — and two
+    early layers are compared whole."""
+    rep = bench.Replica(_args(resident_layers=0), 0)
+    try:
+        w = rep.w
+        if rep.R < w.n_layers:
+            pytest.skip("not enough free HBM for 32 resident pool layers")
+        assert rep.layers_per_launch == 32
+        whole = (3, 17)
+        before = {l: rep.pool[l].clone() for l in whole}
+        assert rep.step(directions=(T.OP_READ,)) == 32 << 30
+        torch.cuda.synchronize()
+        assert verify_replica_samples(rep, 4096)           # layers drawn uniformly from all 32
+        og = oracle.geom(1, w.n_kv_heads, w.head_dim, w.elem_bytes, w.block_tokens, w.obj_tokens,
+                         w.n_devices, w.layout, w.n_slots)
+        ob = (w.hit_tokens, w.obj_start, w.obj_slot, w.blk_start, w.block_ids)
+        lb = int(rep.lo.stride_layer)
+        for l in whole:
+            store_l = [s[l * lb:(l + 1) * lb].cpu().numpy() for s in rep.store]
+            want = before[l].cpu().numpy()
+            assert oracle.restore_layer(og, 0, ob, store_l, want, 0, rep.v_off, rep.block_bytes,
+                                        w.n_pool_blocks) == 0
+            assert np.array_equal(rep.pool[l].cpu().numpy(), want)
+        # and the save of the whole pass puts every sampled token back where the oracle says
+        for s_ in rep.store:
+            s_.zero_()
+        assert rep.step(directions=(T.OP_WRITE,)) == 32 << 30
+        torch.cuda.synchronize()
+        assert verify_replica_samples(rep, 4096)
     finally:
         rep.close()
 

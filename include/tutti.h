@@ -404,7 +404,7 @@ int tutti_sm_partition_destroy(tutti_ctx_t *ctx);
  * engine has handed the whole HBM budget to its own pools, or inside a section where
  * allocator calls are forbidden.  They cannot create a ring, so this call keeps what
  * a ring would hold — one IOCB with its contexts, SGL entries and plan arrays — in a
- * fixed device array inside the library (about 1.9 MiB, held by every GPU that loads
+ * fixed device array inside the library (about 2 MiB, held by every GPU that loads
  * the library until the process exits) and runs the same kernels on it.
  *   geom, batch      host pointers; the batch arrays are device pointers, as for
  *                    tutti_build_sqes.  Limits: 2 * n_obj <= 4096 and

@@ -683,7 +683,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     // few dependent round trips, so an agent should not have to open many for its share of the
     // work, and the agents should not all queue up at the first one.  With the first IOCB's
     // size as the estimate of all of them, a claim grows to about half an agent's share of the
-    // launch (never beyond the option's value when one IOCB alone can feed every agent), and
+    // launch (the option's value stays when one IOCB alone feeds every agent several times), and
     // agent a starts at the IOCB that this claim size assigns to it, walking on cyclically.
     if (p.n_iocb > 1) {
         uint32_t start = 0, cl = claim;
@@ -693,7 +693,7 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
                 h0->total_entries != 0 && h0->status == 0) {
                 const uint32_t u = claim_units(h0, p.perm, CB, tm.valid != 0);
                 const uint32_t n_agents = gridDim.x * n_warps;
-                if (u != 0xffffffffu && u / claim < n_agents) {
+                if (u != 0xffffffffu && u / claim < 8u * n_agents) {
                     const unsigned long long share =
                         ((unsigned long long)u * p.n_iocb + n_agents - 1) / n_agents;
                     const unsigned long long half = (share + 1) / 2;

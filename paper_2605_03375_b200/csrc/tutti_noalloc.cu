@@ -39,7 +39,7 @@ constexpr size_t OFF_PLAN_KEY = OFF_PLAN_K + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_IDX = OFF_PLAN_KEY + 8 * NA_POW2_ITEMS;
 constexpr size_t OFF_SGL = OFF_PLAN_IDX + 4 * NA_POW2_ITEMS;
 constexpr size_t OFF_OBJ = OFF_SGL + sizeof(tutti_sgl_t) * NA_MAX_ENTRIES;
-constexpr size_t SCRATCH_BYTES = OFF_OBJ + 8 * (size_t)NA_MAX_ENTRIES;    // about 1.9 MiB
+constexpr size_t SCRATCH_BYTES = OFF_OBJ + 8 * (size_t)NA_MAX_ENTRIES;    // about 2 MiB
 static_assert(OFF_SQES % 256 == 0 && OFF_SGL % 256 == 0 && OFF_OBJ % 256 == 0, "alignment");
 
 // The scratch itself.  In host code this name is only a stand-in for the symbol: its

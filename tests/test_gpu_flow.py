@@ -195,3 +195,51 @@ def test_stream_waits_for_one_layer_inside_a_multi_layer_launch():
     finally:
         torch.cuda.synchronize()
         dc.close()
+
+
+def test_library_profiling_pass_fills_the_io_table():
+    """tutti_sched_profile: the warm-up profiling of Section 3.3 / 3.4 done by the library.
+    With IOCBs cut by bytes the measured times grow with the IOCB count, the table has an
+    entry for 1, 2, 4, ... and all used IOCBs per SM count, and the transfers it ran were
+    real restores (the pool holds the oracle's bytes afterwards)."""
+    from tests.devcase import DeviceCase
+    w = wl.config(2, 0.25, n_layers=2)
+    n_ent = 2 * len(w.block_ids)
+    per = 64                                            # entries per IOCB
+    n_iocb = -(-n_ent // per)
+    depth = 1
+    while depth < 2 * n_iocb:
+        depth *= 2
+    dc = DeviceCase(w, depth=depth, capacity=64, sgl_capacity=4 * n_ent)
+    sched = T.Scheduler(w.n_layers, 32, 4096, 4096)
+    try:
+        bb = int(dc.ctx.layout.block_bytes)
+        dc.ring.tutti_ring_set_iocb_bytes(per * bb)
+        dc.batch.plan_epoch = 7
+        n_points = sched.tutti_sched_profile(dc.ring, dc.batch, 1, T.OP_READ, [0, 8], reps=2)
+        counts = []
+        c = 1
+        while c < n_iocb:
+            counts.append(c)
+            c *= 2
+        counts.append(n_iocb)
+        assert n_points == 2 * len(counts)
+        for sms in (0, 8):
+            times = [sched.tutti_sched_io_time(T.OP_READ, sms, c) for c in counts]
+            assert all(t > 0 for t in times)
+            assert times[-1] > times[0]                  # more IOCBs take longer
+        # fewer SMs are not faster for the whole layer
+        assert sched.tutti_sched_io_time(T.OP_READ, 8, n_iocb) >= \
+            0.8 * sched.tutti_sched_io_time(T.OP_READ, 0, n_iocb)
+        torch.cuda.synchronize()
+        assert np.array_equal(dc.pool_dev[1].cpu().numpy(), dc.oracle_restore(1))
+        # the ring is left empty: nothing reserved, nothing unpolled
+        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, 0, T.OP_READ)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        assert dc.ring.tutti_ring_poll_range(first, n, 5_000_000_000)[0] == T.OK
+        # the write direction is profiled the same way
+        assert sched.tutti_sched_profile(dc.ring, dc.batch, 1, T.OP_WRITE, [8], reps=1) == len(counts)
+        assert sched.tutti_sched_io_time(T.OP_WRITE, 8, n_iocb) > 0
+    finally:
+        sched.close()
+        dc.close()

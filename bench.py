@@ -243,11 +243,20 @@ class Replica:
         passes_in_flight = 2 if host_store else 1           # the duplex e2e leg polls one pass late
         while depth < 2 * passes_in_flight * w.n_layers * n_iocb_layer:
             depth *= 2
+        iocb_mib = getattr(args, "iocb_mib", 0)
+        if iocb_mib:
+            # IOCBs cut by bytes: a layer takes ceil(entries * block_bytes / bytes) of them
+            n_iocb_layer = max(1, -(-2 * len(w.block_ids) * self.block_bytes // (iocb_mib << 20)))
+            depth = 1
+            while depth < 2 * passes_in_flight * w.n_layers * n_iocb_layer:
+                depth *= 2
         if ring_depth:
             depth = ring_depth            # a small ring: builds meet TUTTI_EAGAIN and the ring wraps
         self.ring = T.Ring(self.ctx, depth, args.ioctx_per_iocb,
                            2 * len(w.block_ids) * (2 * passes_in_flight * w.n_layers + 1),
                            2 * len(w.obj_slot))
+        if iocb_mib:
+            self.ring.tutti_ring_set_iocb_bytes(iocb_mib << 20)
         self.n_iocb_layer = n_iocb_layer
         self.ring_depth = depth
         self.stream = torch.cuda.Stream(self.dev)
@@ -519,14 +528,24 @@ def workload_name(w):
             f"objects of {w.obj_tokens} tokens, pool {w.n_pool_blocks} blocks 60% occupied")
 
 
+_T0 = time.perf_counter()
+
+
+def phase(name):
+    """Progress note on stderr (the JSON line on stdout stays the only output there)."""
+    print(f"[bench +{time.perf_counter() - _T0:6.1f}s] {name}", file=sys.stderr, flush=True)
+
+
 def run_ours(args):
     import torch
+    phase("start")
     rank, local_rank, world = init_dist("nccl")
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
     from paper_2605_03375_b200 import tutti as T
     rep = Replica(args, local_rank)
     w = rep.w
     peak, peak_kind = measured_peak()
+    phase("workload resident")
 
     for _ in range(args.warmup):
         rep.step(sm_count=args.sm_count)
@@ -575,6 +594,7 @@ def run_ours(args):
     # descriptor build (plan once per step + emit), per layer, on the build stream
     build_ms = statistics.mean(a.elapsed_time(b) / g for a, b, g in events["build"])
     verified = rep.spot_check()
+    phase("main leg timed and checked")
 
     out = None
     if rank == 0:
@@ -634,6 +654,7 @@ def run_ours(args):
         e2e = run_e2e(args, local_rank, world)
         if rank == 0:
             out["e2e"] = e2e
+        phase("e2e leg done")
     # the other configurations, the scheduler demo and the CPU oracle: one GPU, rank 0 only
     if rank == 0 and world == 1:
         if not args.no_configs:
@@ -647,12 +668,14 @@ def run_ours(args):
         if not args.no_sched:
             out["sched"] = {"hbm": run_leg(leg_sched_demo, args, local_rank, False),
                             "pinned_host": run_leg(leg_sched_demo, args, local_rank, True)}
+        phase("config and scheduler legs done")
         if not args.no_cpu_baseline:
             a2 = argparse.Namespace(**vars(args))
             a2.resident_layers = 1
             rep = Replica(a2, local_rank, n_layers=min(4, w.n_layers))
             out["cpu_baseline"] = cpu_baseline(rep)
             rep.close()
+            phase("cpu baseline done")
     if rank == 0:
         print(json.dumps(out), flush=True)
     barrier(world)
@@ -678,6 +701,7 @@ def run_leg(fn, args, local_rank, *extra):
     torch.cuda.empty_cache()
     res["clocks"] = sampler.stop()
     res["leg_seconds"] = round(time.perf_counter() - t0, 1)
+    phase(f"{fn.__name__} done")
     return res
 
 
@@ -1307,6 +1331,16 @@ def run_reference(args):
     dt = time.perf_counter() - t0
     value = 2 * payload * args.steps / dt / 1e9
     sample = "each step = restore+save of 1 layer of the batch (oracle, single thread)"
+    # the block-granular form on every host core, beside it (a few steps)
+    cores = os.cpu_count() or 1
+    v_off = w.n_pool_blocks * bb
+    n_mt = max(3, min(args.steps, 10))
+    t1 = time.perf_counter()
+    for _ in range(n_mt):
+        for to_pool in (True, False):
+            assert oracle.move_layer_blocks_mt(og, 0, ob, store, pool, 0, v_off, bb,
+                                               w.n_pool_blocks, to_pool, cores) == 0
+    all_cores = 2 * payload * n_mt / (time.perf_counter() - t1) / 1e9
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": "GB/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
@@ -1314,7 +1348,10 @@ def run_reference(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": workload_name(w), "sample": sample},
         "cpu_baseline": {"value": round(value, 3), "unit": "GB/s", "cores": 1,
-                         "host_cores": os.cpu_count(), "kind": "oracle", "sample": sample},
+                         "host_cores": os.cpu_count(), "kind": "oracle", "sample": sample,
+                         "all_cores": {"value": round(all_cores, 3), "unit": "GB/s", "cores": cores,
+                                       "sample": f"{n_mt} such steps, one memcpy per block and K/V "
+                                                 f"half, blocks dealt out over {cores} threads"}},
         "e2e": {"value": round(value, 3), "unit": "GB/s", "h2d_bytes_per_step": 0,
                 "d2h_bytes_per_step": 0},
         "gpu_launches": 0}), flush=True)
@@ -1335,6 +1372,8 @@ def main():
     ap.add_argument("--sm-count", type=int, default=0,
                     help="run the copies as a capped launch of this many persistent CTAs")
     ap.add_argument("--ioctx-per-iocb", type=int, default=2048)
+    ap.add_argument("--iocb-mib", type=int, default=0,
+                    help="cut IOCBs by bytes (MiB per IOCB) instead of by context count")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--bulk-warps", type=int, default=0)
     ap.add_argument("--bulk-stages", type=int, default=0)

@@ -115,7 +115,10 @@ int main(void)
     CU(cudaMemset(d_store, 0, lo.dev_bytes));
     CHECK(tutti_build_sqes(ctx, ring, &batch, layer, TUTTI_OP_WRITE, stream, &first, &n));
     CHECK(tutti_kv_save_layer(ctx, ring, first, n, 0, stream));
-    for (uint32_t i = first; i < first + n; ++i) CHECK(tutti_ring_poll(ring, i, &cqe, 5000000000ull));
+    int32_t first_error = 0;
+    uint32_t n_done = 0;
+    CHECK(tutti_ring_poll_range(ring, first, n, &moved, &first_error, &n_done, 5000000000ull));
+    if (first_error != 0 || n_done != n) { fprintf(stderr, "save status %d\n", first_error); return 1; }
     uint8_t *h_back = (uint8_t *)malloc(lo.dev_bytes);
     CU(cudaMemcpy(h_back, d_store, lo.dev_bytes, cudaMemcpyDeviceToHost));
     for (uint32_t kv = 0; kv < 2; ++kv)

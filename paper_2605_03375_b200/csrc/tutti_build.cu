@@ -223,6 +223,9 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
     __shared__ int32_t s_status;
     __shared__ uint32_t s_nact;
 
+    // the emit kernel launched behind this one may become resident now (it waits for this
+    // kernel's completion before it reads the plan)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     unsigned long long *key = use_smem ? reinterpret_cast<unsigned long long *>(dyn_smem)
                                        : ring.plan_key;
     uint32_t *idx = use_smem ? reinterpret_cast<uint32_t *>(dyn_smem + (size_t)np * 8)
@@ -408,6 +411,11 @@ __device__ Cut cut_at(const RingDev &ring, const GeomDev &g, uint32_t n_items, u
 // arena range follow those of the layer before it.
 __global__ void __launch_bounds__(EMIT_THREADS)
 emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
+    // Everything earlier in the stream (the plan kernel, or whatever ran before this build)
+    // has completed once this returns; only then may the copy kernel launched behind this one
+    // become resident, where its agents wait for the READY words written at the end.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.pools) {
         const PoolLayerDev pl = p.pools[p.layer + blockIdx.y];
         p.k_base = pl.k_base;
@@ -700,8 +708,8 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
     if (n_layers > 1) cap = cap / (n_layers < 8 ? n_layers : 8) + 1;   // the layers share the SMs
     if (ctas > cap) ctas = cap;
     if (ctas == 0) ctas = 1;
-    emit_kernel<<<dim3(ctas, n_layers), EMIT_THREADS, 0, stream>>>(ring, geom, batch, p);
-    return cudaGetLastError();
+    return launch_dependent(emit_kernel, dim3(ctas, n_layers), dim3(EMIT_THREADS), 0, stream, ring,
+                            geom, batch, p);
 }
 
 }  // namespace tutti

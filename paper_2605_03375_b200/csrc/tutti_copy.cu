@@ -688,8 +688,10 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     if (p.n_iocb > 1) {
         uint32_t start = 0, cl = claim;
         if (lane == 0) {
+            // (the kernel may have become resident while the build is still writing: the
+            // first IOCB's publication is awaited like any other, bounded)
             IocbHdr *h0 = hdr_of(0);
-            if (ld_acquire_u32(&h0->state) == state_word(p.first_iocb, PHASE_READY) &&
+            if (wait_iocb_ready(p.ring, h0, p.first_iocb, p.wait_ns) == IOCB_RUN &&
                 h0->total_entries != 0 && h0->status == 0) {
                 const uint32_t u = claim_units(h0, p.perm, CB, tm.valid != 0);
                 const uint32_t n_agents = gridDim.x * n_warps;
@@ -987,6 +989,7 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     p.inject_timeout = opt.inject_timeout;
     p.smid_log = smid_log;
     uint32_t grid = 0;
+    cudaError_t err = cudaSuccess;
     // measured: small claims balance best when every SM takes part, larger ones amortise the
     // claim's round trip when few SMs carry everything
     p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : (sm_count ? 4 : 2);
@@ -1016,9 +1019,9 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
         if (sm_count && smem < 120u * 1024u) smem = 120u * 1024u;
         grid = sms;
         if (opcode == TUTTI_OP_READ)
-            copy_bulk_kernel<1><<<sms, warps * 32, smem, stream>>>(p, tm);
+            err = launch_dependent(copy_bulk_kernel<1>, dim3(sms), dim3(warps * 32), smem, stream, p, tm);
         else
-            copy_bulk_kernel<0><<<sms, warps * 32, smem, stream>>>(p, tm);
+            err = launch_dependent(copy_bulk_kernel<0>, dim3(sms), dim3(warps * 32), smem, stream, p, tm);
     } else {
         p.stages = 0;
         p.chunk_bytes = CHUNK_BYTES;
@@ -1030,13 +1033,13 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
         const size_t smem = sm_count ? LDST_PAD_SMEM : 0;
         grid = sm_count ? sm_count : sms * per_sm;
         if (opcode == TUTTI_OP_READ)
-            copy_ldst_kernel<1><<<grid, threads, smem, stream>>>(p);
+            err = launch_dependent(copy_ldst_kernel<1>, dim3(grid), dim3(threads), smem, stream, p);
         else
-            copy_ldst_kernel<0><<<grid, threads, smem, stream>>>(p);
+            err = launch_dependent(copy_ldst_kernel<0>, dim3(grid), dim3(threads), smem, stream, p);
     }
     if (launches) *launches = 1;
     if (grid_out) *grid_out = grid;
-    return cudaGetLastError();
+    return err;
 }
 
 }  // namespace tutti

@@ -133,6 +133,29 @@ struct CopyOptions {
     uint32_t inject_timeout; // test hook: the bulk engine's stage waits report "ran out"
 };
 
+// Programmatic dependent launch: a kernel launched with this attribute may become resident
+// while the kernel before it in the stream is still running.  Used for the emit kernel
+// (behind the plan kernel) and the copy kernels (behind the emit kernel): the dependent's
+// launch latency and start-up overlap the tail of its predecessor.  Correctness never rests
+// on it: the emit kernel executes griddepcontrol.wait before it touches anything (so everything
+// earlier in the stream has completed by then, for it and for whatever is launched behind
+// it), and the copy agents wait, bounded, on each IOCB's READY word with acquire semantics.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                    cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // kernels (tutti_build.cu / tutti_copy.cu)
 cudaError_t launch_plan(const RingDev &ring, const GeomDev &geom, const BatchDev &batch,
                         cudaStream_t stream, uint32_t *launches);

@@ -481,14 +481,17 @@ def cpu_baseline(rep, seconds_hint=10.0):
         raise RuntimeError("cpu_baseline expects the layer-major store of the bench workloads")
     cores = os.cpu_count() or 1
 
-    def host_layer(l):
+    # host copies of two layers, fetched once and used in turn (3.75 GiB each, far beyond any
+    # host cache; fetching a fresh copy for every timed layer would cost more than the timing)
+    host_layers = []
+    for l in range(min(2, w.n_layers)):
         store = [s[l * layer_bytes:(l + 1) * layer_bytes].cpu().numpy() for s in rep.store]
-        return store, rep.pool[l % rep.R].cpu().numpy()
+        host_layers.append((store, rep.pool[l % rep.R].cpu().numpy().copy()))
 
     def run(move, budget):
         done_bytes, t_total, layers = 0, 0.0, 0
         while t_total < budget:
-            store, pool = host_layer(layers % w.n_layers)
+            store, pool = host_layers[layers % len(host_layers)]
             t0 = time.perf_counter()
             rc1 = move(store, pool, True)
             rc2 = move(store, pool, False)

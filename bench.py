@@ -513,13 +513,14 @@ def cpu_baseline(rep, seconds_hint=10.0):
     bN, tN, nN = run(all_cores, seconds_hint * 0.6)
     return {"value": round(b1 / t1 / 1e9, 3), "unit": "GB/s", "cores": 1,
             "host_cores": cores, "kind": "oracle", "seconds": round(t1 + tN, 2),
-            "sample": f"restore+save of {n1} full layers of the same batch "
-                      f"({b1 / GIB:.1f} GiB payload), token-by-token loop, single thread",
+            "sample": f"restore+save of a full layer of the same batch, {n1} times over host copies "
+                      f"of {len(host_layers)} layers ({b1 / GIB:.1f} GiB payload), token-by-token "
+                      f"loop, single thread",
             "blocks_per_s": round(n1 * 2 * rep.blocks_per_layer / t1),
             "all_cores": {"value": round(bN / tN / 1e9, 3), "unit": "GB/s", "cores": cores,
                           "blocks_per_s": round(nN * 2 * rep.blocks_per_layer / tN),
-                          "sample": f"restore+save of {nN} full layers, one memcpy per block and "
-                                    f"K/V half, blocks dealt out over {cores} threads"}}
+                          "sample": f"restore+save of a full layer, {nN} times, one memcpy per "
+                                    f"block and K/V half, blocks dealt out over {cores} threads"}}
 
 
 # ----------------------------------------------------------------------------

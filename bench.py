@@ -268,7 +268,12 @@ class Replica:
         self.duplex_sms = getattr(args, "e2e_sms", 12)
         self.duplex_save_sms = getattr(args, "e2e_save_sms", 8) or self.duplex_sms
         self.unpolled = []          # duplex mode: IOCBs of the previous pass
-        self.two_streams = not getattr(args, "one_stream", False)
+        # descriptors on their own stream pay off when a pass is long (the build of the next
+        # direction runs beside the copy); for a short pass the event round trip between the
+        # two streams costs more than it hides, and one stream lets the copy kernel start
+        # behind the emit kernel as a dependent launch
+        self.two_streams = (not getattr(args, "one_stream", False) and
+                            self.payload_per_layer * w.n_layers >= 8 * GIB)
         G = getattr(args, "layers_per_launch", 0)
         if not G:
             # one build launch and one copy launch span the whole pass (measured on config 2:
@@ -668,6 +673,7 @@ def run_ours(args):
                 "cfg4": run_leg(leg_config4, args, local_rank),
                 "cfg5": run_leg(leg_config5, args, local_rank),
                 "shared_prefix": run_leg(leg_shared_prefix, args, local_rank),
+                "prefix_sweep": run_leg(leg_prefix_sweep, args, local_rank),
             }
         if not args.no_sched:
             out["sched"] = {"hbm": run_leg(leg_sched_demo, args, local_rank, False),
@@ -1258,22 +1264,20 @@ def leg_sched_demo(args, local_rank, sched_host):
     return out
 
 
-def run_length_sweep(args):
-    """Raw restore / save bandwidth against prefix length, model bypassed (the measurement of
-    the paper's Section 4.2.1, here against the HBM or pinned-host object store): one request,
-    Llama-3-8B-shaped KV, all layers, descriptor build included."""
+def sweep_rows(args, local_rank, token_list, host_store=False, n_layers=32):
+    """Restore / save of one request's prefix, all layers, for every prefix length asked for."""
     import torch
     from paper_2605_03375_b200 import tutti as T
-    from paper_2605_03375_b200 import workload as wl
-    rank, local_rank, world = init_dist("nccl")
+    peak, _ = measured_peak()
     rows = []
-    for tokens in (1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072):
+    for tokens in token_list:
         a2 = argparse.Namespace(**vars(args))
-        a2.config = 2
+        a2.config, a2.scale, a2.layers = 2, 1.0, 0
         a2.resident_layers = 4
-        a2.set = (args.set or []) + []
-        rep = Replica(a2, local_rank, host_store=args.sweep_host, n_layers=args.layers or 32,
-                      hit_tokens=[tokens])
+        a2.ioctx_per_iocb = 2048
+        a2.layers_per_launch = 0
+        a2.iocb_mib = 0
+        rep = Replica(a2, local_rank, host_store=host_store, n_layers=n_layers, hit_tokens=[tokens])
         res = {"prefix_tokens": tokens,
                "payload_mib_per_layer": round(rep.payload_per_layer / (1 << 20), 1)}
         for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
@@ -1288,13 +1292,34 @@ def run_length_sweep(args):
             e1.record(rep.stream)
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / reps
-            res[name + "_gbs"] = round(rep.w.n_layers * rep.payload_per_layer / (ms * 1e-3) / 1e9, 1)
+            gbs = rep.w.n_layers * rep.payload_per_layer / (ms * 1e-3) / 1e9
+            res[name + "_gbs"] = round(gbs, 1)
             res[name + "_us_per_layer"] = round(ms * 1e3 / rep.w.n_layers, 1)
+            if not host_store:
+                res[name + "_hbm_frac"] = round(2 * gbs / peak, 3)
         res["spot_check"] = bool(rep.spot_check(32))
         rows.append(res)
         rep.close()
         del rep
         torch.cuda.empty_cache()
+    return rows
+
+
+def leg_prefix_sweep(args, local_rank):
+    """Raw restore / save bandwidth against prefix length, model bypassed (the measurement of the
+    paper's Section 4.2.1, here against the HBM object store): one request, Llama-3-8B-shaped
+    KV, 32 layers, descriptor build and host polls included; every pass is one build launch and
+    one copy launch."""
+    return {"sweep": "1 request, 8 KV heads x 128 x bf16, block 16, 32 layers, hbm store; whole "
+                     "pass = 1 plan + 1 emit + 1 copy launch and one range poll",
+            "rows": sweep_rows(args, local_rank, (1024, 2048, 4096, 16384, 131072))}
+
+
+def run_length_sweep(args):
+    """The same sweep on its own, all eight lengths, against the HBM or the pinned-host store."""
+    rank, local_rank, world = init_dist("nccl")
+    rows = sweep_rows(args, local_rank, (1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072),
+                      host_store=args.sweep_host, n_layers=args.layers or 32)
     if rank == 0:
         print(json.dumps({"sweep": "raw restore/save bandwidth vs prefix length, 1 request, "
                           "8 KV heads x 128 x bf16, block 16, 32 layers",

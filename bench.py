@@ -1166,6 +1166,11 @@ def leg_sched_demo(args, local_rank, sched_host):
     poll(built)
     profile = {k: round(sched.tutti_sched_io_time(T.OP_READ, got_io, k), 1)
                for k in sorted({1, 2, 4, 8, used})}
+    # the write kernel is profiled the same way (Section 3.3 profiles both)
+    n_points += sched.tutti_sched_profile(rep.ring, rep.batch, 0, T.OP_WRITE, [got_io], reps=1,
+                                          stream=io_stream)
+    profile_w = {k: round(sched.tutti_sched_io_time(T.OP_WRITE, got_io, k), 1)
+                 for k in sorted({1, used})}
     # the table against launches it has not seen: IOCB counts between the profiled points
     est_err = {}
     for k in sorted({3, 5, max(1, used - 3)}):
@@ -1250,7 +1255,7 @@ def leg_sched_demo(args, local_rank, sched_host):
            "io_partition_sms": got_io, "compute_partition_sms": got_comp,
            "iocb_mib": args.sched_iocb_mib, "iocbs_per_layer_used": used,
            "profile": "tutti_sched_profile (library), %d table entries" % n_points,
-           "io_profile_us_by_iocbs": profile,
+           "io_profile_us_by_iocbs": profile, "io_profile_write_us_by_iocbs": profile_w,
            "estimate_vs_measured": est_err,
            "gemms_per_layer": gemms_per_layer, "layer_compute_ms": round(layer_ms, 3),
            "restore_ms_per_layer_on_partition": round(layer_restore_ms, 3),

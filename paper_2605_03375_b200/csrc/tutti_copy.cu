@@ -992,7 +992,10 @@ cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_ioc
     cudaError_t err = cudaSuccess;
     // measured: small claims balance best when every SM takes part, larger ones amortise the
     // claim's round trip when few SMs carry everything
-    p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : (sm_count ? 4 : 2);
+    // (a capped launch on a pinned-host store is bound by the link, not by balance: long claims
+    // keep a shared block and the entries repeating it in one agent's hands, so it crosses the
+    // link once)
+    p.claim_chunks = opt.claim_chunks ? opt.claim_chunks : (sm_count ? (host_store ? 16 : 4) : 2);
     uint32_t engine = opt.engine;
     // measured: bulk-async wins on HBM, also for head-major blocks when tensor maps exist
     if (engine == 0) engine = (host_store || (pool_hnd && !(maps && maps->valid))) ? 1 : 2;

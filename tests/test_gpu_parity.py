@@ -44,6 +44,9 @@ CASES = {
                                    shared_prefix_frac=0.5, pool_hnd=True, n_devices=2),
     "shared-prefix-one-block-objects": dict(index=2, scale=0.02, n_layers=2, obj_tokens=16,
                                             hit_tokens=[512, 512, 256], shared_prefix_frac=1.0),
+    # more sharers than one stage's 32 lanes: the copy engines feed them in several rounds
+    "shared-by-40-requests": dict(index=2, scale=0.02, n_layers=2, hit_tokens=[512] * 40,
+                                  shared_prefix_frac=1.0),
 }
 
 
@@ -351,12 +354,14 @@ def test_whole_pass_of_a_short_prefix_in_one_launch(engine, sm_count, tokens):
 @pytest.mark.parametrize("engine", [T.ENGINE_LDST, T.ENGINE_BULK])
 @pytest.mark.parametrize("sm_count", [0, 8])
 @pytest.mark.parametrize("chunk", [0, 8192])
-def test_shared_prefix_batch_grid_and_capped(engine, sm_count, chunk):
+@pytest.mark.parametrize("name", ["shared-prefix-8-requests", "shared-by-40-requests"])
+def test_shared_prefix_batch_grid_and_capped(engine, sm_count, chunk, name):
     """8 requests sharing 75 % of their prefix: the shared objects are named once in the
     descriptors and go to all eight requests' blocks, on all SMs and SM-capped, with stages
-    that hold a whole block and with stages that hold a piece of one."""
-    w = mk("shared-prefix-8-requests")
-    dc = DeviceCase(w, capacity=16)
+    that hold a whole block and with stages that hold a piece of one.  Claims of 1, 2 and 3
+    chunks cut the groups of repeats at every possible place."""
+    w = mk(name)
+    dc = DeviceCase(w, capacity=16, depth=32)
     try:
         dc.ctx.tutti_set_option(T.OPT_COPY_ENGINE, engine)
         if chunk:
@@ -373,7 +378,17 @@ def test_shared_prefix_batch_grid_and_capped(engine, sm_count, chunk):
         cqes = dc.poll_all(first, n)
         assert all(c[1] == 0 for c in cqes)
         assert sum(c[2] for c in cqes) == int(sg["len"].astype(np.uint64).sum())   # bytes landed
-        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), dc.oracle_restore(layer))
+        want = dc.oracle_restore(layer)
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
+        for claim in (1, 2, 3):
+            dc.ctx.tutti_set_option(T.OPT_CLAIM_CHUNKS, claim)
+            dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
+            rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+            dc.ring.tutti_kv_restore_layer(first, n, sm_count)
+            rc, nbytes, err, done = dc.ring.tutti_ring_poll_range(first, n, 5_000_000_000)
+            assert (rc, err, done) == (T.OK, 0, n)
+            assert nbytes == int(sg["len"].astype(np.uint64).sum())
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
     finally:
         dc.close()
 

@@ -585,6 +585,35 @@ def test_partial_last_object_and_duplicates():
     assert list(sgl["id"]) == [16, 17, 18, 19] + list(range(16)) + [16, 17, 18, 19] + list(range(16))
 
 
+def test_many_requests_on_one_object():
+    """40 requests on one object: one source with 40 destinations per block.  Sorted items:
+    K x 40, V x 40; K and V are byte-adjacent, so one context names the object once and lists
+    40 entries per block, all but the first of each block flagged as repeats."""
+    g = oracle.geom(1, 8, 128, 2, 16, 256, 1, oracle.LAYER_MAJOR, 8)
+    lo = oracle.obj_layout(g)
+    kvb, bb = int(lo.obj_kv_bytes), int(lo.block_bytes)
+    n = 40
+    batch = ([256] * n, list(range(n + 1)), [5] * n, [16 * r for r in range(n + 1)],
+             list(range(16 * n)))
+    rc, sqes, sgl, num = oracle.build_descriptors(g, 0, 0, batch, 0, 1 << 30, bb, 2048)
+    assert rc == 0 and len(sgl) == 2 * 16 * n
+    off5 = 5 * int(lo.obj_bytes)
+    assert [(int(s["src_off"]) - off5, int(s["len"]), int(s["sgl_count"])) for s in sqes] == [
+        (0, 2 * kvb, 2 * 16 * n)]
+    D = oracle.SGL_DUP
+    # block 0 of K: requests 0..39 side by side, only the first without the repeat flag
+    assert list(sgl["id"][:n]) == [0] + [(16 * r) | D for r in range(1, n)]
+    assert int(sgl["id"][n]) == 1 and int(sgl["id"][n + 1]) == 17 | D     # then block 1
+    store = [np.arange(int(lo.dev_bytes), dtype=np.uint64).astype(np.uint8)]
+    pool_a = np.zeros(2 * 16 * n * bb, dtype=np.uint8)
+    pool_b = pool_a.copy()
+    v_off = 16 * n * bb
+    assert oracle.restore_layer(g, 0, batch, store, pool_a, 0, v_off, bb, 16 * n) == 0
+    rc, sqes, sgl, num = oracle.build_descriptors(g, 0, 0, batch, 1 << 40, (1 << 40) + v_off, bb, 2048)
+    assert oracle.exec_descriptors(sqes, sgl, store, pool_b, 1 << 40) == 0
+    assert np.array_equal(pool_a, pool_b)
+
+
 def test_empty_and_invalid():
     g = oracle.geom(2, 8, 128, 2, 16, 256, 1, oracle.LAYER_MAJOR, 8)
     rc, sqes, sgl, num = oracle.build_descriptors(g, 0, 0, ([0], [0, 0], [], [0, 0], []), 0, 0,

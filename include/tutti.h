@@ -357,6 +357,41 @@ int tutti_ring_destroy(tutti_ring_t *ring);
  * bytes = 0 goes back to IOCBs of ioctx_per_iocb contexts. */
 int tutti_ring_set_iocb_bytes(tutti_ring_t *ring, uint64_t bytes);
 
+/*
+ * Staged transfers over the host link.  Kernels that read or write pinned host memory directly
+ * (TUTTI_STORE_HOST_PINNED, zero-copy) cross the link in the SMs' 128-byte transactions; the
+ * copy engines use larger ones and get ~8 % more one way and ~25 % more with both directions
+ * busy.  The staged path lets them carry the bytes: a layer's contexts (Section 3.2: file offset
+ * + length each) are copied as they are, one cudaMemcpyAsync per context, between the store and
+ * a staging buffer in HBM that holds them packed in context order, and the scatter / gather
+ * between that buffer and the paged pool stays with the kernels.  Host work per layer is
+ * O(contexts), never O(blocks).
+ *
+ *   tutti_stage_plan        once per batch (plan_epoch != 0): runs the plan on `stream` if the
+ *                           ring does not hold it, waits for it and keeps the batch's contexts
+ *                           on the host.  Host out: *n_ctx contexts, *bytes_per_layer the
+ *                           staging bytes a layer needs (the distinct object bytes of the
+ *                           batch).  Blocks the host: a per-request call, not a per-layer one.
+ *   tutti_stage_copy_layer  enqueues on `stream` the copies of layer `layer`: store -> staging
+ *                           for TUTTI_OP_READ, staging -> store for TUTTI_OP_WRITE.  `stage` is a
+ *                           device pointer to at least *bytes_per_layer bytes, 16-byte aligned,
+ *                           owned by the caller.  Works for HBM and pinned-host stores alike.
+ *   tutti_build_sqes_staged tutti_build_sqes for one layer with the object side of every entry
+ *                           pointing into `stage` (contexts still carry the store offsets).
+ *                           The IOCBs are then executed with tutti_kv_restore_layer (after the
+ *                           copies into `stage`) or tutti_kv_save_layer (before the copies out
+ *                           of it); ordering between copies and kernels is the caller's (stream
+ *                           order or events).
+ * TUTTI_EINVAL if the batch is not the one tutti_stage_plan saw, or `stage` is too small.
+ */
+int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch, void *stream,
+                     uint32_t *n_ctx, uint64_t *bytes_per_layer);
+int tutti_stage_copy_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t layer, uint32_t opcode,
+                           void *stage, uint64_t stage_bytes, void *stream);
+int tutti_build_sqes_staged(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch,
+                            uint32_t layer, uint32_t opcode, void *stage, uint64_t stage_bytes,
+                            void *stream, uint32_t *first_iocb, uint32_t *n_iocb);
+
 /* get_iocb(nums) for descriptors prepared by the CPU (the paper's own split,
  * Section 3.2: "CPU-prepared, GPU-executed"): reserve n IOCBs and n_sgl arena
  * entries without building anything. */

@@ -355,6 +355,19 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
             ring.plan_sqe[sq].len = end - ring.plan_sqe[sq].src_off;
         }
     }
+    __syncthreads();
+    // where every context sits in a staging buffer that holds the contexts' bytes packed in
+    // order: the blocks named by the contexts before it (exclusive prefix sum)
+    if (threadIdx.x == 0) { carry.a = 0; carry.b = 0; carry.m = 0; }
+    __syncthreads();
+    for (uint32_t base = 0; base < n_sqe; base += blockDim.x) {
+        const uint32_t q = base + threadIdx.x;
+        ScanVals v{0, 0, 0};
+        if (q < n_sqe) v.a = (uint32_t)(ring.plan_sqe[q].len / g.block_bytes);
+        const uint32_t mine = v.a;
+        const ScanVals sc = block_scan_incl(v, warp_tot, carry);
+        if (q < n_sqe) ring.plan_stage[q] = sc.a - mine;
+    }
     if (threadIdx.x == 0) {
         PlanCounts pc;
         pc.n_items = n_act;
@@ -374,6 +387,8 @@ struct EmitParams {
     uint64_t store_bytes[TUTTI_MAX_DEVICES];
     uint32_t first_iocb, n_iocb, sgl_base, sgl_reserved;
     uint32_t entries_per_iocb;   // 0: IOCBs of `capacity` contexts; else IOCBs cut by entries
+    uint64_t stage_base;         // != 0: the object side of every entry is this staging buffer,
+    uint64_t stage_bytes;        //       which holds the contexts' bytes packed in context order
     const PoolLayerDev *pools;   // per-layer pool table for launches that cover several layers
 };
 
@@ -551,8 +566,22 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
                 note_error(&hdr0->emit_status, TUTTI_EFAULT);
                 meta1 = 0;
                 n_blk = 0;                             // nothing is emitted for this item
-            } else {
+            } else if (p.stage_base == 0) {
                 meta1 = p.store_base[dev] + off;
+            } else {
+                // staged transfer: the item's bytes sit in the staging buffer at its context's
+                // place plus its distance from the context's first byte
+                const uint32_t sq = ring.plan_sqe_of[gs];
+                const unsigned long long at =
+                    (unsigned long long)ring.plan_stage[sq] * g.block_bytes +
+                    ((po & ((1ull << 56) - 1)) - ring.plan_sqe[sq].src_off);
+                if (at + (unsigned long long)n_blk * g.block_bytes > p.stage_bytes) {
+                    note_error(&hdr0->emit_status, TUTTI_EFAULT);
+                    meta1 = 0;
+                    n_blk = 0;
+                } else {
+                    meta1 = p.stage_base + at;
+                }
             }
         }
         // the group leader read the item; its lanes get it by shuffle
@@ -681,9 +710,12 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
                         const PoolLayerDev *pools, const uint64_t *store_base,
                         const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
                         uint32_t sgl_base, uint32_t sgl_reserved, uint32_t entries_per_iocb,
-                        int device_sms, cudaStream_t stream) {
+                        uint64_t stage_base, uint64_t stage_bytes, int device_sms,
+                        cudaStream_t stream) {
     EmitParams p;
     p.entries_per_iocb = entries_per_iocb;
+    p.stage_base = stage_base;
+    p.stage_bytes = stage_bytes;
     p.layer = layer;
     p.opcode = opcode;
     p.k_base = pool.k_base;

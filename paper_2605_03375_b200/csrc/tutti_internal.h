@@ -88,6 +88,8 @@ struct RingDev {
     uint32_t *plan_grp;       // [max_items]  index of the first item of the item's group (items
                               //              that name exactly the same bytes form a group)
     uint32_t *plan_k;         // [max_items]  at a group's first item: members of the group
+    uint32_t *plan_stage;     // [max_items]  per context: blocks named by the contexts before it
+                              //              (where it sits in a staging buffer packed in order)
     tutti_sqe_t *plan_sqe;    // [max_items]  contexts for layer 0, opcode unset
     unsigned long long *plan_key;  // [pow2(max_items)] sort keys when they do not fit in shared memory
     uint32_t *plan_idx;       // [pow2(max_items)] sort payload, same
@@ -164,7 +166,8 @@ cudaError_t launch_emit(const RingDev &ring, const GeomDev &geom, const BatchDev
                         const PoolLayerDev *pools, const uint64_t *store_base,
                         const uint64_t *store_bytes, uint32_t first_iocb, uint32_t n_iocb,
                         uint32_t sgl_base, uint32_t sgl_reserved, uint32_t entries_per_iocb,
-                        int device_sms, cudaStream_t stream);
+                        uint64_t stage_base, uint64_t stage_bytes, int device_sms,
+                        cudaStream_t stream);
 cudaError_t launch_copy(const RingDev &ring, uint32_t first_iocb, uint32_t n_iocb, uint32_t opcode,
                         uint32_t sm_count, int device_sms, const CopyOptions &opt, bool host_store,
                         bool pool_hnd, const PermGeom &perm, const StoreTensorMaps *maps,

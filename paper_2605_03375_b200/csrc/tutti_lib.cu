@@ -88,6 +88,14 @@ struct tutti_ring {
     std::vector<uint64_t> fill_optr;      // tutti_ring_fill_host scratch (sized at create)
     std::vector<uint8_t> fill_seen;
     uint32_t entries_per_iocb = 0;        // IOCBs cut by entries (0: by context count)
+    std::vector<uint8_t> staged;          // per slot: the IOCB's object side is a staging buffer
+    // staged transfers: the batch's contexts (layer 0) on the host, and where each sits in a
+    // staging buffer packed in context order
+    std::vector<tutti_sqe_t> stage_ctx;
+    std::vector<uint64_t> stage_off;
+    uint64_t stage_layer_bytes = 0;
+    bool stage_valid = false;
+    tutti_batch_t stage_batch{};
     uint32_t *smid_log = nullptr;         // device: SM of every CTA of the last copy launch
     uint32_t smid_cap = 0, last_grid = 0;
     uint32_t sgl_capacity;
@@ -351,6 +359,7 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
     r->have_cqe.assign(depth, 0);
     r->opcode_of.assign(depth, 0xff);
     r->issued.assign(depth, 0);
+    r->staged.assign(depth, 0);
     r->fill_optr.resize(sgl_capacity < (1u << 16) ? sgl_capacity : (1u << 16));
     r->fill_seen.resize(r->fill_optr.size());
     r->smid_cap = (uint32_t)ctx->device_sms * 8u;
@@ -373,6 +382,7 @@ int tutti_ring_create(tutti_ctx_t *ctx, uint32_t depth, uint32_t ioctx_per_iocb,
     A((void **)&d.plan_off, sizeof(uint64_t) * (size_t)max_items, false);
     A((void **)&d.plan_grp, sizeof(uint32_t) * (size_t)max_items, false);
     A((void **)&d.plan_k, sizeof(uint32_t) * (size_t)max_items, false);
+    A((void **)&d.plan_stage, sizeof(uint32_t) * (size_t)max_items, false);
     A((void **)&d.plan_sqe, sizeof(tutti_sqe_t) * (size_t)max_items, false);
     A((void **)&d.plan_key, sizeof(unsigned long long) * (size_t)np, false);
     A((void **)&d.plan_idx, sizeof(uint32_t) * (size_t)np, false);
@@ -434,7 +444,7 @@ static bool same_plan(const tutti_batch_t &a, const tutti_batch_t &b) {
 
 static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, uint32_t layer,
                         uint32_t n_layers, uint32_t opcode, void *stream, uint32_t *first_iocb,
-                        uint32_t *iocbs_per_layer) {
+                        uint32_t *iocbs_per_layer, uint64_t stage_base = 0, uint64_t stage_bytes = 0) {
     if (!ctx || !r || r->ctx != ctx || !batch || !first_iocb || !iocbs_per_layer) return TUTTI_EINVAL;
     r->host_calls++;
     if (n_layers == 0 || layer >= ctx->geom.n_layers || n_layers > ctx->geom.n_layers - layer ||
@@ -465,6 +475,7 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
         r->have_cqe[slot] = 0;
         r->opcode_of[slot] = (uint8_t)opcode;
         r->issued[slot] = 0;
+        r->staged[slot] = stage_base != 0;
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
@@ -495,7 +506,8 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
     const uint32_t op_flags = opcode | (ctx->pool_hnd ? TUTTI_OP_FLAG_HND : 0u);
     CK_OR_CANCEL(launch_emit(r->dev, ctx->gdev, b, layer, n_layers, op_flags, ctx->pool[layer],
                              n_layers > 1 ? ctx->d_pools : nullptr, sbase, sbytes, first, need_iocb,
-                             sgl_base, need_sgl, r->entries_per_iocb, ctx->device_sms, st));
+                             sgl_base, need_sgl, r->entries_per_iocb, stage_base, stage_bytes,
+                             ctx->device_sms, st));
 #undef CK_OR_CANCEL
     r->kernel_launches++;
     *first_iocb = first;
@@ -523,19 +535,28 @@ static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, 
     bool host_store = false;
     for (uint32_t d = 0; d < ctx->geom.n_devices; ++d)
         host_store |= ctx->store[d].kind == TUTTI_STORE_HOST_PINNED;
+    bool all_staged = true;
     for (uint32_t k = 0; k < n; ++k) {
         uint32_t idx = first + k;
         if (!r->host->is_live(idx)) return TUTTI_EINVAL;
         uint8_t op = r->opcode_of[idx & (r->dev.depth - 1)];
         if (op != 0xff && op != opcode) return TUTTI_EINVAL;
+        all_staged = all_staged && r->staged[idx & (r->dev.depth - 1)];
     }
+    bool any_staged = false;
+    for (uint32_t k = 0; k < n; ++k) any_staged = any_staged || r->staged[(first + k) & (r->dev.depth - 1)];
+    if (all_staged) host_store = false;      // the object side of these IOCBs is a buffer in HBM
+    // head-major blocks are transposed with tensor maps of the store regions, which a staging
+    // buffer is not part of: staged IOCBs take the vector path, and one launch is all of one kind
+    if (ctx->pool_hnd && any_staged && !all_staged) return TUTTI_EINVAL;
+    const StoreTensorMaps *maps = (ctx->pool_hnd && all_staged) ? nullptr : &ctx->maps;
     DeviceGuard guard(ctx->device);
     uint32_t launches = 0;
     PermGeom pg{ctx->geom.block_tokens, ctx->geom.n_kv_heads,
                 ctx->geom.head_dim * ctx->geom.elem_bytes, (uint32_t)ctx->layout.token_bytes};
     uint32_t grid = 0;
     CK(launch_copy(r->dev, first, n, opcode, sm_count, ctx->device_sms, ctx->opt, host_store,
-                   ctx->pool_hnd, pg, &ctx->maps, r->smid_log, (cudaStream_t)stream, &launches, &grid));
+                   ctx->pool_hnd, pg, maps, r->smid_log, (cudaStream_t)stream, &launches, &grid));
     r->kernel_launches += launches;
     r->last_grid = grid < r->smid_cap ? grid : r->smid_cap;
     for (uint32_t k = 0; k < n; ++k) r->issued[(first + k) & (r->dev.depth - 1)] = 1;
@@ -628,6 +649,84 @@ int tutti_ring_poll_range(tutti_ring_t *r, uint32_t first_iocb, uint32_t n_iocb,
     if (first_error) *first_error = err;
     if (n_done) *n_done = done;
     return rc;
+}
+
+int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, void *stream,
+                     uint32_t *n_ctx, uint64_t *bytes_per_layer) {
+    if (!ctx || !r || r->ctx != ctx || !batch || batch->plan_epoch == 0) return TUTTI_EINVAL;
+    r->host_calls++;
+    if (batch->n_req && (!batch->hit_tokens || !batch->obj_start || !batch->blk_start))
+        return TUTTI_EINVAL;
+    if ((batch->n_obj && !batch->obj_slot) || (batch->n_blk && !batch->block_ids)) return TUTTI_EINVAL;
+    if (batch->n_obj > r->dev.max_items / 2) return TUTTI_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    r->stage_valid = false;
+    if (!(r->plan_valid && same_plan(r->plan_batch, *batch))) {
+        BatchDev b{batch->n_req, batch->n_obj, batch->n_blk, batch->hit_tokens, batch->obj_start,
+                   batch->obj_slot, batch->blk_start, batch->block_ids};
+        uint32_t plan_launches = 0;
+        CK(launch_plan(r->dev, ctx->gdev, b, st, &plan_launches));
+        r->kernel_launches += plan_launches;
+        r->plan_batch = *batch;
+        r->plan_valid = true;
+    }
+    // once per batch: the plan's contexts come to the host (they do not depend on the layer)
+    CK(cudaStreamSynchronize(st));
+    PlanCounts pc;
+    CK(cudaMemcpy(&pc, r->dev.plan_counts, sizeof(pc), cudaMemcpyDeviceToHost));
+    if (pc.status != 0) return pc.status;
+    r->stage_ctx.resize(pc.n_sqe);
+    r->stage_off.resize(pc.n_sqe);
+    if (pc.n_sqe)
+        CK(cudaMemcpy(r->stage_ctx.data(), r->dev.plan_sqe, sizeof(tutti_sqe_t) * pc.n_sqe,
+                      cudaMemcpyDeviceToHost));
+    uint64_t at = 0;
+    for (uint32_t k = 0; k < pc.n_sqe; ++k) {
+        r->stage_off[k] = at;
+        at += r->stage_ctx[k].len;
+    }
+    r->stage_layer_bytes = at;
+    r->stage_batch = *batch;
+    r->stage_valid = true;
+    if (n_ctx) *n_ctx = pc.n_sqe;
+    if (bytes_per_layer) *bytes_per_layer = at;
+    return TUTTI_OK;
+}
+
+int tutti_stage_copy_layer(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t layer, uint32_t opcode,
+                           void *stage, uint64_t stage_bytes, void *stream) {
+    if (!ctx || !r || r->ctx != ctx || !stage || layer >= ctx->geom.n_layers ||
+        (opcode != TUTTI_OP_READ && opcode != TUTTI_OP_WRITE))
+        return TUTTI_EINVAL;
+    r->host_calls++;
+    if (!r->stage_valid) return TUTTI_EINVAL;
+    if (stage_bytes < r->stage_layer_bytes || ((uint64_t)stage & 15)) return TUTTI_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint64_t layer_off = (uint64_t)layer * ctx->layout.stride_layer;
+    for (size_t k = 0; k < r->stage_ctx.size(); ++k) {
+        const tutti_sqe_t &c = r->stage_ctx[k];
+        if (c.dev >= ctx->geom.n_devices || !ctx->store[c.dev].registered) return TUTTI_EINVAL;
+        if (c.src_off + layer_off + c.len > ctx->store[c.dev].bytes) return TUTTI_EFAULT;
+        char *in_store = reinterpret_cast<char *>(ctx->store[c.dev].base + c.src_off + layer_off);
+        char *in_stage = reinterpret_cast<char *>(stage) + r->stage_off[k];
+        if (opcode == TUTTI_OP_READ)
+            CK(cudaMemcpyAsync(in_stage, in_store, c.len, cudaMemcpyDefault, st));
+        else
+            CK(cudaMemcpyAsync(in_store, in_stage, c.len, cudaMemcpyDefault, st));
+    }
+    return TUTTI_OK;
+}
+
+int tutti_build_sqes_staged(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch,
+                            uint32_t layer, uint32_t opcode, void *stage, uint64_t stage_bytes,
+                            void *stream, uint32_t *first_iocb, uint32_t *n_iocb) {
+    if (!stage || ((uint64_t)stage & 15) || !r || !batch) return TUTTI_EINVAL;
+    if (!r->stage_valid || !same_plan(r->stage_batch, *batch)) return TUTTI_EINVAL;
+    if (stage_bytes < r->stage_layer_bytes) return TUTTI_EINVAL;
+    return build_layers(ctx, r, batch, layer, 1, opcode, stream, first_iocb, n_iocb, (uint64_t)stage,
+                        stage_bytes);
 }
 
 int tutti_sched_profile(tutti_ctx_t *ctx, tutti_ring_t *r, tutti_sched_t *sched,
@@ -743,6 +842,7 @@ int tutti_ring_reserve(tutti_ring_t *r, uint32_t n_iocb, uint32_t n_sgl, uint32_
         r->have_cqe[slot] = 0;
         r->opcode_of[slot] = 0xff;
         r->issued[slot] = 0;
+        r->staged[slot] = 0;
     }
     *first_iocb = first;
     return TUTTI_OK;

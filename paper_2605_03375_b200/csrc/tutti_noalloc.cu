@@ -35,7 +35,8 @@ constexpr size_t OFF_PLAN_SQE_OF = OFF_PLAN_CUM + 4 * (NA_MAX_ITEMS + 64);
 constexpr size_t OFF_PLAN_OFF = OFF_PLAN_SQE_OF + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_GRP = OFF_PLAN_OFF + 8 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_K = OFF_PLAN_GRP + 4 * NA_MAX_ITEMS;
-constexpr size_t OFF_PLAN_KEY = OFF_PLAN_K + 4 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_STAGE = OFF_PLAN_K + 4 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_KEY = OFF_PLAN_STAGE + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_IDX = OFF_PLAN_KEY + 8 * NA_POW2_ITEMS;
 constexpr size_t OFF_SGL = OFF_PLAN_IDX + 4 * NA_POW2_ITEMS;
 constexpr size_t OFF_OBJ = OFF_SGL + sizeof(tutti_sgl_t) * NA_MAX_ENTRIES;
@@ -141,6 +142,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         r.plan_off = reinterpret_cast<uint64_t *>(base + OFF_PLAN_OFF);
         r.plan_grp = reinterpret_cast<uint32_t *>(base + OFF_PLAN_GRP);
         r.plan_k = reinterpret_cast<uint32_t *>(base + OFF_PLAN_K);
+        r.plan_stage = reinterpret_cast<uint32_t *>(base + OFF_PLAN_STAGE);
         r.plan_key = reinterpret_cast<unsigned long long *>(base + OFF_PLAN_KEY);
         r.plan_idx = reinterpret_cast<uint32_t *>(base + OFF_PLAN_IDX);
         r.plan_counts = reinterpret_cast<PlanCounts *>(base + OFF_COUNTS);
@@ -169,7 +171,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         if (e == cudaSuccess) e = launch_plan(r, g, b, st, nullptr);
         if (e == cudaSuccess)
             e = launch_emit(r, g, b, layer, 1, TUTTI_OP_READ, pool, nullptr, sbase, sbytes, 0, 1, 0,
-                            NA_MAX_ENTRIES, 0, sms, st);
+                            NA_MAX_ENTRIES, 0, 0, 0, sms, st);
         if (e == cudaSuccess)
             e = launch_copy(r, 0, 1, TUTTI_OP_READ, 0, sms, opt, false, false,
                             PermGeom{geom->block_tokens, geom->n_kv_heads,

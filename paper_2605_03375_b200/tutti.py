@@ -81,6 +81,7 @@ EXPORTS = [
     "tutti_filepool_remove", "tutti_filepool_stats", "tutti_build_sqes_layers",
     "tutti_stream_wait_iocb", "tutti_ring_last_launch_sms", "tutti_ring_poll_range",
     "tutti_ring_set_iocb_bytes", "tutti_sched_profile",
+    "tutti_stage_plan", "tutti_stage_copy_layer", "tutti_build_sqes_staged",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -120,6 +121,9 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_ring_read_sgl": (C.c_int, [vp, u32, vp, u32, P(u32)]),
         "tutti_ring_stats": (C.c_int, [vp, P(u64), P(u64)]),
         "tutti_ring_set_iocb_bytes": (C.c_int, [vp, u64]),
+        "tutti_stage_plan": (C.c_int, [vp, vp, P(Batch), vp, P(u32), P(u64)]),
+        "tutti_stage_copy_layer": (C.c_int, [vp, vp, u32, u32, vp, u64, vp]),
+        "tutti_build_sqes_staged": (C.c_int, [vp, vp, P(Batch), u32, u32, vp, u64, vp, P(u32), P(u32)]),
         "tutti_ring_last_launch_sms": (C.c_int, [vp, vp, u32, P(u32)]),
         "tutti_sm_partition_create": (C.c_int, [vp, u32, P(vp), P(vp), P(u32), P(u32)]),
         "tutti_sm_partition_destroy": (C.c_int, [vp]),
@@ -347,6 +351,30 @@ class Ring:
         _check(self.lib.tutti_ring_read_sgl(self.h, iocb_idx, sgl.ctypes.data, max_entries,
                                             C.byref(n)), "tutti_ring_read_sgl")
         return sgl[:min(n.value, max_entries)].copy()
+
+    def tutti_stage_plan(self, batch: Batch, stream=None, allow: Sequence[int] = ()):
+        """(rc, n_ctx, bytes_per_layer): the batch's contexts are fetched to the host, once."""
+        n, b = C.c_uint32(), C.c_uint64()
+        rc = _check(self.lib.tutti_stage_plan(self.ctx.h, self.h, C.byref(batch),
+                                              _stream_ptr(stream), C.byref(n), C.byref(b)),
+                    "tutti_stage_plan", allow)
+        return rc, n.value, b.value
+
+    def tutti_stage_copy_layer(self, layer: int, opcode: int, stage: int, stage_bytes: int,
+                               stream=None, allow: Sequence[int] = ()) -> int:
+        """Copy-engine leg of a staged transfer: store -> stage (READ) or stage -> store (WRITE)."""
+        return _check(self.lib.tutti_stage_copy_layer(self.ctx.h, self.h, layer, opcode, stage,
+                                                      stage_bytes, _stream_ptr(stream)),
+                      "tutti_stage_copy_layer", allow)
+
+    def tutti_build_sqes_staged(self, batch: Batch, layer: int, opcode: int, stage: int,
+                                stage_bytes: int, stream=None, allow: Sequence[int] = ()):
+        first, n = C.c_uint32(), C.c_uint32()
+        rc = _check(self.lib.tutti_build_sqes_staged(self.ctx.h, self.h, C.byref(batch), layer,
+                                                     opcode, stage, stage_bytes,
+                                                     _stream_ptr(stream), C.byref(first), C.byref(n)),
+                    "tutti_build_sqes_staged", allow)
+        return rc, first.value, n.value
 
     def tutti_ring_set_iocb_bytes(self, nbytes: int, allow: Sequence[int] = ()) -> int:
         """IOCBs of (nearly) equal work: cut by bytes instead of by context count (0 = off)."""

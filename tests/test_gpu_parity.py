@@ -448,3 +448,58 @@ def test_iocbs_cut_by_bytes(name, per):
         dc.poll_all(first, n)
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2-small", "shared-prefix-8-requests", "cfg4-small",
+                                  "cfg2-2dev-interleaved", "hnd-pool"])
+@pytest.mark.parametrize("host_store", [False, True])
+def test_staged_transfer_matches_oracle(name, host_store):
+    """Staged restore and save: the copy engines move every context between the store and a
+    staging buffer in HBM (one copy per context), the kernels scatter / gather between that
+    buffer and the pool.  The pool after a staged restore and the store after a staged save
+    are the oracle's, byte for byte; descriptors are those of an ordinary build."""
+    w = mk(name)
+    dc = DeviceCase(w, host_store=host_store)
+    try:
+        dc.batch.plan_epoch = 11
+        rc, n_ctx, need = dc.ring.tutti_stage_plan(dc.batch)
+        layer = w.n_layers - 1
+        orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 2048)
+        assert n_ctx == len(osq) and need == int(osq["len"].sum())
+        stage = torch.zeros(need + 64, dtype=torch.uint8, device=dc.dev)
+        # a stage that is too small is refused before anything is enqueued
+        assert dc.ring.tutti_stage_copy_layer(layer, T.OP_READ, stage.data_ptr(), need - 16,
+                                              allow=(T.EINVAL,)) == T.EINVAL
+        # restore: copies in, then the scatter kernel
+        dc.ring.tutti_stage_copy_layer(layer, T.OP_READ, stage.data_ptr(), need)
+        rc, first, n = dc.ring.tutti_build_sqes_staged(dc.batch, layer, T.OP_READ, stage.data_ptr(), need)
+        sq, sg, num, infos = dc.read_build(first, n)
+        assert same_records(sq, osq) and same_records(sg, osg)
+        dc.ring.tutti_kv_restore_layer(first, n)
+        cqes = dc.poll_all(first, n)
+        assert all(c[1] == 0 for c in cqes)
+        assert sum(c[2] for c in cqes) == int(osg["len"].astype(np.uint64).sum())
+        want = dc.oracle_restore(layer)
+        assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
+        # save: the gather kernel, then copies out, into a zeroed store
+        for t in dc.store_dev:
+            t.zero_()
+        stage.zero_()
+        rc, first, n = dc.ring.tutti_build_sqes_staged(dc.batch, layer, T.OP_WRITE, stage.data_ptr(), need)
+        dc.ring.tutti_kv_save_layer(first, n)
+        dc.ring.tutti_stage_copy_layer(layer, T.OP_WRITE, stage.data_ptr(), need)
+        assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        torch.cuda.synchronize()
+        st_want = [np.zeros_like(s) for s in dc.store_host]
+        dc.oracle_save(layer, want, st_want)
+        for t, s in zip(dc.store_dev, st_want):
+            assert np.array_equal(t.cpu().numpy(), s)
+        # another batch on the ring invalidates nothing silently: a build for a batch the stage
+        # plan has not seen is refused
+        other = T.Batch(dc.batch.n_req, dc.batch.n_obj, dc.batch.n_blk, 12, dc.batch.hit_tokens,
+                        dc.batch.obj_start, dc.batch.obj_slot, dc.batch.blk_start, dc.batch.block_ids)
+        rc, *_ = dc.ring.tutti_build_sqes_staged(other, layer, T.OP_READ, stage.data_ptr(), need,
+                                                 allow=(T.EINVAL,))
+        assert rc == T.EINVAL
+    finally:
+        dc.close()

@@ -263,6 +263,9 @@ class Replica:
         self.build_stream = torch.cuda.Stream(self.dev)
         self.write_stream = torch.cuda.Stream(self.dev)
         self.saved_ev = {}          # duplex mode: last save of every layer
+        self.stage_build = torch.cuda.Stream(self.dev)
+        self.stage_bufs = None      # staged mode: two staging buffers per direction
+        self.stage_ev = {}
         # duplex mode: each direction on a few SMs, so that both kernels are resident at once
         # (the host link, not the SM count, bounds them)
         self.duplex_sms = getattr(args, "e2e_sms", 12)
@@ -432,6 +435,83 @@ class Replica:
         self.unpolled = [(fr, L * per_r), (fw, L * per_w)]
         return total
 
+    def step_staged(self, upload_tables=False):
+        """One pass of staged transfers with both directions of the host link busy: the copy
+        engines carry every layer's contexts between the pinned-host store and two pairs of
+        staging buffers in HBM (tutti_stage_copy_layer: one copy per context), the kernels
+        scatter staging -> pool and gather pool -> staging on all SMs in between.  Per layer:
+        copy in -> restore kernel -> save kernel -> copy out; the copy-in of layer l+1 and the
+        copy-out of layer l-1 run beside them on their own streams.  Completions of a pass are
+        polled after the next pass has been issued."""
+        T, torch = self.T, self.torch
+        sK, sIn, sOut, sb = self.stream, self.build_stream, self.write_stream, self.stage_build
+        L = self.w.n_layers
+        self.epoch += 1
+        self.batch.plan_epoch = self.epoch
+        if upload_tables:
+            with torch.cuda.stream(sb):
+                for h, d in zip(self.tables_host, self.tables_dev):
+                    d.copy_(h, non_blocking=True)
+        rc, n_ctx, need = self.ring.tutti_stage_plan(self.batch, stream=sb)     # once per batch
+        self.stage_ctx_mib = need / max(n_ctx, 1) / 2**20
+        if self.stage_bufs is None or self.stage_bufs[0].numel() < need:
+            self.stage_bufs = [torch.empty(need, dtype=torch.uint8, device=self.dev) for _ in range(4)]
+        in_bufs, out_bufs = self.stage_bufs[:2], self.stage_bufs[2:]
+        issued = []
+        for l in range(L):
+            si, so = in_bufs[l % 2], out_bufs[l % 2]
+            # copy in: the staging buffer is free once the restore kernel two layers back is done,
+            # and the store's bytes of this layer are final once its last copy-out has landed
+            for ev in (self.stage_ev.get(("restored", l - 2)), self.stage_ev.get(("out", l, "prev"))):
+                if ev is not None:
+                    sIn.wait_event(ev)
+            self.ring.tutti_stage_copy_layer(l, T.OP_READ, si.data_ptr(), need, stream=sIn)
+            ev_in = torch.cuda.Event()
+            ev_in.record(sIn)
+            rc, fr, nr = self.ring.tutti_build_sqes_staged(self.batch, l, T.OP_READ, si.data_ptr(), need, stream=sb)
+            rc, fw, nw = self.ring.tutti_build_sqes_staged(self.batch, l, T.OP_WRITE, so.data_ptr(), need, stream=sb)
+            built = torch.cuda.Event()
+            built.record(sb)
+            sK.wait_event(ev_in)
+            sK.wait_event(built)
+            self.ring.tutti_kv_restore_layer(fr, nr, 0, stream=sK)
+            ev_r = torch.cuda.Event()
+            ev_r.record(sK)
+            self.stage_ev[("restored", l)] = ev_r
+            ev = self.stage_ev.get(("out", l - 2))
+            if ev is not None:
+                sK.wait_event(ev)                      # the out buffer has been copied out
+            self.ring.tutti_kv_save_layer(fw, nw, 0, stream=sK)
+            ev_g = torch.cuda.Event()
+            ev_g.record(sK)
+            sOut.wait_event(ev_g)
+            self.ring.tutti_stage_copy_layer(l, T.OP_WRITE, so.data_ptr(), need, stream=sOut)
+            ev_o = torch.cuda.Event()
+            ev_o.record(sOut)
+            self.stage_ev[("out", l)] = ev_o
+            issued += [(fr, nr), (fw, nw)]
+        # bookkeeping for the next pass: its buffers and its store bytes depend on this pass
+        nxt = {}
+        for l in range(L):
+            nxt[("out", l, "prev")] = self.stage_ev[("out", l)]
+        nxt[("restored", -2)] = self.stage_ev.get(("restored", L - 2))
+        nxt[("restored", -1)] = self.stage_ev.get(("restored", L - 1))
+        nxt[("out", -2)] = self.stage_ev.get(("out", L - 2))
+        nxt[("out", -1)] = self.stage_ev.get(("out", L - 1))
+        self.stage_ev = nxt
+        total = self.poll_list(self.unpolled)
+        self.unpolled = issued
+        return total
+
+    def finish_staged(self):
+        """Join the copy-out stream into the kernel stream and poll what is outstanding."""
+        for key, ev in self.stage_ev.items():
+            if ev is not None:
+                self.stream.wait_event(ev)
+        total = self.poll_list(self.unpolled)
+        self.unpolled = []
+        return total
+
     def finish_duplex(self):
         """Join the save stream into the restore stream and poll what is outstanding."""
         for ev in self.saved_ev.values():
@@ -440,7 +520,7 @@ class Replica:
         self.unpolled = []
         return total
 
-    def spot_check(self, n_samples=256):
+    def spot_check(self, n_samples=256, original=False):
         """Guard against timing a kernel that did no work: for random (token, head) rows the
         bytes in the pool must equal the bytes in the store, located with the library's own
         layout (tutti_obj_layout strides) and the host copies of the tables.  This is a
@@ -467,6 +547,11 @@ class Replica:
             b = self.pool[l % self.R][po:po + row]
             if not torch.equal(a, b):
                 return False
+            if original:
+                # restore-then-save passes leave the store as it was generated
+                g = self.wl.fill_u16_torch(w.seed, STREAM_STORE + d, so // 2, row // 2, self.dev)
+                if not torch.equal(a, g.view(torch.uint8)):
+                    return False
         return True
 
 
@@ -843,65 +928,87 @@ def run_e2e(args, local_rank, world):
     a2.layers_per_launch = 4
     rep = Replica(a2, local_rank, host_store=True, n_layers=L_host)
     passes = max(1, 32 // L_host) if args.config in (2, 5) else 1
-    duplex = not args.e2e_serial
-    if duplex:
-        rep.ctx.tutti_set_option(rep.T.OPT_COPY_ENGINE, rep.T.ENGINE_BULK)
-    times = {}
-
-    def one_pass():
-        if duplex:
-            return rep.step_duplex(upload_tables=True, group=args.e2e_group, times=times)
-        return rep.step(upload_tables=True)
-    one_pass()
-    if duplex:
-        rep.finish_duplex()
-    torch.cuda.synchronize()
-    times.clear()
-    barrier(world)
     steps = max(1, min(args.steps, 3))
-    t0 = time.perf_counter()
-    e0 = torch.cuda.Event(enable_timing=True)
-    e1 = torch.cuda.Event(enable_timing=True)
-    e0.record(rep.stream)
-    moved = 0
-    for _ in range(steps * passes):
-        moved += one_pass()
-    if duplex:
-        moved += rep.finish_duplex()
-    e1.record(rep.stream)
-    torch.cuda.synchronize()
-    wall_ms = (time.perf_counter() - t0) * 1e3
-    ms = max_over_ranks(max(e0.elapsed_time(e1), wall_ms), world, rep.dev) / steps
     layers = L_host * passes
     payload = 2 * layers * rep.payload_per_layer
-    assert moved == payload * steps, (moved, payload * steps)
-    ok = rep.spot_check(64)
-    per_dir = None
-    if duplex and times:
-        # each direction's own rate: its bytes over the time its stream was busy with them
-        per_dir = {}
-        for key, a, b in (("restore_gbs", "r0", "r1"), ("save_gbs", "w0", "w1")):
-            busy = times[a][0].elapsed_time(times[b][-1])
-            per_dir[key] = round(steps * layers * rep.payload_per_layer / (busy * 1e-3) / 1e9, 2)
+    T = rep.T
+
+    def measure(mode):
+        """ms per step of one mode: 'zero_copy' (the kernels read and write the store over the
+        link), 'staged' (copy engines on the link, kernels on HBM) or 'serial'."""
+        times = {}
+        if mode == "zero_copy":
+            rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, T.ENGINE_BULK)
+            one_pass = lambda: rep.step_duplex(upload_tables=True, group=args.e2e_group, times=times)
+            finish = rep.finish_duplex
+        elif mode == "staged":
+            rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, args.engine or T.ENGINE_AUTO)
+            one_pass = lambda: rep.step_staged(upload_tables=True)
+            finish = rep.finish_staged
+        else:
+            one_pass = lambda: rep.step(upload_tables=True)
+            finish = lambda: 0
+        one_pass()
+        finish()
+        torch.cuda.synchronize()
+        times.clear()
+        barrier(world)
+        t0 = time.perf_counter()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(rep.stream)
+        moved = 0
+        for _ in range(steps * passes):
+            moved += one_pass()
+        moved += finish()
+        e1.record(rep.stream)
+        torch.cuda.synchronize()
+        wall_ms = (time.perf_counter() - t0) * 1e3
+        ms = max_over_ranks(max(e0.elapsed_time(e1), wall_ms), world, rep.dev) / steps
+        assert moved == payload * steps, (mode, moved, payload * steps)
+        if not rep.spot_check(64, original=True):
+            raise RuntimeError(f"e2e {mode}: spot check failed")
+        res = {"gbs": round(sum_over_ranks(float(payload), world, rep.dev) / (ms * 1e-3) / 1e9, 2),
+               "ms_per_step": round(ms, 2)}
+        if mode == "staged":
+            # the copy engines' rate depends on the size of a contiguous copy (here, a context)
+            res["mean_copy_mib"] = round(rep.stage_ctx_mib, 2)
+        if mode == "zero_copy" and times:
+            # each direction's own rate: its bytes over the time its stream was busy with them
+            for key, a, b in (("restore_gbs", "r0", "r1"), ("save_gbs", "w0", "w1")):
+                busy = times[a][0].elapsed_time(times[b][-1])
+                res[key] = round(steps * layers * rep.payload_per_layer / (busy * 1e-3) / 1e9, 2)
+        return res
+
+    modes = {"serial": ["serial"], "zero_copy": ["zero_copy"], "staged": ["staged"],
+             "both": ["zero_copy", "staged"]}["serial" if args.e2e_serial else args.e2e_mode]
+    res = {m: measure(m) for m in modes}
+    best = max(res, key=lambda m: res[m]["gbs"])
     link = host_link_gbs(rep.dev) if world == 1 else None
     link_duplex = host_link_duplex_gbs(rep.dev) if world == 1 else None
     h2d = layers * rep.payload_per_layer + passes * rep.table_bytes
     d2h = layers * rep.payload_per_layer + 2 * layers * 32
-    value = sum_over_ranks(float(payload), world, rep.dev) / (ms * 1e-3) / 1e9
-    rep.close()
-    out = {"value": round(value, 2), "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
-           "d2h_bytes_per_step": int(d2h), "ms_per_step": round(ms, 2),
-           "spot_check": bool(ok),
+    if best == "staged":
+        d2h += passes * 24 * len(rep.w.obj_slot)       # the batch's contexts, fetched once per pass
+    describe = {
+        "zero_copy": f"zero-copy duplex: the kernels read and write the pinned-host store over "
+                     f"the link; groups of {args.e2e_group} layers saved while the next group is "
+                     f"restored; restore on {rep.duplex_sms} SMs, save on {rep.duplex_save_sms} SMs",
+        "staged": "staged duplex: copy engines move each layer's contexts between the pinned-host "
+                  "store and staging buffers in HBM (one copy per context), the kernels scatter "
+                  "and gather between staging and pool on all SMs; copy-in of the next layer and "
+                  "copy-out of the previous one run beside them",
+        "serial": "serial: all restores, then all saves"}
+    out = {"value": res[best]["gbs"], "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(d2h), "ms_per_step": res[best]["ms_per_step"],
+           "spot_check": True,
            "host_link_duplex_gbs": None if link_duplex is None else round(link_duplex, 1),
-           "link_frac": None if link_duplex is None else round(value / link_duplex, 4),
-           "mode": f"duplex: groups of {args.e2e_group} layers saved while the next group is "
-                   f"restored (both directions of the host link busy); restore on "
-                   f"{rep.duplex_sms} SMs, save on {rep.duplex_save_sms} SMs"
-                   if duplex else "serial: all restores, then all saves",
-           "store": f"pinned host memory, zero-copy; {L_host} layers resident, "
+           "link_frac": None if link_duplex is None else round(res[best]["gbs"] / link_duplex, 4),
+           "mode": describe[best],
+           "modes": {m: dict(r, what=describe[m]) for m, r in res.items()},
+           "store": f"pinned host memory; {L_host} layers resident, "
                     f"{passes} passes per step = {layers} layer transfers each way"}
-    if per_dir:
-        out.update(per_dir)
+    rep.close()
     if link is not None:
         out["host_link_h2d_gbs"], out["host_link_d2h_gbs"] = round(link[0], 2), round(link[1], 2)
     return out
@@ -1420,6 +1527,8 @@ def main():
                     help="e2e leg, duplex mode: SMs of the save direction")
     ap.add_argument("--e2e-group", type=int, default=2,
                     help="e2e leg, duplex mode: layers per copy launch")
+    ap.add_argument("--e2e-mode", choices=["both", "zero_copy", "staged"], default="both",
+                    help="e2e leg: kernels on the link (zero_copy), copy engines on the link (staged)")
     ap.add_argument("--e2e-serial", action="store_true",
                     help="e2e leg: restore pass then save pass instead of overlapping them")
     ap.add_argument("--gemm-iters", type=int, default=20)

@@ -222,3 +222,46 @@ def test_config5_capped_restore_beside_a_gemm(sm_count):
         rep.ctx.tutti_sm_partition_destroy()
     finally:
         rep.close()
+
+
+def test_config2_staged_duplex_pass_from_pinned_host():
+    """The staged pass the bench's end-to-end leg times (copy engines between the pinned-host
+    store and staging buffers in HBM, kernels between staging and pool, both directions at
+    once): after it, every layer's pool is the oracle's restore, and the store, which every
+    layer was saved back to, still holds its bytes."""
+    rep = bench.Replica(_args(config=2, layers=3, resident_layers=3), 0, host_store=True)
+    try:
+        w = rep.w
+        assert (w.n_req, len(w.block_ids)) == (8, 16384)
+        before = [p.clone() for p in rep.pool]
+        orig = [s.clone() for s in rep.store]
+        moved = rep.step_staged(upload_tables=True)
+        moved += rep.finish_staged()
+        torch.cuda.synchronize()
+        assert moved == 2 * w.n_layers * rep.payload_per_layer
+        assert verify_replica_samples(rep, 256)
+        for l in range(w.n_layers):
+            _whole_layer_check(rep, l, before[l])
+        for s, o in zip(rep.store, orig):
+            assert torch.equal(s, o)
+        # the save half on its own: into a zeroed store, the covered bytes come back
+        for s in rep.store:
+            s.zero_()
+        need = rep.stage_bufs[2].numel()
+        l = w.n_layers - 1
+        rc, fw, nw = rep.ring.tutti_build_sqes_staged(rep.batch, l, T.OP_WRITE,
+                                                      rep.stage_bufs[2].data_ptr(), need,
+                                                      stream=rep.stream)
+        rep.ring.tutti_kv_save_layer(fw, nw, 0, stream=rep.stream)
+        rep.ring.tutti_stage_copy_layer(l, T.OP_WRITE, rep.stage_bufs[2].data_ptr(), need,
+                                        stream=rep.stream)
+        assert rep.poll_list([(fw, nw)]) == rep.payload_per_layer
+        torch.cuda.synchronize()
+        lb = int(rep.lo.stride_layer)
+        for s, o in zip(rep.store, orig):
+            cov = s != 0
+            assert torch.equal(s[cov], o[cov])
+            assert int(cov[l * lb:(l + 1) * lb].sum()) > 0.9 * rep.payload_per_layer
+            assert int(cov.sum()) == int(cov[l * lb:(l + 1) * lb].sum())
+    finally:
+        rep.close()

@@ -435,17 +435,18 @@ class Replica:
         self.unpolled = [(fr, L * per_r), (fw, L * per_w)]
         return total
 
-    def step_staged(self, upload_tables=False):
+    def step_staged(self, upload_tables=False, directions=(0, 1)):
         """One pass of staged transfers with both directions of the host link busy: the copy
         engines carry every layer's contexts between the pinned-host store and two pairs of
         staging buffers in HBM (tutti_stage_copy_layer: one copy per context), the kernels
         scatter staging -> pool and gather pool -> staging on all SMs in between.  Per layer:
         copy in -> restore kernel -> save kernel -> copy out; the copy-in of layer l+1 and the
         copy-out of layer l-1 run beside them on their own streams.  Completions of a pass are
-        polled after the next pass has been issued."""
+        polled after the next pass has been issued.  `directions` may name one direction only."""
         T, torch = self.T, self.torch
         sK, sIn, sOut, sb = self.stream, self.build_stream, self.write_stream, self.stage_build
         L = self.w.n_layers
+        do_r, do_w = T.OP_READ in directions, T.OP_WRITE in directions
         self.epoch += 1
         self.batch.plan_epoch = self.epoch
         if upload_tables:
@@ -458,47 +459,57 @@ class Replica:
             self.stage_bufs = [torch.empty(need, dtype=torch.uint8, device=self.dev) for _ in range(4)]
         in_bufs, out_bufs = self.stage_bufs[:2], self.stage_bufs[2:]
         issued = []
+        prev, cur = self.stage_ev, {}
+        def last(kind, l):
+            """Events that free the staging buffer layer l + 2 is about to use: `kind` of layer
+            l of this pass, or, before layer 0, of the last two layers of the previous pass
+            (either may have used that buffer, depending on the parity of L)."""
+            if l >= 0:
+                return [cur.get((kind, l))]
+            return [prev.get((kind, L - 1)), prev.get((kind, L - 2))]
         for l in range(L):
             si, so = in_bufs[l % 2], out_bufs[l % 2]
-            # copy in: the staging buffer is free once the restore kernel two layers back is done,
-            # and the store's bytes of this layer are final once its last copy-out has landed
-            for ev in (self.stage_ev.get(("restored", l - 2)), self.stage_ev.get(("out", l, "prev"))):
-                if ev is not None:
-                    sIn.wait_event(ev)
-            self.ring.tutti_stage_copy_layer(l, T.OP_READ, si.data_ptr(), need, stream=sIn)
-            ev_in = torch.cuda.Event()
-            ev_in.record(sIn)
-            rc, fr, nr = self.ring.tutti_build_sqes_staged(self.batch, l, T.OP_READ, si.data_ptr(), need, stream=sb)
-            rc, fw, nw = self.ring.tutti_build_sqes_staged(self.batch, l, T.OP_WRITE, so.data_ptr(), need, stream=sb)
+            if do_r:
+                # copy in: the staging buffer is free once the restore kernel two layers back is
+                # done, and the store's bytes of this layer are final once its last copy-out
+                # has landed
+                for ev in last("restored", l - 2) + [prev.get(("out", l))]:
+                    if ev is not None:
+                        sIn.wait_event(ev)
+                self.ring.tutti_stage_copy_layer(l, T.OP_READ, si.data_ptr(), need, stream=sIn)
+                ev_in = torch.cuda.Event()
+                ev_in.record(sIn)
+                rc, fr, nr = self.ring.tutti_build_sqes_staged(self.batch, l, T.OP_READ, si.data_ptr(),
+                                                               need, stream=sb)
+                issued.append((fr, nr))
+            if do_w:
+                rc, fw, nw = self.ring.tutti_build_sqes_staged(self.batch, l, T.OP_WRITE, so.data_ptr(),
+                                                               need, stream=sb)
+                issued.append((fw, nw))
             built = torch.cuda.Event()
             built.record(sb)
-            sK.wait_event(ev_in)
             sK.wait_event(built)
-            self.ring.tutti_kv_restore_layer(fr, nr, 0, stream=sK)
-            ev_r = torch.cuda.Event()
-            ev_r.record(sK)
-            self.stage_ev[("restored", l)] = ev_r
-            ev = self.stage_ev.get(("out", l - 2))
-            if ev is not None:
-                sK.wait_event(ev)                      # the out buffer has been copied out
-            self.ring.tutti_kv_save_layer(fw, nw, 0, stream=sK)
-            ev_g = torch.cuda.Event()
-            ev_g.record(sK)
-            sOut.wait_event(ev_g)
-            self.ring.tutti_stage_copy_layer(l, T.OP_WRITE, so.data_ptr(), need, stream=sOut)
-            ev_o = torch.cuda.Event()
-            ev_o.record(sOut)
-            self.stage_ev[("out", l)] = ev_o
-            issued += [(fr, nr), (fw, nw)]
-        # bookkeeping for the next pass: its buffers and its store bytes depend on this pass
-        nxt = {}
-        for l in range(L):
-            nxt[("out", l, "prev")] = self.stage_ev[("out", l)]
-        nxt[("restored", -2)] = self.stage_ev.get(("restored", L - 2))
-        nxt[("restored", -1)] = self.stage_ev.get(("restored", L - 1))
-        nxt[("out", -2)] = self.stage_ev.get(("out", L - 2))
-        nxt[("out", -1)] = self.stage_ev.get(("out", L - 1))
-        self.stage_ev = nxt
+            if do_r:
+                sK.wait_event(ev_in)
+                self.ring.tutti_kv_restore_layer(fr, nr, 0, stream=sK)
+                ev_r = torch.cuda.Event()
+                ev_r.record(sK)
+                cur[("restored", l)] = ev_r
+            if do_w:
+                for ev in last("out", l - 2):
+                    if ev is not None:
+                        sK.wait_event(ev)              # the out buffer has been copied out
+                self.ring.tutti_kv_save_layer(fw, nw, 0, stream=sK)
+                ev_g = torch.cuda.Event()
+                ev_g.record(sK)
+                sOut.wait_event(ev_g)
+                self.ring.tutti_stage_copy_layer(l, T.OP_WRITE, so.data_ptr(), need, stream=sOut)
+                ev_o = torch.cuda.Event()
+                ev_o.record(sOut)
+                cur[("out", l)] = ev_o
+        for key, ev in prev.items():
+            cur.setdefault(key, ev)                     # a direction this pass did not run
+        self.stage_ev = cur
         total = self.poll_list(self.unpolled)
         self.unpolled = issued
         return total
@@ -1097,6 +1108,25 @@ def leg_config3(args, local_rank):
                 "payload_gbs": round(gbs, 2), "ms_per_layer": round(ms, 3),
                 "link_frac": round(gbs / link, 4), "hbm_frac": round(gbs / peak, 5),
                 "blocks_per_s": round(rep.blocks_per_layer / (ms * 1e-3))}
+    # the same transfers staged: copy engines on the link, kernels between staging and pool
+    rep.ctx.tutti_set_option(T.OPT_COPY_ENGINE, T.ENGINE_AUTO)
+    for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
+        rep.step_staged(directions=dirs)
+        rep.finish_staged()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(rep.stream)
+        for _ in range(passes):
+            rep.step_staged(directions=dirs)
+        rep.finish_staged()
+        e1.record(rep.stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / (passes * L_host)
+        gbs = rep.payload_per_layer / (ms * 1e-3) / 1e9
+        link = h2d if name == "restore" else d2h
+        out[f"{name}_staged"] = {"payload_gbs": round(gbs, 2), "ms_per_layer": round(ms, 3),
+                                 "link_frac": round(gbs / link, 4),
+                                 "mean_copy_mib": round(rep.stage_ctx_mib, 2)}
     out["spot_check"] = bool(rep.spot_check())
     rep.close()
     return out

@@ -266,6 +266,8 @@ class Replica:
         self.stage_build = torch.cuda.Stream(self.dev)
         self.stage_bufs = None      # staged mode: two staging buffers per direction
         self.stage_ev = {}
+        # staged mode: contexts below this size stay on the zero-copy path
+        self.stage_min_bytes = int(getattr(args, "stage_min_mib", 2.0) * 2**20)
         # duplex mode: each direction on a few SMs, so that both kernels are resident at once
         # (the host link, not the SM count, bounds them)
         self.duplex_sms = getattr(args, "e2e_sms", 12)
@@ -453,8 +455,11 @@ class Replica:
             with torch.cuda.stream(sb):
                 for h, d in zip(self.tables_host, self.tables_dev):
                     d.copy_(h, non_blocking=True)
-        rc, n_ctx, need = self.ring.tutti_stage_plan(self.batch, stream=sb)     # once per batch
-        self.stage_ctx_mib = need / max(n_ctx, 1) / 2**20
+        rc, n_ctx, n_st, need = self.ring.tutti_stage_plan(self.batch, self.stage_min_bytes,
+                                                           stream=sb)         # once per batch
+        self.stage_ctx_mib = need / max(n_st, 1) / 2**20
+        self.stage_frac = need / self.payload_per_layer      # no shared objects in these legs
+        need = max(need, 16)
         if self.stage_bufs is None or self.stage_bufs[0].numel() < need:
             self.stage_bufs = [torch.empty(need, dtype=torch.uint8, device=self.dev) for _ in range(4)]
         in_bufs, out_bufs = self.stage_bufs[:2], self.stage_bufs[2:]
@@ -984,6 +989,8 @@ def run_e2e(args, local_rank, world):
         if mode == "staged":
             # the copy engines' rate depends on the size of a contiguous copy (here, a context)
             res["mean_copy_mib"] = round(rep.stage_ctx_mib, 2)
+            res["staged_frac"] = round(rep.stage_frac, 4)
+            res["stage_min_mib"] = args.stage_min_mib
         if mode == "zero_copy" and times:
             # each direction's own rate: its bytes over the time its stream was busy with them
             for key, a, b in (("restore_gbs", "r0", "r1"), ("save_gbs", "w0", "w1")):
@@ -1559,6 +1566,8 @@ def main():
                     help="e2e leg, duplex mode: layers per copy launch")
     ap.add_argument("--e2e-mode", choices=["both", "zero_copy", "staged"], default="both",
                     help="e2e leg: kernels on the link (zero_copy), copy engines on the link (staged)")
+    ap.add_argument("--stage-min-mib", type=float, default=2.0,
+                    help="staged transfers: contexts smaller than this stay on the zero-copy path")
     ap.add_argument("--e2e-serial", action="store_true",
                     help="e2e leg: restore pass then save pass instead of overlapping them")
     ap.add_argument("--gemm-iters", type=int, default=20)

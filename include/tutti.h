@@ -369,23 +369,30 @@ int tutti_ring_set_iocb_bytes(tutti_ring_t *ring, uint64_t bytes);
  *
  *   tutti_stage_plan        once per batch (plan_epoch != 0): runs the plan on `stream` if the
  *                           ring does not hold it, waits for it and keeps the batch's contexts
- *                           on the host.  Host out: *n_ctx contexts, *bytes_per_layer the
- *                           staging bytes a layer needs (the distinct object bytes of the
- *                           batch).  Blocks the host: a per-request call, not a per-layer one.
+ *                           on the host.  A context of at least min_ctx_bytes is staged; a
+ *                           smaller one keeps its entries pointing into the store and is moved
+ *                           by the kernels alone (a copy engine pays a fixed start-up per copy:
+ *                           below about 2 MiB per copy the zero-copy path is the faster one);
+ *                           0 stages every context.  Host out: *n_ctx contexts, *n_staged of
+ *                           them staged, *bytes_per_layer the staging bytes a layer needs (the
+ *                           distinct object bytes of the staged contexts).  Blocks the host: a
+ *                           per-request call, not a per-layer one.
  *   tutti_stage_copy_layer  enqueues on `stream` the copies of layer `layer`: store -> staging
  *                           for TUTTI_OP_READ, staging -> store for TUTTI_OP_WRITE.  `stage` is a
  *                           device pointer to at least *bytes_per_layer bytes, 16-byte aligned,
  *                           owned by the caller.  Works for HBM and pinned-host stores alike.
  *   tutti_build_sqes_staged tutti_build_sqes for one layer with the object side of every entry
- *                           pointing into `stage` (contexts still carry the store offsets).
+ *                           of a staged context pointing into `stage` (contexts still carry the
+ *                           store offsets).
  *                           The IOCBs are then executed with tutti_kv_restore_layer (after the
  *                           copies into `stage`) or tutti_kv_save_layer (before the copies out
  *                           of it); ordering between copies and kernels is the caller's (stream
  *                           order or events).
  * TUTTI_EINVAL if the batch is not the one tutti_stage_plan saw, or `stage` is too small.
  */
-int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch, void *stream,
-                     uint32_t *n_ctx, uint64_t *bytes_per_layer);
+int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch,
+                     uint64_t min_ctx_bytes, void *stream, uint32_t *n_ctx, uint32_t *n_staged,
+                     uint64_t *bytes_per_layer);
 int tutti_stage_copy_layer(tutti_ctx_t *ctx, tutti_ring_t *ring, uint32_t layer, uint32_t opcode,
                            void *stage, uint64_t stage_bytes, void *stream);
 int tutti_build_sqes_staged(tutti_ctx_t *ctx, tutti_ring_t *ring, const tutti_batch_t *batch,

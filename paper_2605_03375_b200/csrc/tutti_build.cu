@@ -356,18 +356,6 @@ plan_kernel(RingDev ring, GeomDev g, BatchDev b, uint32_t np, int use_smem, int 
         }
     }
     __syncthreads();
-    // where every context sits in a staging buffer that holds the contexts' bytes packed in
-    // order: the blocks named by the contexts before it (exclusive prefix sum)
-    if (threadIdx.x == 0) { carry.a = 0; carry.b = 0; carry.m = 0; }
-    __syncthreads();
-    for (uint32_t base = 0; base < n_sqe; base += blockDim.x) {
-        const uint32_t q = base + threadIdx.x;
-        ScanVals v{0, 0, 0};
-        if (q < n_sqe) v.a = (uint32_t)(ring.plan_sqe[q].len / g.block_bytes);
-        const uint32_t mine = v.a;
-        const ScanVals sc = block_scan_incl(v, warp_tot, carry);
-        if (q < n_sqe) ring.plan_stage[q] = sc.a - mine;
-    }
     if (threadIdx.x == 0) {
         PlanCounts pc;
         pc.n_items = n_act;
@@ -566,8 +554,9 @@ emit_kernel(RingDev ring, GeomDev g, BatchDev b, EmitParams p) {
                 note_error(&hdr0->emit_status, TUTTI_EFAULT);
                 meta1 = 0;
                 n_blk = 0;                             // nothing is emitted for this item
-            } else if (p.stage_base == 0) {
-                meta1 = p.store_base[dev] + off;
+            } else if (p.stage_base == 0 ||
+                       ring.plan_stage[ring.plan_sqe_of[gs]] == STAGE_NONE) {
+                meta1 = p.store_base[dev] + off;       // this context's bytes stay in the store
             } else {
                 // staged transfer: the item's bytes sit in the staging buffer at its context's
                 // place plus its distance from the context's first byte

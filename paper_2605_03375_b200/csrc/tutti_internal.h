@@ -71,6 +71,9 @@ struct StoreDev {
 };
 
 // Device-side view of a ring, passed by value to kernels.
+// plan_stage[] of a context that is not staged (its entries keep pointing into the store)
+constexpr uint32_t STAGE_NONE = 0xffffffffu;
+
 struct RingDev {
     IocbHdr *hdrs;            // [depth]
     tutti_sqe_t *sqes;        // [depth * capacity]
@@ -88,8 +91,8 @@ struct RingDev {
     uint32_t *plan_grp;       // [max_items]  index of the first item of the item's group (items
                               //              that name exactly the same bytes form a group)
     uint32_t *plan_k;         // [max_items]  at a group's first item: members of the group
-    uint32_t *plan_stage;     // [max_items]  per context: blocks named by the contexts before it
-                              //              (where it sits in a staging buffer packed in order)
+    uint32_t *plan_stage;     // [max_items]  per context: its place in a staging buffer, in blocks, or
+                              //              STAGE_NONE; written by the host (tutti_stage_plan)
     tutti_sqe_t *plan_sqe;    // [max_items]  contexts for layer 0, opcode unset
     unsigned long long *plan_key;  // [pow2(max_items)] sort keys when they do not fit in shared memory
     uint32_t *plan_idx;       // [pow2(max_items)] sort payload, same

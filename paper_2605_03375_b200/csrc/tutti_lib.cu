@@ -88,13 +88,15 @@ struct tutti_ring {
     std::vector<uint64_t> fill_optr;      // tutti_ring_fill_host scratch (sized at create)
     std::vector<uint8_t> fill_seen;
     uint32_t entries_per_iocb = 0;        // IOCBs cut by entries (0: by context count)
-    std::vector<uint8_t> staged;          // per slot: the IOCB's object side is a staging buffer
+    std::vector<uint8_t> staged;          // per slot: 0 the object side of the IOCB is the store,
+                                          // 1 a staging buffer, 2 either, context by context
     // staged transfers: the batch's contexts (layer 0) on the host, and where each sits in a
     // staging buffer packed in context order
     std::vector<tutti_sqe_t> stage_ctx;
     std::vector<uint64_t> stage_off;
     uint64_t stage_layer_bytes = 0;
     bool stage_valid = false;
+    bool stage_all = true;                // every context of the stage plan goes through staging
     tutti_batch_t stage_batch{};
     uint32_t *smid_log = nullptr;         // device: SM of every CTA of the last copy launch
     uint32_t smid_cap = 0, last_grid = 0;
@@ -475,7 +477,7 @@ static int build_layers(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *
         r->have_cqe[slot] = 0;
         r->opcode_of[slot] = (uint8_t)opcode;
         r->issued[slot] = 0;
-        r->staged[slot] = stage_base != 0;
+        r->staged[slot] = stage_base == 0 ? 0 : (r->stage_all ? 1 : 2);
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t st = (cudaStream_t)stream;
@@ -535,21 +537,25 @@ static int issue(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t first, uint32_t n, 
     bool host_store = false;
     for (uint32_t d = 0; d < ctx->geom.n_devices; ++d)
         host_store |= ctx->store[d].kind == TUTTI_STORE_HOST_PINNED;
-    bool all_staged = true;
+    bool all_staged = true, any_staged = false;
     for (uint32_t k = 0; k < n; ++k) {
         uint32_t idx = first + k;
         if (!r->host->is_live(idx)) return TUTTI_EINVAL;
         uint8_t op = r->opcode_of[idx & (r->dev.depth - 1)];
         if (op != 0xff && op != opcode) return TUTTI_EINVAL;
-        all_staged = all_staged && r->staged[idx & (r->dev.depth - 1)];
+        const uint8_t sg = r->staged[idx & (r->dev.depth - 1)];
+        all_staged = all_staged && sg == 1;
+        any_staged = any_staged || sg != 0;
     }
-    bool any_staged = false;
-    for (uint32_t k = 0; k < n; ++k) any_staged = any_staged || r->staged[(first + k) & (r->dev.depth - 1)];
     if (all_staged) host_store = false;      // the object side of these IOCBs is a buffer in HBM
     // head-major blocks are transposed with tensor maps of the store regions, which a staging
-    // buffer is not part of: staged IOCBs take the vector path, and one launch is all of one kind
-    if (ctx->pool_hnd && any_staged && !all_staged) return TUTTI_EINVAL;
-    const StoreTensorMaps *maps = (ctx->pool_hnd && all_staged) ? nullptr : &ctx->maps;
+    // buffer is not part of: a launch with staged IOCBs takes the vector path, which follows any
+    // address; staged and unstaged IOCBs do not share a launch there
+    if (ctx->pool_hnd && any_staged) {
+        for (uint32_t k = 0; k < n; ++k)
+            if (r->staged[(first + k) & (r->dev.depth - 1)] == 0) return TUTTI_EINVAL;
+    }
+    const StoreTensorMaps *maps = (ctx->pool_hnd && any_staged) ? nullptr : &ctx->maps;
     DeviceGuard guard(ctx->device);
     uint32_t launches = 0;
     PermGeom pg{ctx->geom.block_tokens, ctx->geom.n_kv_heads,
@@ -651,8 +657,9 @@ int tutti_ring_poll_range(tutti_ring_t *r, uint32_t first_iocb, uint32_t n_iocb,
     return rc;
 }
 
-int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch, void *stream,
-                     uint32_t *n_ctx, uint64_t *bytes_per_layer) {
+int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *batch,
+                     uint64_t min_ctx_bytes, void *stream, uint32_t *n_ctx, uint32_t *n_staged,
+                     uint64_t *bytes_per_layer) {
     if (!ctx || !r || r->ctx != ctx || !batch || batch->plan_epoch == 0) return TUTTI_EINVAL;
     r->host_calls++;
     if (batch->n_req && (!batch->hit_tokens || !batch->obj_start || !batch->blk_start))
@@ -681,15 +688,34 @@ int tutti_stage_plan(tutti_ctx_t *ctx, tutti_ring_t *r, const tutti_batch_t *bat
     if (pc.n_sqe)
         CK(cudaMemcpy(r->stage_ctx.data(), r->dev.plan_sqe, sizeof(tutti_sqe_t) * pc.n_sqe,
                       cudaMemcpyDeviceToHost));
+    // a context of at least min_ctx_bytes goes through the staging buffer, packed behind the
+    // staged contexts before it; a smaller one stays with the kernels (a copy engine pays a
+    // fixed start-up per copy)
     uint64_t at = 0;
+    uint32_t staged = 0;
+    const uint64_t bb = ctx->layout.block_bytes;
+    std::vector<uint32_t> place(pc.n_sqe);
     for (uint32_t k = 0; k < pc.n_sqe; ++k) {
-        r->stage_off[k] = at;
-        at += r->stage_ctx[k].len;
+        if (r->stage_ctx[k].len >= min_ctx_bytes) {
+            if (at / bb >= STAGE_NONE) return TUTTI_EINVAL;
+            r->stage_off[k] = at;
+            place[k] = (uint32_t)(at / bb);
+            at += r->stage_ctx[k].len;
+            ++staged;
+        } else {
+            r->stage_off[k] = UINT64_MAX;
+            place[k] = STAGE_NONE;
+        }
     }
+    if (pc.n_sqe)
+        CK(cudaMemcpy(r->dev.plan_stage, place.data(), sizeof(uint32_t) * pc.n_sqe,
+                      cudaMemcpyHostToDevice));
     r->stage_layer_bytes = at;
+    r->stage_all = (staged == pc.n_sqe);
     r->stage_batch = *batch;
     r->stage_valid = true;
     if (n_ctx) *n_ctx = pc.n_sqe;
+    if (n_staged) *n_staged = staged;
     if (bytes_per_layer) *bytes_per_layer = at;
     return TUTTI_OK;
 }
@@ -707,6 +733,7 @@ int tutti_stage_copy_layer(tutti_ctx_t *ctx, tutti_ring_t *r, uint32_t layer, ui
     const uint64_t layer_off = (uint64_t)layer * ctx->layout.stride_layer;
     for (size_t k = 0; k < r->stage_ctx.size(); ++k) {
         const tutti_sqe_t &c = r->stage_ctx[k];
+        if (r->stage_off[k] == UINT64_MAX) continue;          // not staged: the kernels move it
         if (c.dev >= ctx->geom.n_devices || !ctx->store[c.dev].registered) return TUTTI_EINVAL;
         if (c.src_off + layer_off + c.len > ctx->store[c.dev].bytes) return TUTTI_EFAULT;
         char *in_store = reinterpret_cast<char *>(ctx->store[c.dev].base + c.src_off + layer_off);

@@ -121,7 +121,7 @@ def load(path: Optional[str] = None) -> C.CDLL:
         "tutti_ring_read_sgl": (C.c_int, [vp, u32, vp, u32, P(u32)]),
         "tutti_ring_stats": (C.c_int, [vp, P(u64), P(u64)]),
         "tutti_ring_set_iocb_bytes": (C.c_int, [vp, u64]),
-        "tutti_stage_plan": (C.c_int, [vp, vp, P(Batch), vp, P(u32), P(u64)]),
+        "tutti_stage_plan": (C.c_int, [vp, vp, P(Batch), u64, vp, P(u32), P(u32), P(u64)]),
         "tutti_stage_copy_layer": (C.c_int, [vp, vp, u32, u32, vp, u64, vp]),
         "tutti_build_sqes_staged": (C.c_int, [vp, vp, P(Batch), u32, u32, vp, u64, vp, P(u32), P(u32)]),
         "tutti_ring_last_launch_sms": (C.c_int, [vp, vp, u32, P(u32)]),
@@ -352,13 +352,16 @@ class Ring:
                                             C.byref(n)), "tutti_ring_read_sgl")
         return sgl[:min(n.value, max_entries)].copy()
 
-    def tutti_stage_plan(self, batch: Batch, stream=None, allow: Sequence[int] = ()):
-        """(rc, n_ctx, bytes_per_layer): the batch's contexts are fetched to the host, once."""
-        n, b = C.c_uint32(), C.c_uint64()
-        rc = _check(self.lib.tutti_stage_plan(self.ctx.h, self.h, C.byref(batch),
-                                              _stream_ptr(stream), C.byref(n), C.byref(b)),
+    def tutti_stage_plan(self, batch: Batch, min_ctx_bytes: int = 0, stream=None,
+                         allow: Sequence[int] = ()):
+        """(rc, n_ctx, n_staged, bytes_per_layer): the batch's contexts are fetched to the host,
+        once; contexts below min_ctx_bytes stay on the zero-copy path."""
+        n, ns, b = C.c_uint32(), C.c_uint32(), C.c_uint64()
+        rc = _check(self.lib.tutti_stage_plan(self.ctx.h, self.h, C.byref(batch), min_ctx_bytes,
+                                              _stream_ptr(stream), C.byref(n), C.byref(ns),
+                                              C.byref(b)),
                     "tutti_stage_plan", allow)
-        return rc, n.value, b.value
+        return rc, n.value, ns.value, b.value
 
     def tutti_stage_copy_layer(self, layer: int, opcode: int, stage: int, stage_bytes: int,
                                stream=None, allow: Sequence[int] = ()) -> int:

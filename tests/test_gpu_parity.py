@@ -453,7 +453,8 @@ def test_iocbs_cut_by_bytes(name, per):
 @pytest.mark.parametrize("name", ["cfg2-small", "shared-prefix-8-requests", "cfg4-small",
                                   "cfg2-2dev-interleaved", "hnd-pool"])
 @pytest.mark.parametrize("host_store", [False, True])
-def test_staged_transfer_matches_oracle(name, host_store):
+@pytest.mark.parametrize("min_ctx", [0, "median"])
+def test_staged_transfer_matches_oracle(name, host_store, min_ctx):
     """Staged restore and save: the copy engines move every context between the store and a
     staging buffer in HBM (one copy per context), the kernels scatter / gather between that
     buffer and the pool.  The pool after a staged restore and the store after a staged save
@@ -462,10 +463,15 @@ def test_staged_transfer_matches_oracle(name, host_store):
     dc = DeviceCase(w, host_store=host_store)
     try:
         dc.batch.plan_epoch = 11
-        rc, n_ctx, need = dc.ring.tutti_stage_plan(dc.batch)
         layer = w.n_layers - 1
         orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, 2048)
-        assert n_ctx == len(osq) and need == int(osq["len"].sum())
+        # "median": the contexts below the median length stay on the zero-copy path (their
+        # entries keep pointing into the store), the others go through the staging buffer
+        lens = osq["len"].astype(np.uint64)
+        min_ctx = int(np.median(lens)) if min_ctx == "median" else 0
+        rc, n_ctx, n_st, need = dc.ring.tutti_stage_plan(dc.batch, min_ctx)
+        assert n_ctx == len(osq) and n_st == int((lens >= min_ctx).sum())
+        assert need == int(lens[lens >= min_ctx].sum())
         stage = torch.zeros(need + 64, dtype=torch.uint8, device=dc.dev)
         # a stage that is too small is refused before anything is enqueued
         assert dc.ring.tutti_stage_copy_layer(layer, T.OP_READ, stage.data_ptr(), need - 16,

@@ -509,3 +509,71 @@ def test_staged_transfer_matches_oracle(name, host_store, min_ctx):
         assert rc == T.EINVAL
     finally:
         dc.close()
+
+
+@pytest.mark.parametrize("name", ["cfg2-small", "shared-prefix-8-requests", "cfg4-small"])
+@pytest.mark.parametrize("sm_count", [0, 8])
+def test_staged_transfer_with_cut_iocbs_on_a_wrapping_ring(name, sm_count):
+    """Staged transfers composed with the rest: IOCBs cut by bytes (several per layer, a context
+    split between two of them), a ring so small that it wraps and a build meets TUTTI_EAGAIN
+    until the host has polled, capped and all-SM launches, every layer in turn, both directions.
+    Descriptors are the oracle's for the cut build, bytes are the oracle's."""
+    w = mk(name)
+    n_ent = 2 * len(w.block_ids)
+    per = max(3, n_ent // 5)                      # about 5 IOCBs per layer
+    per_layer = -(-n_ent // per)
+    depth = 1
+    while depth < 2 * per_layer:
+        depth *= 2                                # room for two builds, not for three
+    dc = DeviceCase(w, depth=depth, capacity=2048, sgl_capacity=3 * n_ent, host_store=True)
+    try:
+        bb = int(dc.ctx.layout.block_bytes)
+        dc.ring.tutti_ring_set_iocb_bytes(per * bb)
+        dc.batch.plan_epoch = 5
+        rc, n_ctx, n_st, need = dc.ring.tutti_stage_plan(dc.batch, 0)
+        stage_in = torch.zeros(need, dtype=torch.uint8, device=dc.dev)
+        stage_out = torch.zeros(need, dtype=torch.uint8, device=dc.dev)
+        orig = [s.copy() for s in dc.store_host]
+        outstanding = []
+        saw_eagain = False
+        for it in range(3 * w.n_layers):
+            layer = it % w.n_layers
+            dc.pool_dev[layer].copy_(torch.from_numpy(dc.pool_host[layer]))
+            want = dc.oracle_restore(layer)
+            for op, stage in ((T.OP_READ, stage_in), (T.OP_WRITE, stage_out)):
+                if op == T.OP_READ:
+                    dc.ring.tutti_stage_copy_layer(layer, T.OP_READ, stage.data_ptr(), need)
+                rc, first, n = dc.ring.tutti_build_sqes_staged(dc.batch, layer, op, stage.data_ptr(),
+                                                               need, allow=(T.EAGAIN,))
+                if rc == T.EAGAIN:
+                    saw_eagain = True
+                    for f, k in outstanding:
+                        rcp, nbytes, err, done = dc.ring.tutti_ring_poll_range(f, k, 5_000_000_000)
+                        assert (rcp, err, done) == (T.OK, 0, k)
+                    outstanding = []
+                    rc, first, n = dc.ring.tutti_build_sqes_staged(dc.batch, layer, op,
+                                                                   stage.data_ptr(), need)
+                assert n == per_layer
+                if it < w.n_layers:
+                    sq, sg, num, infos = dc.read_build(first, n)
+                    orc, osq, osg, onum = dc.oracle_descriptors(layer, op, 2048, per)
+                    assert orc == 0 and same_records(sq, osq) and same_records(sg, osg)
+                    assert list(num[:len(onum)]) == list(onum)
+                if op == T.OP_READ:
+                    dc.ring.tutti_kv_restore_layer(first, n, sm_count)
+                else:
+                    dc.ring.tutti_kv_save_layer(first, n, sm_count)
+                    dc.ring.tutti_stage_copy_layer(layer, T.OP_WRITE, stage.data_ptr(), need)
+                outstanding.append((first, n))
+            torch.cuda.synchronize()
+            assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
+        for f, k in outstanding:
+            rcp, nbytes, err, done = dc.ring.tutti_ring_poll_range(f, k, 5_000_000_000)
+            assert (rcp, err, done) == (T.OK, 0, k)
+        assert saw_eagain
+        # restore then save leaves the store as it was
+        torch.cuda.synchronize()
+        for t, s in zip(dc.store_dev, orig):
+            assert np.array_equal(t.cpu().numpy(), s)
+    finally:
+        dc.close()

@@ -1,5 +1,6 @@
 """Seeded random geometries and batches: every case checks descriptors, restore and save
-against the oracle, with a random engine, SM cap and IOCB capacity.  Also two rings driven
+against the oracle, with a random engine, SM cap and IOCB capacity, a third of them as staged
+transfers.  Also two rings driven
 concurrently on two streams."""
 import numpy as np
 import pytest
@@ -53,7 +54,30 @@ def test_random_case(seed):
         sm_count = int(rng.choice([0, 0, 3, 16]))
         layer = int(rng.integers(0, w.n_layers))
         flag = oracle.OP_HND if w.pool_hnd else 0
-        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_READ)
+        # a third of the cases move the bytes staged (copy engine between store and a staging
+        # buffer, kernels between that buffer and the pool), with every context staged or only
+        # those of at least the median length
+        srng = np.random.default_rng(7000 + seed)
+        staged = srng.random() < 0.35
+        stage = None
+        if staged:
+            orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, capacity)
+            lens = osq["len"].astype(np.uint64)
+            min_ctx = int(np.median(lens)) if (len(lens) and srng.random() < 0.5) else 0
+            dc.batch.plan_epoch = 1 + seed
+            rc, n_ctx, n_st, need = dc.ring.tutti_stage_plan(dc.batch, min_ctx)
+            assert (n_ctx, n_st) == (len(lens), int((lens >= min_ctx).sum()))
+            assert need == int(lens[lens >= min_ctx].sum())
+            stage = torch.zeros(max(need, 16), dtype=torch.uint8, device=dc.dev)
+
+        def build(op):
+            if not staged:
+                return dc.ring.tutti_build_sqes(dc.batch, layer, op)
+            if op == T.OP_READ:
+                dc.ring.tutti_stage_copy_layer(layer, op, stage.data_ptr(), stage.numel())
+            return dc.ring.tutti_build_sqes_staged(dc.batch, layer, op, stage.data_ptr(), stage.numel())
+
+        rc, first, n = build(T.OP_READ)
         sq, sg, num, infos = dc.read_build(first, n)
         orc, osq, osg, onum = dc.oracle_descriptors(layer, oracle.OP_READ, capacity)
         assert orc == 0 and all(i.status == 0 for i in infos)
@@ -68,9 +92,12 @@ def test_random_case(seed):
         assert np.array_equal(dc.pool_dev[layer].cpu().numpy(), want)
         for t in dc.store_dev:
             t.zero_()
-        rc, first, n = dc.ring.tutti_build_sqes(dc.batch, layer, T.OP_WRITE)
+        rc, first, n = build(T.OP_WRITE)
         dc.ring.tutti_kv_save_layer(first, n, sm_count)
+        if staged:
+            dc.ring.tutti_stage_copy_layer(layer, T.OP_WRITE, stage.data_ptr(), stage.numel())
         assert all(c[1] == 0 for c in dc.poll_all(first, n))
+        torch.cuda.synchronize()
         st_want = [np.zeros_like(s) for s in dc.store_host]
         dc.oracle_save(layer, want, st_want)
         for t, s in zip(dc.store_dev, st_want):

@@ -35,8 +35,7 @@ constexpr size_t OFF_PLAN_SQE_OF = OFF_PLAN_CUM + 4 * (NA_MAX_ITEMS + 64);
 constexpr size_t OFF_PLAN_OFF = OFF_PLAN_SQE_OF + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_GRP = OFF_PLAN_OFF + 8 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_K = OFF_PLAN_GRP + 4 * NA_MAX_ITEMS;
-constexpr size_t OFF_PLAN_STAGE = OFF_PLAN_K + 4 * NA_MAX_ITEMS;
-constexpr size_t OFF_PLAN_KEY = OFF_PLAN_STAGE + 4 * NA_MAX_ITEMS;
+constexpr size_t OFF_PLAN_KEY = OFF_PLAN_K + 4 * NA_MAX_ITEMS;
 constexpr size_t OFF_PLAN_IDX = OFF_PLAN_KEY + 8 * NA_POW2_ITEMS;
 constexpr size_t OFF_SGL = OFF_PLAN_IDX + 4 * NA_POW2_ITEMS;
 constexpr size_t OFF_OBJ = OFF_SGL + sizeof(tutti_sgl_t) * NA_MAX_ENTRIES;
@@ -142,7 +141,7 @@ extern "C" int tutti_kv_restore_layer_noalloc(const tutti_geom_t *geom, int devi
         r.plan_off = reinterpret_cast<uint64_t *>(base + OFF_PLAN_OFF);
         r.plan_grp = reinterpret_cast<uint32_t *>(base + OFF_PLAN_GRP);
         r.plan_k = reinterpret_cast<uint32_t *>(base + OFF_PLAN_K);
-        r.plan_stage = reinterpret_cast<uint32_t *>(base + OFF_PLAN_STAGE);
+        r.plan_stage = nullptr;                   // staged transfers are not offered here
         r.plan_key = reinterpret_cast<unsigned long long *>(base + OFF_PLAN_KEY);
         r.plan_idx = reinterpret_cast<uint32_t *>(base + OFF_PLAN_IDX);
         r.plan_counts = reinterpret_cast<PlanCounts *>(base + OFF_COUNTS);

@@ -634,7 +634,9 @@ def cpu_baseline(rep, seconds_hint=10.0):
 # ----------------------------------------------------------------------------
 def workload_name(w):
     return (f"cfg{w.name[3:]}: {w.n_layers} layers x {w.n_req} requests x "
-            f"{int(w.hit_tokens.mean())} tokens, 8 KV heads x 128 x bf16, block {w.block_tokens}, "
+            f"{int(w.hit_tokens.mean())} tokens, {w.n_kv_heads} KV heads x {w.head_dim} x "
+            f"{ {1: 'fp8', 2: 'bf16', 4: 'fp32'}.get(w.elem_bytes, str(w.elem_bytes) + ' B') }, "
+            f"block {w.block_tokens}, "
             f"objects of {w.obj_tokens} tokens, pool {w.n_pool_blocks} blocks 60% occupied")
 
 
@@ -1422,11 +1424,14 @@ def sweep_rows(args, local_rank, token_list, host_store=False, n_layers=32):
     for tokens in token_list:
         a2 = argparse.Namespace(**vars(args))
         a2.config, a2.scale, a2.layers = 2, 1.0, 0
-        a2.resident_layers = 4
+        # every layer has a pool buffer of its own: one launch moves all layers, its agents work
+        # on several layers at once, and layers that shared a buffer would meet in L2
+        a2.resident_layers = n_layers
         a2.ioctx_per_iocb = 2048
         a2.layers_per_launch = 0
         a2.iocb_mib = 0
         rep = Replica(a2, local_rank, host_store=host_store, n_layers=n_layers, hit_tokens=[tokens])
+        assert rep.R == n_layers
         res = {"prefix_tokens": tokens,
                "payload_mib_per_layer": round(rep.payload_per_layer / (1 << 20), 1)}
         for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):

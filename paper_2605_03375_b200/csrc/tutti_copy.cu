@@ -685,6 +685,11 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
     // size as the estimate of all of them, a claim grows to about half an agent's share of the
     // launch (the option's value stays when one IOCB alone feeds every agent several times), and
     // agent a starts at the IOCB that this claim size assigns to it, walking on cyclically.
+    // Half a share is too coarse a grain once the share is large (IOCBs of tens of MiB: the
+    // last claims would decide when the launch ends): beyond MID_CLAIM units the claim stops
+    // there and the agents are dealt out evenly over the IOCBs instead, so that each still
+    // opens about one IOCB and takes its share from it in several claims.
+    constexpr uint32_t MID_CLAIM = 8;
     if (p.n_iocb > 1) {
         uint32_t start = 0, cl = claim;
         if (lane == 0) {
@@ -700,9 +705,15 @@ copy_bulk_kernel(CopyParams p, const __grid_constant__ StoreTensorMaps tm) {
                         ((unsigned long long)u * p.n_iocb + n_agents - 1) / n_agents;
                     const unsigned long long half = (share + 1) / 2;
                     if (half > cl) cl = (uint32_t)(half < u ? half : u);
-                    const uint32_t per = u / cl + (u % cl != 0);       // agents one IOCB feeds
                     const uint32_t agent = warp * gridDim.x + blockIdx.x;
-                    start = min(agent / per, p.n_iocb - 1);
+                    if (cl > MID_CLAIM && cl > claim) {
+                        cl = max(MID_CLAIM, claim);
+                        start = min((uint32_t)((unsigned long long)agent * p.n_iocb / n_agents),
+                                    p.n_iocb - 1);
+                    } else {
+                        const uint32_t per = u / cl + (u % cl != 0);   // agents one IOCB feeds
+                        start = min(agent / per, p.n_iocb - 1);
+                    }
                 }
             }
         }

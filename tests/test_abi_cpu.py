@@ -184,3 +184,17 @@ def test_hostring_cancel_last_restores_the_previous_state():
     assert r.reserve(4, 100) == (0, 0, 0)
     assert r.release(1) == 0
     assert r.cancel_last(0) == T.EINVAL                 # already partly consumed
+
+
+def test_null_handles_are_refused_without_a_gpu():
+    """Entry points that take a context and a ring answer TUTTI_EINVAL for null handles before
+    they touch the device: no GPU is needed to see that."""
+    lib = T.load()
+    n, ns, b, f, k = C.c_uint32(), C.c_uint32(), C.c_uint64(), C.c_uint32(), C.c_uint32()
+    assert lib.tutti_stage_plan(None, None, None, 0, None, C.byref(n), C.byref(ns), C.byref(b)) == T.EINVAL
+    assert lib.tutti_stage_copy_layer(None, None, 0, T.OP_READ, None, 0, None) == T.EINVAL
+    assert lib.tutti_build_sqes_staged(None, None, None, 0, T.OP_READ, None, 0, None,
+                                       C.byref(f), C.byref(k)) == T.EINVAL
+    assert lib.tutti_build_sqes(None, None, None, 0, T.OP_READ, None, C.byref(f), C.byref(k)) == T.EINVAL
+    assert lib.tutti_kv_restore_layer(None, None, 0, 1, 0, None) == T.EINVAL
+    assert lib.tutti_kv_save_layer(None, None, 0, 1, 0, None) == T.EINVAL

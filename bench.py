@@ -1451,18 +1451,31 @@ def sweep_rows(args, local_rank, token_list, host_store=False, n_layers=32):
         assert rep.R == n_layers
         res = {"prefix_tokens": tokens,
                "payload_mib_per_layer": round(rep.payload_per_layer / (1 << 20), 1)}
-        for name, dirs in (("restore", (T.OP_READ,)), ("save", (T.OP_WRITE,))):
+        L, st = rep.w.n_layers, rep.stream
+        for name, op in (("restore", T.OP_READ), ("save", T.OP_WRITE)):
+            issue = rep.ring.tutti_kv_restore_layer if op == T.OP_READ else rep.ring.tutti_kv_save_layer
+
+            def one_pass():
+                # a pass as a user issues it: one build call and one copy launch for all layers,
+                # then the completions of every layer
+                rep.epoch += 1
+                rep.batch.plan_epoch = rep.epoch
+                rc, first, per = rep.ring.tutti_build_sqes_layers(rep.batch, 0, L, op, stream=st)
+                issue(first, L * per, 0, stream=st)
+                rc, nbytes, err, done = rep.ring.tutti_ring_poll_range(first, L * per, 20_000_000_000)
+                assert (rc, err, nbytes) == (T.OK, 0, L * rep.payload_per_layer)
             for _ in range(2):
-                rep.step(directions=dirs)
+                one_pass()
             torch.cuda.synchronize()
-            reps = 5 if tokens <= 16384 else 2
+            reps = 10 if tokens <= 16384 else 3
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(rep.stream)
+            t0 = time.perf_counter()
+            e0.record(st)
             for _ in range(reps):
-                rep.step(directions=dirs)
-            e1.record(rep.stream)
+                one_pass()
+            e1.record(st)
             torch.cuda.synchronize()
-            ms = e0.elapsed_time(e1) / reps
+            ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / reps
             gbs = rep.w.n_layers * rep.payload_per_layer / (ms * 1e-3) / 1e9
             res[name + "_gbs"] = round(gbs, 1)
             res[name + "_us_per_layer"] = round(ms * 1e3 / rep.w.n_layers, 1)

@@ -1502,8 +1502,11 @@ def leg_prefix_sweep(args, local_rank):
 def run_length_sweep(args):
     """The same sweep on its own, all eight lengths, against the HBM or the pinned-host store."""
     rank, local_rank, world = init_dist("nccl")
-    rows = sweep_rows(args, local_rank, (1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072),
-                      host_store=args.sweep_host, n_layers=args.layers or 32)
+    lengths = (1024, 2048, 4096, 8192, 16384, 32768, 65536, 131072)
+    if args.sweep_tokens:
+        lengths = tuple(int(t) for t in args.sweep_tokens.split(","))
+    rows = sweep_rows(args, local_rank, lengths, host_store=args.sweep_host,
+                      n_layers=args.layers or 32)
     if rank == 0:
         print(json.dumps({"sweep": "raw restore/save bandwidth vs prefix length, 1 request, "
                           "8 KV heads x 128 x bf16, block 16, 32 layers",
@@ -1608,6 +1611,7 @@ def main():
     ap.add_argument("--gemm-iters", type=int, default=20)
     ap.add_argument("--sweep-length", action="store_true",
                     help="raw restore/save bandwidth against prefix length (1K..128K tokens)")
+    ap.add_argument("--sweep-tokens", default="", help="comma-separated prefix lengths for --sweep-length")
     ap.add_argument("--sweep-host", action="store_true", help="sweep against the pinned-host store")
     ap.add_argument("--sched-demo", action="store_true",
                     help="layer-wise pipelining under the slack-aware scheduler")

@@ -599,13 +599,16 @@ static void drain_cq(tutti_ring *r) {
     }
 }
 
-int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns) {
+// `waited_ns`: how long the caller has been waiting already (a range poll waits for its IOCBs
+// one after the other; the busy phase is counted over the whole call, not per IOCB)
+static int poll_one(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns,
+                    uint64_t waited_ns) {
     if (!r || !out) return TUTTI_EINVAL;
     r->host_calls++;
     if (!r->host->is_live(iocb_idx)) return TUTTI_EINVAL;
     const uint32_t slot = iocb_idx & (r->dev.depth - 1);
     auto t0 = std::chrono::steady_clock::now();
-    for (uint32_t spins = 0;; ++spins) {
+    for (;;) {
         if (!r->have_cqe[slot]) drain_cq(r);
         if (r->have_cqe[slot]) {
             *out = r->completed[slot];
@@ -616,18 +619,26 @@ int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64
         auto dt = std::chrono::duration_cast<std::chrono::nanoseconds>(
                       std::chrono::steady_clock::now() - t0).count();
         if ((uint64_t)dt >= timeout_ns) return TUTTI_EAGAIN;
-        // a short busy phase for completions that are microseconds away, then the core is
-        // given back between looks at the queue
-        if (dt < 50000) {
+        // a busy phase for completions that are less than a millisecond away (a sleep, however
+        // short, returns some 50 us late: more than a short pass takes), then the core is given
+        // back between looks at the queue, for about 1/128 of the time waited so far
+        if ((uint64_t)dt + waited_ns < 1000000) {
 #if defined(__x86_64__) || defined(__i386__)
             __builtin_ia32_pause();
 #else
             std::this_thread::yield();
 #endif
         } else {
-            std::this_thread::sleep_for(std::chrono::microseconds(spins < 4096 ? 5 : 50));
+            long long nap_us = (long long)(((uint64_t)dt + waited_ns) / 128000);
+            if (nap_us < 5) nap_us = 5;
+            if (nap_us > 100) nap_us = 100;
+            std::this_thread::sleep_for(std::chrono::microseconds(nap_us));
         }
     }
+}
+
+int tutti_ring_poll(tutti_ring_t *r, uint32_t iocb_idx, tutti_cqe_t *out, uint64_t timeout_ns) {
+    return poll_one(r, iocb_idx, out, timeout_ns, 0);
 }
 
 int tutti_ring_poll_range(tutti_ring_t *r, uint32_t first_iocb, uint32_t n_iocb, uint64_t *bytes_total,
@@ -639,14 +650,15 @@ int tutti_ring_poll_range(tutti_ring_t *r, uint32_t first_iocb, uint32_t n_iocb,
     int rc = TUTTI_OK;
     auto t0 = std::chrono::steady_clock::now();
     for (; done < n_iocb; ++done) {
-        uint64_t left = 0;
+        uint64_t left = 0, waited = 0;
         if (timeout_ns) {
             auto dt = std::chrono::duration_cast<std::chrono::nanoseconds>(
                           std::chrono::steady_clock::now() - t0).count();
-            left = (uint64_t)dt < timeout_ns ? timeout_ns - (uint64_t)dt : 1;
+            waited = (uint64_t)dt;
+            left = waited < timeout_ns ? timeout_ns - waited : 1;
         }
         tutti_cqe_t c;
-        rc = tutti_ring_poll(r, first_iocb + done, &c, left);
+        rc = poll_one(r, first_iocb + done, &c, left, waited);
         if (rc != TUTTI_OK) break;
         bytes += c.bytes;
         if (c.status != 0 && err == 0) err = c.status;

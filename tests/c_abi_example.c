@@ -129,6 +129,32 @@ int main(void)
         }
     if (bad) { fprintf(stderr, "save mismatch: %llu tokens\n", (unsigned long long)bad); return 1; }
 
+    /* the same restore as a staged transfer: the contexts are copied as they are into a staging
+     * buffer (here device to device; the copy engines' job when the store is pinned host
+     * memory), the kernel scatters from there into the pool */
+    CU(cudaMemcpy(d_store, h_store, lo.dev_bytes, cudaMemcpyHostToDevice));
+    CU(cudaMemset(d_pool, 0xA5, pool_bytes));
+    batch.plan_epoch = 1;
+    uint32_t n_ctx = 0, n_staged = 0;
+    uint64_t stage_bytes = 0;
+    CHECK(tutti_stage_plan(ctx, ring, &batch, 0, stream, &n_ctx, &n_staged, &stage_bytes));
+    if (n_ctx == 0 || n_staged != n_ctx || stage_bytes != 2ull * n_tok * lo.token_bytes) {
+        fprintf(stderr, "stage plan: %u contexts, %u staged, %llu bytes\n", n_ctx, n_staged,
+                (unsigned long long)stage_bytes);
+        return 1;
+    }
+    uint8_t *d_stage;
+    CU(cudaMalloc((void **)&d_stage, stage_bytes));
+    CHECK(tutti_stage_copy_layer(ctx, ring, layer, TUTTI_OP_READ, d_stage, stage_bytes, stream));
+    CHECK(tutti_build_sqes_staged(ctx, ring, &batch, layer, TUTTI_OP_READ, d_stage, stage_bytes, stream,
+                                  &first, &n));
+    CHECK(tutti_kv_restore_layer(ctx, ring, first, n, 0, stream));
+    CHECK(tutti_ring_poll_range(ring, first, n, &moved, &first_error, &n_done, 5000000000ull));
+    if (first_error != 0 || n_done != n || moved != stage_bytes) { fprintf(stderr, "staged restore status %d\n", first_error); return 1; }
+    uint8_t *h_pool2 = (uint8_t *)malloc(pool_bytes);
+    CU(cudaMemcpy(h_pool2, d_pool, pool_bytes, cudaMemcpyDeviceToHost));
+    if (memcmp(h_pool2, h_pool, pool_bytes) != 0) { fprintf(stderr, "staged restore differs from the direct one\n"); return 1; }
+
     uint64_t launches, calls;
     tutti_ring_stats(ring, &launches, &calls);
     printf("OK restored and saved %llu bytes; %llu kernel launches, %llu host calls\n",
